@@ -1,0 +1,418 @@
+#!/usr/bin/env python
+"""Benchmark of the batched CartPole step on B200: env-steps/s of the fused rollout
+(headline), the fused per-step kernel and the unfused per-op ladder, each with its
+roofline fraction, plus the CPU oracle timed on the host cores as a baseline.
+
+    python bench.py --gpus 1 --steps 20 --warmup 3
+    python -m torch.distributed.run --nnodes=1 --nproc-per-node N ... bench.py --gpus N ...
+    python bench.py --impl reference      # the scalar CPU oracle on the same workload
+
+One "step" is one pass of the whole hot path over one batch: one fused-rollout launch
+covering every environment and all T time steps of the workload (action, dynamics,
+termination, reward, restart for every env-step). Inputs are synthetic and fully
+defined by (n_envs, T, seed): start states and actions are a counter hash evaluated
+inside the kernels, so there is nothing to stage in HBM for the headline path.
+Rank 0 prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "env_steps_per_sec"
+UNIT = "env-steps/s"
+SMS = 148
+# Algorithmic thread-level operations per env-step of each rollout variant (see the design doc,
+# "Rollout kernel: operation count") and algorithmic HBM bytes per env-step of the step paths.
+ALG_OPS = {"random": 150.0, "linear": 152.0, "mlp": 540.0}
+STEP_BYTES = 37.0      # 16 in + 16 out + 4 reward + 1 done, hashed action
+LADDER_BYTES = 375.0   # sum over the 46 one-op kernels of their input and output planes
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "sm_max_mhz": float(p.get("sm_max_mhz", 1965.0)), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+# ------------------------------------------------------------------------------ reference arm
+def run_reference(args) -> None:
+    """The scalar CPU oracle, as it stands, on the headline workload's config. Each step is a
+    bounded sample (the first `sample_envs` environments for all T time steps)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import cartpole_oracle as oracle
+    from paper_2301_13062_b200 import inputs
+    w = inputs.WORKLOADS[args.workload]
+    cores = min(host_cores(), 256)
+    weights = inputs.policy_weights(w.policy, w.policy_seed) if w.policy else None
+    sample = min(w.n_envs, 1 << 17)
+    for _ in range(args.warmup):
+        oracle.rollout(sample, w.T, w.seed, w.policy, weights, per_env=True, nthreads=cores)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.rollout(sample, w.T, w.seed, w.policy, weights, per_env=True, nthreads=cores)
+    dt = time.perf_counter() - t0
+    value = sample * w.T * args.steps / dt
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{w.name}: {w.n_envs} envs x {w.T} steps, fused rollout, policy={w.policy}",
+                   "sample": f"first {sample} envs x {w.T} steps per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"first {sample} envs x {w.T} steps, {args.steps} repeats"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------ our arm
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3", help="headline rollout workload (c1, c3, c4, c5, paper)")
+    ap.add_argument("--no-paths", action="store_true", help="skip the ladder / fused-step / other-config lines")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    ap.add_argument("--step-envs", type=int, default=1 << 24, help="batch of the HBM-bound fused-step measurement")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_2301_13062_b200 import binding as cp
+    from paper_2301_13062_b200 import inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    cp.lib()
+    peaks = load_peaks()
+    peak_inst = SMS * 4 * 32 * peaks["sm_max_mhz"] * 1e6  # thread-instructions/s at the maximum SM clock
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t[0])
+
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")  # > 126 MB L2
+
+    def timed(fn, steps, warmup, flush=True):
+        """Sum of per-iteration CUDA-event times on the launching stream (ms), L2 flushed
+        between iterations outside the timed events; max over ranks."""
+        for _ in range(warmup):
+            fn()
+        barrier()
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        launches0 = cp.cp_launch_count()
+        for a, b in evs:
+            if flush:
+                flush_buf.fill_(1)
+            a.record()
+            fn()
+            b.record()
+        barrier()
+        launches = cp.cp_launch_count() - launches0
+        ms = sum(a.elapsed_time(b) for a, b in evs)
+        return max_over_ranks(ms), launches
+
+    # ---- headline: fused rollout ----
+    w = inputs.WORKLOADS[args.workload]
+    pol_name = {0: "random", 1: "linear", 2: "mlp"}[w.policy]
+    weights = inputs.policy_weights(w.policy, w.policy_seed) if w.policy else None
+    pol = cp.policy(w.policy, weights) if w.policy else None
+    n, T = w.n_envs, w.T
+    env_offset = rank * n  # weak scaling: every rank runs a full batch on its own env range
+    ret = torch.empty(n, dtype=torch.float32, device="cuda")
+    cnt = torch.empty(n, dtype=torch.int32, device="cuda")
+    tot = torch.zeros(2, dtype=torch.int64, device="cuda")
+    outs = {"ep_return_sum": ret, "ep_count": cnt, "totals": tot}
+    if w.streams:
+        outs["reward_stream"] = torch.empty(T, n, dtype=torch.float32, device="cuda")
+        outs["done_bits"] = torch.empty(T, (n + 31) // 32, dtype=torch.int32, device="cuda")
+
+    def rollout_step():
+        cp.cp_rollout_shard(env_offset, n, T, w.seed, pol, **outs)
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ms, launches = timed(rollout_step, args.steps, args.warmup)
+    clocks = sampler.stop() if rank == 0 else {}
+    ms_per_step = ms / args.steps
+    value = world * n * T / (ms_per_step * 1e-3)
+    ops = ALG_OPS[pol_name]
+    ach = n * T * ops / (ms_per_step * 1e-3)
+    roofline = {"bound": "alu", "kernel": "rollout_kernel", "achieved": ach / 1e12, "peak": peak_inst / 1e12,
+                "unit": "Tinst/s", "frac": ach / peak_inst, "traffic": None,
+                "algorithmic_ops_per_env_step": ops,
+                "peak_source": f"148 SMs x 4 schedulers x 32 lanes x {peaks['sm_max_mhz']:.0f} MHz ({peaks['source']} max clock)"}
+    if w.streams:
+        roofline["stream_write_gbs"] = n * T * 4.125 / (ms_per_step * 1e-3) / 1e9
+        roofline["stream_write_frac_of_hbm"] = roofline["stream_write_gbs"] / peaks["hbm_gbs"]
+
+    # ---- end to end through the C ABI with host buffers ----
+    h_ret = torch.empty(n, dtype=torch.float32).pin_memory()
+    h_cnt = torch.empty(n, dtype=torch.int32).pin_memory()
+    h_tot = torch.empty(2, dtype=torch.int64).pin_memory()
+
+    def e2e_step():
+        cp.cp_rollout_host(n, T, w.seed, pol, h_ret, h_cnt, h_tot)
+
+    e2e_ms, _ = timed(e2e_step, max(3, args.steps // 2), 3)
+    e2e_ms /= max(3, args.steps // 2)
+    e2e = {"value": world * n * T / (e2e_ms * 1e-3), "unit": UNIT,
+           "h2d_bytes_per_step": int(4 * inputs.N_WEIGHTS[w.policy]) + 24, "d2h_bytes_per_step": 8 * n + 16,
+           "ms_per_step": e2e_ms,
+           "note": "cp_rollout_host: host scalars (n_envs, T, seed) and policy weights in, per-env returns and "
+                   "counts copied to pinned host memory, stream synchronised, every step"}
+
+    paths = {}
+    if not args.no_paths and rank == 0:
+        paths = measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args)
+
+    cpu = None
+    if not args.no_cpu and rank == 0:
+        from oracle import cartpole_oracle as oracle
+        cores = min(host_cores(), 256)
+        sample = min(n, 1 << 20)
+        t0 = time.perf_counter()
+        o = oracle.rollout(sample, T, w.seed, w.policy, weights, nthreads=cores)
+        dt = time.perf_counter() - t0
+        same = float((o["ep_return_sum"] == ret[:sample].cpu().numpy()).mean()) if env_offset == 0 else None
+        cpu = {"value": sample * T / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"first {sample} envs x {T} steps of the workload, one pass, {dt:.2f} s",
+               "returns_identical_to_gpu": same}
+
+    if world > 1:
+        dist.all_reduce(tot)  # the only exchange the path has: 16 bytes, outside the timed region
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"{w.name}: {n} envs x {T} steps per GPU, fused rollout, policy={pol_name}, "
+                                   f"seed={w.seed}" + (", reward+done streams" if w.streams else ""),
+                       "l2": "flushed between iterations (256 MiB fill outside the timed events)",
+                       "envs_per_gpu": n, "T": T},
+            "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "roofline": roofline,
+            "cpu_baseline": cpu, "paths": paths,
+            "paper_context": {"hardware": "RTX 2080 Ti, 2048 envs x 10000 steps", "eager_vs_baseline": 0.13,
+                              "fused_step_vs_baseline": 3.41, "unroll10_vs_fused_step": 3.5,
+                              "hand_cuda_vs_best_xla": 2.7},
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args) -> dict:
+    """Ladder, fused step and the other rollout configurations (rank 0, one GPU each)."""
+    out = {}
+    hbm = peaks["hbm_gbs"] * 1e9
+
+    def step_setup(n):
+        stride = (n + 3) // 4 * 4
+        a = torch.zeros(4, stride, device="cuda")
+        b = torch.zeros(4, stride, device="cuda")
+        sa, sb = cp.cp_wrap(a, n, 0), cp.cp_wrap(b, n, 0)
+        cp.cp_fill_start(sa)
+        reward = torch.empty(n, device="cuda")
+        done = torch.empty(n, dtype=torch.uint8, device="cuda")
+        return a, b, sa, sb, reward, done
+
+    # fused step, HBM-bound size: ping-pong between two batches
+    n = args.step_envs
+    a, b, sa, sb, reward, done = step_setup(n)
+    for _ in range(40):  # reach the steady-state mix of restarts
+        cp.cp_step(sa, None, sb, reward, done)
+        cp.cp_step(sb, None, sa, reward, done)
+    state = {"flip": False}
+
+    def fused_step():
+        if state["flip"]:
+            cp.cp_step(sb, None, sa, reward, done)
+        else:
+            cp.cp_step(sa, None, sb, reward, done)
+        state["flip"] = not state["flip"]
+
+    ms, _ = timed(fused_step, 20, 4)
+    ms /= 20
+    gbs = n * STEP_BYTES / (ms * 1e-3) / 1e9
+    out["fused_step_hbm"] = {"n_envs": n, "ms_per_launch": ms, "env_steps_per_sec": n / (ms * 1e-3),
+                             "roofline": {"bound": "hbm", "kernel": "step_kernel", "achieved": gbs,
+                                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs * 1e9 / hbm,
+                                          "traffic": None, "bytes_per_env_step": STEP_BYTES}}
+    # ladder at the same size
+    ws = torch.empty(cp.cp_unfused_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+
+    def ladder_step():
+        cp.cp_set_time(sa, 41)
+        cp.cp_step_unfused(sa, None, sb, reward, done, ws)
+
+    ms, launches = timed(ladder_step, 5, 3)
+    ms /= 5
+    gbs = n * LADDER_BYTES / (ms * 1e-3) / 1e9
+    out["ladder_hbm"] = {"n_envs": n, "ms_per_step": ms, "launches_per_step": launches // 5,
+                         "env_steps_per_sec": n / (ms * 1e-3),
+                         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                      "frac": gbs * 1e9 / hbm, "bytes_per_env_step": LADDER_BYTES}}
+    del a, b, sa, sb, reward, done, ws
+    torch.cuda.empty_cache()
+
+    # config 2: 65,536 envs, per-step launches (launch-bound), 1,000 steps per timed iteration
+    w2 = inputs.WORKLOADS["c2"]
+    n = w2.n_envs
+    a, b, sa, sb, reward, done = step_setup(n)
+    ws = torch.empty(cp.cp_unfused_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+
+    def c2_fused():
+        cp.cp_set_time(sa, 0)
+        for _ in range(w2.T):
+            cp.cp_step(sa, None, sa, reward, done)
+
+    def c2_ladder():
+        cp.cp_set_time(sa, 0)
+        for _ in range(50):
+            cp.cp_step_unfused(sa, None, sb, reward, done, ws)
+            cp.cp_step_unfused(sb, None, sa, reward, done, ws)
+
+    ms, _ = timed(c2_fused, 3, 3, flush=False)
+    ms /= 3
+    out["c2_fused_step"] = {"n_envs": n, "T": w2.T, "ms_total": ms, "us_per_launch": 1e3 * ms / w2.T,
+                            "env_steps_per_sec": n * w2.T / (ms * 1e-3), "note": "launch-bound: 2.4 MB per launch"}
+    ms, _ = timed(c2_ladder, 3, 3, flush=False)
+    ms /= 3
+    out["c2_ladder"] = {"n_envs": n, "T": 100, "ms_total": ms, "us_per_step": 1e3 * ms / 100,
+                        "env_steps_per_sec": n * 100 / (ms * 1e-3), "launches_per_step": 46}
+    out["ratios"] = {"fused_step_over_ladder_c2": out["c2_fused_step"]["env_steps_per_sec"] / out["c2_ladder"]["env_steps_per_sec"],
+                     "fused_step_over_ladder_hbm": out["fused_step_hbm"]["env_steps_per_sec"] / out["ladder_hbm"]["env_steps_per_sec"]}
+    del a, b, sa, sb, reward, done, ws
+
+    # the other rollout configurations
+    for name in ("c1", "c3", "c4", "c5", "paper"):
+        w = inputs.WORKLOADS[name]
+        if name == args.workload:
+            continue
+        weights = inputs.policy_weights(w.policy, w.policy_seed) if w.policy else None
+        pol = cp.policy(w.policy, weights) if w.policy else None
+        n, T = w.n_envs, w.T
+        outs = {"ep_return_sum": torch.empty(n, device="cuda"), "ep_count": torch.empty(n, dtype=torch.int32, device="cuda"),
+                "totals": torch.zeros(2, dtype=torch.int64, device="cuda")}
+        if w.streams:
+            outs["reward_stream"] = torch.empty(T, n, dtype=torch.float32, device="cuda")
+            outs["done_bits"] = torch.empty(T, (n + 31) // 32, dtype=torch.int32, device="cuda")
+
+        def fn():
+            cp.cp_rollout(n, T, w.seed, pol, **outs)
+
+        k = 5 if n * T > 1e9 else 10
+        ms, _ = timed(fn, k, 3)
+        ms /= k
+        pol_name = {0: "random", 1: "linear", 2: "mlp"}[w.policy]
+        rate = n * T / (ms * 1e-3)
+        entry = {"n_envs": n, "T": T, "policy": pol_name, "ms_per_launch": ms, "env_steps_per_sec": rate,
+                 "alu_frac": rate * ALG_OPS[pol_name] / peak_inst}
+        if w.streams:
+            entry["stream_write_gbs"] = rate * 4.125 / 1e9
+            entry["stream_write_frac_of_hbm"] = rate * 4.125 / hbm
+        out[f"{name}_rollout"] = entry
+        del outs
+        torch.cuda.empty_cache()
+    if "fused_step_hbm" in out and args.workload == "c3":
+        pass
+    return out
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,214 @@
+/*
+ * cartpole.h — C ABI of libcartpole.so: the batched CartPole environment step on
+ * one NVIDIA B200 (sm_100a), in three execution strategies.
+ *
+ * The computation is the "environment update function" of the paper "Operator
+ * Fusion in XLA: Analysis and Evaluation" (Sec. IV, Case Study on Cart-pole):
+ * a chain of elementwise float32 operations over N independent environments —
+ * force from the action, sin/cos of the pole angle, the shared `temp` term,
+ * angular and linear acceleration, four explicit-Euler updates, termination
+ * test, reward, and reset of finished environments — repeated for T steps with
+ * random actions and random start states (Sec. V, 2,048 envs x 10,000 steps).
+ * The three strategies are the rungs of the paper's fusion ladder:
+ *   cp_step_unfused  one kernel per elementwise op, every intermediate in HBM
+ *                    (the eager per-op execution of Sec. V-F);
+ *   cp_step          one fused kernel per step, state passed as four separate
+ *                    planes and kept in registers (Sec. V-C, "no concat");
+ *   cp_rollout       one kernel for all T steps, state in registers across
+ *                    steps (Sec. V-D loop unrolling taken to its limit, and the
+ *                    single-kernel CUDA comparison of Sec. V-G).
+ * Random numbers never need a kernel of their own (Sec. V-A): actions and start
+ * states are a stateless counter hash of (seed, env, step), defined below.
+ *
+ * Conventions
+ *   - Every pointer is marked DEVICE or HOST. Device buffers belong to the caller
+ *     unless stated; the library never frees or reallocates them.
+ *   - Calls enqueue work on the stream set with cp_set_stream (default: the legacy
+ *     default stream) and return without synchronising, unless stated.
+ *   - int functions return CP_OK or a negative code; cp_last_error() gives the text
+ *     for the calling thread. Nothing aborts, traps or throws.
+ *   - State layout: four float32 planes x | x_dot | theta | theta_dot; element i of
+ *     plane p is planes[p * plane_stride + i]. Vector (16-byte) access is used when
+ *     planes is 16-byte aligned and plane_stride is a multiple of 4; any other
+ *     layout takes a scalar path with identical results.
+ *   - Environment i of a batch has global id env_offset + i; all hashing uses the
+ *     global id, so results do not depend on how environments are sharded.
+ *
+ * Arithmetic (identical in all three strategies, bit for bit)
+ *   constants  g=9.8f m_pole=0.1f m_total=1.1f l=0.5f pml=0.05f F=10.0f tau=0.02f
+ *              ft=(float)(4/3) x_max=2.4f theta_max=(float)(12*2*pi/360)
+ *   force = a ? +F : -F;  s = sinf(theta); c = cosf(theta)
+ *   temp  = (force + (pml*(thd*thd))*s) / m_total
+ *   thacc = (g*s - c*temp) / (l*(ft - (m_pole*(c*c))/m_total))
+ *   xacc  = temp - ((pml*thacc)*c)/m_total
+ *   x' = x + tau*xd; xd' = xd + tau*xacc; th' = th + tau*thd; thd' = thd + tau*thacc
+ *   every operation rounded once to float32 (no fused multiply-add, IEEE division,
+ *   accurate sinf/cosf; no fast-math);
+ *   done = x'<-x_max | x'>x_max | th'<-theta_max | th'>theta_max  (strict, on the
+ *   updated state); reward = 1.0f for every step (each step starts from a live
+ *   state; the terminating step counts); a finished environment continues from a
+ *   fresh start state and reports done=1 for that step.
+ *
+ * Counter hash (uint32 arithmetic mod 2^32)
+ *   MA=0x6A09E667 MB=0xBB67AE85 MG=0x9E3779B1
+ *   mix32(h): h^=h>>16; h*=MA; h^=h>>15; h*=MB; h^=h>>16
+ *   salt(seed,stream) = mix32(mix32(seed^MG)+stream)         stream 0 actions, 1 starts
+ *   K0 = mix32(env ^ salt); K1 = mix32(K0+MG)
+ *   H(K,c): h=K0^c; h=(h^(h>>16))*MA+K1; h=(h^(h>>15))*MB; h^=h>>16
+ *   action(seed,env,t)   = H(K(stream 0), t) >> 31
+ *   start_j(seed,env,t)  = ((float)(H(K(stream 1), 4t+j)>>8) * 2^-24 - 0.5f) * 0.1f,
+ *                          j=0..3 -> x, x_dot, theta, theta_dot of an episode that
+ *                          begins at global time t (initial state: t of the reset;
+ *                          after done at step t: t+1). Needs 4*(t+1) < 2^32.
+ */
+#ifndef CARTPOLE_H_
+#define CARTPOLE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CP_OK 0
+#define CP_EINVAL (-1) /* bad argument: null/misaligned pointer, size out of range, unknown kind */
+#define CP_ECUDA (-2)  /* a CUDA runtime call failed; text in cp_last_error() */
+#define CP_ENOMEM (-3) /* allocation failed, or a caller-supplied workspace is too small */
+
+#define CP_POLICY_RANDOM 0 /* hashed Bernoulli(1/2) action */
+#define CP_POLICY_LINEAR 1 /* argmax(W obs + b), W 2x4 */
+#define CP_POLICY_MLP 2    /* argmax(W2 tanh(W1 obs + b1) + b2), 4 -> 16 -> 2 */
+#define CP_MLP_HIDDEN 16
+#define CP_MAX_T (1LL << 30)
+
+/* Opaque HOST handle of a batch: n_envs, plane_stride, seed, global step t,
+ * env_offset and the DEVICE address of the four state planes. */
+typedef struct cp_state cp_state;
+
+/* Policy evaluated inside the rollout kernel on the state BEFORE the step ("fusing
+ * simulation with neural network inference", the paper's future work, Sec. VI).
+ * weights is a HOST pointer, copied into the launch parameters by the call:
+ *   linear: W[2][4] row-major, b[2]                         (10 floats)
+ *   MLP:    W1[16][4], b1[16], W2[2][16], b2[2]             (114 floats)
+ * Each logit is a left-to-right chain acc = fmaf(w_i, v_i, acc) starting from the
+ * bias; hidden units use accurate tanhf; action = (logit[1] > logit[0]), so a tie
+ * pushes left. */
+typedef struct cp_policy {
+    int32_t kind;
+    const float *weights; /* HOST; NULL for CP_POLICY_RANDOM */
+} cp_policy;
+
+/* Outputs of a rollout; every pointer is DEVICE memory of the caller and may be
+ * NULL (not produced). Per-step planes are time-major so that a warp writes one
+ * contiguous 128-byte line per step. */
+typedef struct cp_returns {
+    float *ep_return_sum;  /* [n_envs] sum of the returns (= lengths) of episodes completed in the T steps */
+    uint32_t *ep_count;    /* [n_envs] number of completed episodes */
+    uint64_t *totals;      /* [2] += {sum of ep_return_sum, sum of ep_count}; caller zeroes before the call */
+    float *reward_stream;  /* [T][n_envs] reward of every step (1.0f) */
+    uint32_t *done_bits;   /* [T][ceil(n_envs/32)] bit (i%32) of word (i/32) = done of env i at that step */
+    uint32_t *action_bits; /* [T][ceil(n_envs/32)] same packing, the action taken */
+    float *final_state;    /* [4][n_envs] state after the last step */
+    float *trajectory;     /* [T][4][n_envs] state after every step, after any reset (validation aid) */
+} cp_returns;
+
+/* ---- the three calls of the hot path ------------------------------------------------ */
+
+/* Sec. V (random start states): allocate a batch of n_envs environments (cudaMalloc,
+ * planes padded to a multiple of 4 floats) and fill it with start states of global time 0.
+ * 1 <= n_envs, n_envs + env_offset(=0) <= 2^32. Returns NULL on error. Free with cp_free. */
+cp_state *cp_reset(int64_t n_envs, uint32_t seed);
+
+/* Sec. IV / Sec. V-C: one fused step of every environment, one kernel launch.
+ *   state      in: batch at global step t.
+ *   action     DEVICE [n_envs] bytes (non-zero = push right), or NULL = hashed action of step t.
+ *   out_state  out: same n_envs; may be `state` itself (in place). Receives t+1 (host side),
+ *              and seed / env_offset of `state`.
+ *   reward     DEVICE [n_envs] float32 or NULL.   done  DEVICE [n_envs] bytes (0/1) or NULL.
+ * Algorithmic HBM traffic: 16 B read + 16 B written per env, + 4 (reward) + 1 (done) [+ 1 action]. */
+int cp_step(cp_state *state, const uint8_t *action, cp_state *out_state, float *reward, uint8_t *done);
+
+/* Sec. V-D / V-G: T steps of n_envs environments in ONE kernel, state in registers for
+ * all T steps; starts from the start states of global time 0 (equal to cp_reset followed by
+ * T cp_step calls with action == NULL, bit for bit). 1 <= T <= CP_MAX_T.
+ * policy NULL or kind CP_POLICY_RANDOM = hashed actions. */
+int cp_rollout(int64_t n_envs, int64_t T, uint32_t seed, const cp_policy *policy, const cp_returns *returns);
+
+/* ---- helpers ------------------------------------------------------------------------- */
+
+/* Sec. V-F (eager per-op execution): the same step as cp_step computed by one kernel per
+ * elementwise operation (45 launches, 46 when the action is hashed), every intermediate a
+ * plane in `workspace` (DEVICE, 256-byte aligned, >= cp_unfused_workspace_bytes(n_envs)).
+ * Results equal cp_step bit for bit. Needs 16-byte aligned planes with plane_stride % 4 == 0.
+ * Unlike cp_step, out_state must not alias state. reward / done as in cp_step (non-NULL). */
+int cp_step_unfused(cp_state *state, const uint8_t *action, cp_state *out_state, float *reward,
+                    uint8_t *done, void *workspace, size_t workspace_bytes);
+size_t cp_unfused_workspace_bytes(int64_t n_envs);
+
+/* Wrap caller-owned DEVICE planes (for example a torch tensor) as a batch at global step t.
+ * plane_stride >= n_envs. The handle does not own the planes. NULL on error. */
+cp_state *cp_wrap(float *planes, int64_t n_envs, int64_t plane_stride, uint32_t seed, uint32_t t,
+                  uint32_t env_offset);
+/* Overwrite the planes with the start states of the batch's current global step t. */
+int cp_fill_start(cp_state *state);
+/* Set the batch's global step (host side only). */
+int cp_set_time(cp_state *state, uint32_t t);
+/* Release the handle (and the planes if cp_reset allocated them). NULL is allowed. */
+void cp_free(cp_state *state);
+/* Read the handle's fields; any out pointer may be NULL. planes is a DEVICE address. */
+int cp_state_info(const cp_state *state, int64_t *n_envs, int64_t *plane_stride, uint32_t *seed,
+                  uint32_t *t, uint32_t *env_offset, float **planes);
+
+/* Hashed actions of global step t for envs env_offset .. env_offset+n_envs-1 -> out DEVICE [n_envs]. */
+int cp_actions(int64_t n_envs, uint32_t seed, uint32_t t, uint32_t env_offset, uint8_t *out);
+
+/* cp_rollout for the env range [env_offset, env_offset + n_envs) of a larger job (one range
+ * per GPU; no exchange is needed besides adding the ranks' `totals`). */
+int cp_rollout_shard(uint32_t env_offset, int64_t n_envs, int64_t T, uint32_t seed,
+                     const cp_policy *policy, const cp_returns *returns);
+
+/* Sec. V-D (k steps per kernel, the knob between cp_step and cp_rollout): advance an existing
+ * batch by T steps in one launch, in place, from its current global step. ep_len DEVICE [n_envs]
+ * (or NULL = all episodes start now) carries the steps already taken in each running episode in
+ * and out, so that consecutive chunks give the same returns as one long rollout.
+ * returns->final_state is ignored (the batch itself is updated); state->t advances by T. */
+int cp_rollout_from(cp_state *state, int64_t T, uint32_t *ep_len, const cp_policy *policy,
+                    const cp_returns *returns);
+
+/* End-to-end forms with HOST buffers (pinned memory recommended): device staging buffers
+ * are owned by the library (grown on demand, released by cp_shutdown); the calls copy in,
+ * launch, copy out and SYNCHRONISE the stream before returning.
+ * cp_rollout_host: h_ep_return_sum [n_envs], h_ep_count [n_envs], h_totals [2] (overwritten). */
+int cp_rollout_host(int64_t n_envs, int64_t T, uint32_t seed, const cp_policy *policy,
+                    float *h_ep_return_sum, uint32_t *h_ep_count, uint64_t *h_totals);
+/* cp_step_host: h_planes_in/out [4][n_envs] (stride n_envs), h_action [n_envs] or NULL,
+ * h_reward [n_envs], h_done [n_envs]; the step at global time t of envs 0..n_envs-1. */
+int cp_step_host(int64_t n_envs, uint32_t seed, uint32_t t, const float *h_planes_in,
+                 const uint8_t *h_action, float *h_planes_out, float *h_reward, uint8_t *h_done);
+/* Free the library-owned staging buffers (synchronises the device). */
+void cp_shutdown(void);
+
+/* Stream used by this thread's later calls (a cudaStream_t; NULL = legacy default stream). */
+void cp_set_stream(void *cuda_stream);
+
+/* Launch tuning, process-wide. key: "rollout_block" (threads per CTA, multiple of 32),
+ * "rollout_ept" (environments per thread: 1, 2 or 4), "rollout_ctas_per_sm" (0 = from the
+ * occupancy calculator), "step_block". Returns CP_EINVAL for an unknown key or value. */
+int cp_tune(const char *key, int value);
+
+/* Number of kernels this library has launched in this process (all threads). */
+uint64_t cp_launch_count(void);
+
+/* Diagnostics: count float32 values v in [lo, hi] (bit patterns, both >= 0, lo <= hi, and their
+ * negatives) for which the fused kernels' sine/cosine differ in any bit from the ladder's
+ * separate sinf / cosf kernels. mismatches DEVICE [1] uint64, caller zeroes. */
+int cp_selftest_sincos(uint32_t lo_bits, uint32_t hi_bits, uint64_t *mismatches);
+
+const char *cp_last_error(void);
+const char *cp_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CARTPOLE_H_ */

@@ -1,0 +1,450 @@
+// extern "C" boundary of libcartpole: argument checking, handle bookkeeping,
+// stream selection and launch of the kernels. No arithmetic of the method lives
+// here except the two per-launch salts of the counter hash.
+#include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+
+#include "../../include/cartpole.h"
+#include "cartpole_device.cuh"
+#include "cartpole_internal.h"
+
+struct cp_state {
+    int64_t n;
+    int64_t stride;
+    uint32_t seed, t, env_offset;
+    float *planes;
+    bool owns;
+};
+
+namespace cp {
+
+LaunchTuning g_tuning;
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+int sm_count() {
+    static int cached = 0;
+    if (cached == 0) {
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+            cached = sms;
+        else
+            return 148;
+    }
+    return cached;
+}
+
+}  // namespace cp
+
+namespace {
+
+thread_local cudaStream_t tl_stream = nullptr;
+thread_local char tl_error[512] = "";
+
+int fail(int code, const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(tl_error, sizeof tl_error, fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+int cuda_fail(cudaError_t e, const char *what) {
+    return fail(CP_ECUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+inline bool is_aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+bool state_vec_ok(const cp_state *s) { return is_aligned(s->planes, 16) && (s->stride % 4) == 0; }
+
+int check_state(const cp_state *s, const char *name) {
+    if (!s) return fail(CP_EINVAL, "%s is NULL", name);
+    if (!s->planes || s->n <= 0 || s->stride < s->n) return fail(CP_EINVAL, "%s is not a valid batch", name);
+    return CP_OK;
+}
+
+int check_policy(const cp_policy *policy, int *kind) {
+    *kind = policy ? policy->kind : CP_POLICY_RANDOM;
+    if (*kind < CP_POLICY_RANDOM || *kind > CP_POLICY_MLP) return fail(CP_EINVAL, "unknown policy kind %d", *kind);
+    if (*kind != CP_POLICY_RANDOM && !policy->weights) return fail(CP_EINVAL, "policy weights are NULL");
+    return CP_OK;
+}
+
+int check_range(int64_t n_envs, uint32_t env_offset) {
+    if (n_envs <= 0) return fail(CP_EINVAL, "n_envs must be positive (got %lld)", (long long)n_envs);
+    if ((uint64_t)n_envs + env_offset > (1ull << 32))
+        return fail(CP_EINVAL, "env_offset + n_envs exceeds 2^32 environment ids");
+    return CP_OK;
+}
+
+void fill_step_params(cp::StepParams &p, const cp_state *in, cp_state *out, const uint8_t *action, float *reward,
+                      uint8_t *done) {
+    p.in = in->planes;
+    p.in_stride = in->stride;
+    p.out = out->planes;
+    p.out_stride = out->stride;
+    p.n = in->n;
+    p.t = in->t;
+    p.env_offset = in->env_offset;
+    p.salt_a = cp::salt(in->seed, 0u);
+    p.salt_r = cp::salt(in->seed, 1u);
+    p.action = action;
+    p.reward = reward;
+    p.done = done;
+}
+
+int check_step_args(cp_state *state, cp_state *out_state) {
+    int rc;
+    if ((rc = check_state(state, "state")) != CP_OK) return rc;
+    if ((rc = check_state(out_state, "out_state")) != CP_OK) return rc;
+    if (out_state->n != state->n) return fail(CP_EINVAL, "out_state has %lld envs, state has %lld",
+                                              (long long)out_state->n, (long long)state->n);
+    if (state->t >= (1u << 30)) return fail(CP_EINVAL, "global step out of range");
+    return CP_OK;
+}
+
+void advance(cp_state *state, cp_state *out_state, uint32_t steps) {
+    out_state->seed = state->seed;
+    out_state->env_offset = state->env_offset;
+    out_state->t = state->t + steps;
+}
+
+// Rollout shared by cp_rollout / cp_rollout_shard / cp_rollout_from / cp_rollout_host.
+int rollout_impl(uint32_t env_offset, int64_t n_envs, int64_t T, uint32_t seed, uint32_t t0, const cp_policy *policy,
+                 const cp_returns *ret, const float *init_planes, int64_t init_stride, float *out_planes,
+                 int64_t out_stride, uint32_t *ep_len) {
+    int kind, rc;
+    if ((rc = check_range(n_envs, env_offset)) != CP_OK) return rc;
+    if (T <= 0 || T > CP_MAX_T || (int64_t)t0 + T > CP_MAX_T)
+        return fail(CP_EINVAL, "T must be in [1, 2^30] and t0 + T <= 2^30 (got T=%lld, t0=%u)", (long long)T, t0);
+    if ((rc = check_policy(policy, &kind)) != CP_OK) return rc;
+    if (!ret) return fail(CP_EINVAL, "returns is NULL");
+    if (ret->totals && !is_aligned(ret->totals, 8)) return fail(CP_EINVAL, "totals must be 8-byte aligned");
+    cp::RolloutParams p;
+    memset(&p, 0, sizeof p);
+    p.n = n_envs;
+    p.T = (uint32_t)T;
+    p.t0 = t0;
+    p.env_offset = env_offset;
+    p.salt_a = cp::salt(seed, 0u);
+    p.salt_r = cp::salt(seed, 1u);
+    p.init_planes = init_planes;
+    p.init_stride = init_stride;
+    p.out_planes = out_planes;
+    p.out_stride = out_stride;
+    p.ep_len_io = ep_len;
+    p.ep_return_sum = ret->ep_return_sum;
+    p.ep_count = ret->ep_count;
+    p.totals = reinterpret_cast<unsigned long long *>(ret->totals);
+    p.reward_stream = ret->reward_stream;
+    p.done_bits = ret->done_bits;
+    p.action_bits = ret->action_bits;
+    p.trajectory = ret->trajectory;
+    if (kind == CP_POLICY_LINEAR) memcpy(p.w, policy->weights, 10 * sizeof(float));
+    if (kind == CP_POLICY_MLP) memcpy(p.w, policy->weights, 114 * sizeof(float));
+    const bool streams = p.reward_stream || p.done_bits || p.action_bits || p.trajectory;
+    cudaError_t e = cp::launch_rollout(p, kind, streams, tl_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "rollout launch");
+    return CP_OK;
+}
+
+// Library-owned device staging for the HOST-buffer entry points.
+struct Staging {
+    std::mutex mu;
+    void *buf = nullptr;
+    size_t bytes = 0;
+} g_staging;
+
+int staging_reserve(size_t bytes, void **out) {
+    if (g_staging.bytes < bytes) {
+        if (g_staging.buf) {
+            cudaError_t e = cudaFree(g_staging.buf);
+            g_staging.buf = nullptr;
+            g_staging.bytes = 0;
+            if (e != cudaSuccess) return cuda_fail(e, "cudaFree(staging)");
+        }
+        cudaError_t e = cudaMalloc(&g_staging.buf, bytes);
+        if (e != cudaSuccess) {
+            g_staging.buf = nullptr;
+            (void)cudaGetLastError();
+            return fail(CP_ENOMEM, "cudaMalloc(%zu) for staging failed: %s", bytes, cudaGetErrorString(e));
+        }
+        g_staging.bytes = bytes;
+    }
+    *out = g_staging.buf;
+    return CP_OK;
+}
+
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+extern "C" {
+
+cp_state *cp_reset(int64_t n_envs, uint32_t seed) {
+    if (check_range(n_envs, 0) != CP_OK) return nullptr;
+    cp_state *s = new (std::nothrow) cp_state;
+    if (!s) {
+        fail(CP_ENOMEM, "out of host memory");
+        return nullptr;
+    }
+    s->n = n_envs;
+    s->stride = (n_envs + 3) / 4 * 4;
+    s->seed = seed;
+    s->t = 0;
+    s->env_offset = 0;
+    s->owns = true;
+    s->planes = nullptr;
+    cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&s->planes), (size_t)s->stride * 4 * sizeof(float));
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        fail(CP_ENOMEM, "cudaMalloc of %lld envs failed: %s", (long long)n_envs, cudaGetErrorString(e));
+        delete s;
+        return nullptr;
+    }
+    // pad lanes hold start states too, so vector loads never see uninitialised memory
+    e = cp::launch_fill_start(s->planes, s->stride, s->stride, 0, cp::salt(seed, 1u), 0, tl_stream);
+    if (e != cudaSuccess) {
+        cuda_fail(e, "start-state launch");
+        cudaFree(s->planes);
+        delete s;
+        return nullptr;
+    }
+    return s;
+}
+
+cp_state *cp_wrap(float *planes, int64_t n_envs, int64_t plane_stride, uint32_t seed, uint32_t t,
+                  uint32_t env_offset) {
+    if (!planes || !is_aligned(planes, 4)) {
+        fail(CP_EINVAL, "planes is NULL or not float-aligned");
+        return nullptr;
+    }
+    if (check_range(n_envs, env_offset) != CP_OK) return nullptr;
+    if (plane_stride < n_envs) {
+        fail(CP_EINVAL, "plane_stride %lld < n_envs %lld", (long long)plane_stride, (long long)n_envs);
+        return nullptr;
+    }
+    if (t > (1u << 30)) {
+        fail(CP_EINVAL, "global step out of range");
+        return nullptr;
+    }
+    cp_state *s = new (std::nothrow) cp_state;
+    if (!s) {
+        fail(CP_ENOMEM, "out of host memory");
+        return nullptr;
+    }
+    *s = cp_state{n_envs, plane_stride, seed, t, env_offset, planes, false};
+    return s;
+}
+
+int cp_fill_start(cp_state *state) {
+    int rc = check_state(state, "state");
+    if (rc != CP_OK) return rc;
+    cudaError_t e = cp::launch_fill_start(state->planes, state->stride, state->n, state->env_offset,
+                                          cp::salt(state->seed, 1u), state->t, tl_stream);
+    return e == cudaSuccess ? CP_OK : cuda_fail(e, "start-state launch");
+}
+
+int cp_set_time(cp_state *state, uint32_t t) {
+    if (!state) return fail(CP_EINVAL, "state is NULL");
+    if (t > (1u << 30)) return fail(CP_EINVAL, "global step out of range");
+    state->t = t;
+    return CP_OK;
+}
+
+void cp_free(cp_state *state) {
+    if (!state) return;
+    if (state->owns && state->planes) cudaFree(state->planes);
+    delete state;
+}
+
+int cp_state_info(const cp_state *state, int64_t *n_envs, int64_t *plane_stride, uint32_t *seed, uint32_t *t,
+                  uint32_t *env_offset, float **planes) {
+    if (!state) return fail(CP_EINVAL, "state is NULL");
+    if (n_envs) *n_envs = state->n;
+    if (plane_stride) *plane_stride = state->stride;
+    if (seed) *seed = state->seed;
+    if (t) *t = state->t;
+    if (env_offset) *env_offset = state->env_offset;
+    if (planes) *planes = state->planes;
+    return CP_OK;
+}
+
+int cp_step(cp_state *state, const uint8_t *action, cp_state *out_state, float *reward, uint8_t *done) {
+    int rc = check_step_args(state, out_state);
+    if (rc != CP_OK) return rc;
+    if (reward && !is_aligned(reward, 4)) return fail(CP_EINVAL, "reward is not float-aligned");
+    cp::StepParams p;
+    fill_step_params(p, state, out_state, action, reward, done);
+    const bool vec = state_vec_ok(state) && state_vec_ok(out_state) && (!reward || is_aligned(reward, 16)) &&
+                     (!done || is_aligned(done, 4)) && (!action || is_aligned(action, 4));
+    cudaError_t e = cp::launch_step(p, vec, tl_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "step launch");
+    advance(state, out_state, 1);
+    return CP_OK;
+}
+
+size_t cp_unfused_workspace_bytes(int64_t n_envs) {
+    return n_envs > 0 ? cp::ladder_workspace_bytes(n_envs) : 0;
+}
+
+int cp_step_unfused(cp_state *state, const uint8_t *action, cp_state *out_state, float *reward, uint8_t *done,
+                    void *workspace, size_t workspace_bytes) {
+    int rc = check_step_args(state, out_state);
+    if (rc != CP_OK) return rc;
+    if (!reward || !done) return fail(CP_EINVAL, "reward and done must not be NULL for the unfused step");
+    if (!is_aligned(reward, 4)) return fail(CP_EINVAL, "reward is not float-aligned");
+    if (!state_vec_ok(state) || !state_vec_ok(out_state))
+        return fail(CP_EINVAL, "the unfused step needs 16-byte aligned planes with plane_stride %% 4 == 0");
+    if (state->planes == out_state->planes) return fail(CP_EINVAL, "the unfused step cannot run in place");
+    if (!workspace || !is_aligned(workspace, 256)) return fail(CP_EINVAL, "workspace is NULL or not 256-byte aligned");
+    if (workspace_bytes < cp::ladder_workspace_bytes(state->n))
+        return fail(CP_ENOMEM, "workspace has %zu bytes, %zu needed", workspace_bytes,
+                    cp::ladder_workspace_bytes(state->n));
+    cp::StepParams p;
+    fill_step_params(p, state, out_state, action, reward, done);
+    cudaError_t e = cp::launch_ladder(p, workspace, tl_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "ladder launch");
+    advance(state, out_state, 1);
+    return CP_OK;
+}
+
+int cp_actions(int64_t n_envs, uint32_t seed, uint32_t t, uint32_t env_offset, uint8_t *out) {
+    int rc = check_range(n_envs, env_offset);
+    if (rc != CP_OK) return rc;
+    if (!out) return fail(CP_EINVAL, "out is NULL");
+    cudaError_t e = cp::launch_actions(out, n_envs, env_offset, cp::salt(seed, 0u), t, tl_stream);
+    return e == cudaSuccess ? CP_OK : cuda_fail(e, "actions launch");
+}
+
+int cp_rollout(int64_t n_envs, int64_t T, uint32_t seed, const cp_policy *policy, const cp_returns *returns) {
+    return cp_rollout_shard(0, n_envs, T, seed, policy, returns);
+}
+
+int cp_rollout_shard(uint32_t env_offset, int64_t n_envs, int64_t T, uint32_t seed, const cp_policy *policy,
+                     const cp_returns *returns) {
+    if (!returns) return fail(CP_EINVAL, "returns is NULL");
+    return rollout_impl(env_offset, n_envs, T, seed, 0, policy, returns, nullptr, 0, returns->final_state, n_envs,
+                        nullptr);
+}
+
+int cp_rollout_from(cp_state *state, int64_t T, uint32_t *ep_len, const cp_policy *policy,
+                    const cp_returns *returns) {
+    int rc = check_state(state, "state");
+    if (rc != CP_OK) return rc;
+    rc = rollout_impl(state->env_offset, state->n, T, state->seed, state->t, policy, returns, state->planes,
+                      state->stride, state->planes, state->stride, ep_len);
+    if (rc != CP_OK) return rc;
+    state->t += (uint32_t)T;
+    return CP_OK;
+}
+
+int cp_rollout_host(int64_t n_envs, int64_t T, uint32_t seed, const cp_policy *policy, float *h_ep_return_sum,
+                    uint32_t *h_ep_count, uint64_t *h_totals) {
+    int rc = check_range(n_envs, 0);
+    if (rc != CP_OK) return rc;
+    if (!h_ep_return_sum || !h_ep_count || !h_totals) return fail(CP_EINVAL, "a host output pointer is NULL");
+    std::lock_guard<std::mutex> lock(g_staging.mu);
+    const size_t per = round_up((size_t)n_envs * 4, 256);
+    void *buf;
+    if ((rc = staging_reserve(2 * per + 256, &buf)) != CP_OK) return rc;
+    char *base = static_cast<char *>(buf);
+    cp_returns r;
+    memset(&r, 0, sizeof r);
+    r.ep_return_sum = reinterpret_cast<float *>(base);
+    r.ep_count = reinterpret_cast<uint32_t *>(base + per);
+    r.totals = reinterpret_cast<uint64_t *>(base + 2 * per);
+    cudaError_t e = cudaMemsetAsync(r.totals, 0, 16, tl_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+    if ((rc = rollout_impl(0, n_envs, T, seed, 0, policy, &r, nullptr, 0, nullptr, 0, nullptr)) != CP_OK) return rc;
+    e = cudaMemcpyAsync(h_ep_return_sum, r.ep_return_sum, (size_t)n_envs * 4, cudaMemcpyDeviceToHost, tl_stream);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(h_ep_count, r.ep_count, (size_t)n_envs * 4, cudaMemcpyDeviceToHost, tl_stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h_totals, r.totals, 16, cudaMemcpyDeviceToHost, tl_stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(tl_stream);
+    return e == cudaSuccess ? CP_OK : cuda_fail(e, "rollout copy-out");
+}
+
+int cp_step_host(int64_t n_envs, uint32_t seed, uint32_t t, const float *h_planes_in, const uint8_t *h_action,
+                 float *h_planes_out, float *h_reward, uint8_t *h_done) {
+    int rc = check_range(n_envs, 0);
+    if (rc != CP_OK) return rc;
+    if (!h_planes_in || !h_planes_out || !h_reward || !h_done) return fail(CP_EINVAL, "a host pointer is NULL");
+    if (t >= (1u << 30)) return fail(CP_EINVAL, "global step out of range");
+    std::lock_guard<std::mutex> lock(g_staging.mu);
+    const int64_t stride = (n_envs + 63) / 64 * 64;
+    const size_t plane_bytes = (size_t)stride * 4;
+    const size_t byte_plane = round_up((size_t)n_envs, 256);
+    void *buf;
+    if ((rc = staging_reserve(5 * plane_bytes + 2 * byte_plane, &buf)) != CP_OK) return rc;
+    char *base = static_cast<char *>(buf);
+    float *d_planes = reinterpret_cast<float *>(base);
+    float *d_reward = reinterpret_cast<float *>(base + 4 * plane_bytes);
+    uint8_t *d_done = reinterpret_cast<uint8_t *>(base + 5 * plane_bytes);
+    uint8_t *d_action = d_done + byte_plane;
+    cudaError_t e = cudaMemcpy2DAsync(d_planes, plane_bytes, h_planes_in, (size_t)n_envs * 4, (size_t)n_envs * 4, 4,
+                                      cudaMemcpyHostToDevice, tl_stream);
+    if (e == cudaSuccess && h_action)
+        e = cudaMemcpyAsync(d_action, h_action, (size_t)n_envs, cudaMemcpyHostToDevice, tl_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "step copy-in");
+    cp_state s{n_envs, stride, seed, t, 0, d_planes, false};
+    if ((rc = cp_step(&s, h_action ? d_action : nullptr, &s, d_reward, d_done)) != CP_OK) return rc;
+    e = cudaMemcpy2DAsync(h_planes_out, (size_t)n_envs * 4, d_planes, plane_bytes, (size_t)n_envs * 4, 4,
+                          cudaMemcpyDeviceToHost, tl_stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h_reward, d_reward, (size_t)n_envs * 4, cudaMemcpyDeviceToHost, tl_stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h_done, d_done, (size_t)n_envs, cudaMemcpyDeviceToHost, tl_stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(tl_stream);
+    return e == cudaSuccess ? CP_OK : cuda_fail(e, "step copy-out");
+}
+
+void cp_shutdown(void) {
+    std::lock_guard<std::mutex> lock(g_staging.mu);
+    if (g_staging.buf) {
+        cudaDeviceSynchronize();
+        cudaFree(g_staging.buf);
+        g_staging.buf = nullptr;
+        g_staging.bytes = 0;
+    }
+}
+
+void cp_set_stream(void *cuda_stream) { tl_stream = static_cast<cudaStream_t>(cuda_stream); }
+
+int cp_tune(const char *key, int value) {
+    if (!key) return fail(CP_EINVAL, "key is NULL");
+    if (!strcmp(key, "rollout_block")) {
+        if (value < 32 || value > 256 || value % 32) return fail(CP_EINVAL, "rollout_block must be 32..256, multiple of 32");
+        cp::g_tuning.rollout_block = value;
+    } else if (!strcmp(key, "rollout_ept")) {
+        if (value != 0 && value != 1 && value != 2 && value != 4) return fail(CP_EINVAL, "rollout_ept must be 0, 1, 2 or 4");
+        cp::g_tuning.rollout_ept = value;
+    } else if (!strcmp(key, "rollout_ctas_per_sm")) {
+        if (value < 0 || value > 32) return fail(CP_EINVAL, "rollout_ctas_per_sm must be 0..32");
+        cp::g_tuning.rollout_ctas_per_sm = value;
+    } else if (!strcmp(key, "step_block")) {
+        if (value < 32 || value > 256 || value % 32) return fail(CP_EINVAL, "step_block must be 32..256, multiple of 32");
+        cp::g_tuning.step_block = value;
+    } else {
+        return fail(CP_EINVAL, "unknown tuning key '%s'", key);
+    }
+    return CP_OK;
+}
+
+uint64_t cp_launch_count(void) { return cp::g_launches.load(std::memory_order_relaxed); }
+
+int cp_selftest_sincos(uint32_t lo_bits, uint32_t hi_bits, uint64_t *mismatches) {
+    if (!mismatches || !is_aligned(mismatches, 8)) return fail(CP_EINVAL, "mismatches is NULL or misaligned");
+    if (lo_bits > hi_bits || hi_bits >= 0x7F800000u) return fail(CP_EINVAL, "need lo <= hi, both finite and non-negative");
+    cudaError_t e = cp::launch_sincos_selftest(lo_bits, hi_bits, reinterpret_cast<unsigned long long *>(mismatches),
+                                               tl_stream);
+    return e == cudaSuccess ? CP_OK : cuda_fail(e, "self-test launch");
+}
+
+const char *cp_last_error(void) { return tl_error; }
+const char *cp_version(void) { return "cartpole-b200 0.1 (sm_100a)"; }
+
+}  // extern "C"

@@ -1,0 +1,68 @@
+// Host-side declarations shared by the .cu files of libcartpole (not installed).
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace cp {
+
+// Parameters of one fused step launch.
+struct StepParams {
+    const float *in;
+    int64_t in_stride;
+    float *out;
+    int64_t out_stride;
+    int64_t n;
+    uint32_t t, env_offset, salt_a, salt_r;
+    const uint8_t *action;  // or nullptr: hashed
+    float *reward;          // or nullptr
+    uint8_t *done;          // or nullptr
+};
+
+// Parameters of one rollout launch. Weights travel in the launch parameters
+// (constant bank), so every policy FMA reads its weight as an immediate operand.
+struct RolloutParams {
+    int64_t n;
+    int64_t n_tasks;  // warp tasks of 32*EPT envs
+    uint32_t T, t0, env_offset, salt_a, salt_r;
+    const float *init_planes;  // nullptr: start states of time t0
+    int64_t init_stride;
+    float *out_planes;  // nullptr: final state not stored
+    int64_t out_stride;
+    uint32_t *ep_len_io;
+    float *ep_return_sum;
+    uint32_t *ep_count;
+    unsigned long long *totals;
+    float *reward_stream;
+    uint32_t *done_bits;
+    uint32_t *action_bits;
+    float *trajectory;
+    float w[114];
+};
+
+struct LaunchTuning {
+    int rollout_block = 256;
+    int rollout_ept = 0;          // 0: chosen per policy
+    int rollout_ctas_per_sm = 0;  // 0: occupancy calculator
+    int step_block = 256;
+};
+extern LaunchTuning g_tuning;
+
+void count_launch(int n = 1);
+int sm_count();
+
+cudaError_t launch_step(const StepParams &p, bool vec, cudaStream_t s);
+cudaError_t launch_fill_start(float *planes, int64_t stride, int64_t n, uint32_t env_offset, uint32_t salt_r,
+                              uint32_t t, cudaStream_t s);
+cudaError_t launch_actions(uint8_t *out, int64_t n, uint32_t env_offset, uint32_t salt_a, uint32_t t,
+                           cudaStream_t s);
+cudaError_t launch_rollout(RolloutParams &p, int policy, bool streams, cudaStream_t s);
+cudaError_t launch_sincos_selftest(uint32_t lo_bits, uint32_t hi_bits, unsigned long long *mismatches,
+                                   cudaStream_t s);
+
+// The per-op ladder. Workspace layout is private to ladder_kernels.cu.
+size_t ladder_workspace_bytes(int64_t n);
+int ladder_launch_count(bool hashed_action);
+cudaError_t launch_ladder(const StepParams &p, void *workspace, cudaStream_t s);
+
+}  // namespace cp

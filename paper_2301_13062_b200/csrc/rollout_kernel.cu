@@ -1,0 +1,178 @@
+// Fused multi-step rollout: one launch runs all T steps (paper Sec. V-D, loop
+// unrolling, taken to its limit, and the single-kernel CUDA comparison of
+// Sec. V-G). Each environment's state, hash keys and episode counters stay in
+// registers for the whole time loop; HBM sees 8 bytes per environment in total
+// unless per-step streams are requested.
+//
+// Work decomposition: a "warp task" is 32*EPT consecutive environments; lane l
+// owns environments base + j*32 + l (j < EPT), so that per-step stream stores
+// are one contiguous 128-byte line per j and a done/action bitmask word is one
+// warp ballot. Tasks are dealt round-robin to the resident warps (persistent
+// grid, sized from the occupancy calculator times the SM count).
+//
+// The kernel has no shared memory, no inter-warp synchronisation and no waits.
+#include "cartpole_device.cuh"
+#include "cartpole_internal.h"
+
+namespace cp {
+
+template <int POLICY>
+__device__ __forceinline__ uint32_t policy_signbit(const RolloutParams &p, const Keys &ka, uint32_t t,
+                                                   const State &z) {
+    if (POLICY == 0) {
+        return action_signbit(ka, t);
+    } else if (POLICY == 1) {
+        return linear_action(*reinterpret_cast<const LinearW *>(p.w), z);
+    } else {
+        return mlp_action(*reinterpret_cast<const MlpW *>(p.w), z);
+    }
+}
+
+template <int POLICY, int EPT, bool STREAMS>
+__global__ void __launch_bounds__(256) rollout_kernel(const __grid_constant__ RolloutParams p) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const int64_t warps_total = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int64_t words = (p.n + 31) >> 5;
+    unsigned long long tot_ret = 0, tot_cnt = 0;
+
+    for (int64_t task = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); task < p.n_tasks;
+         task += warps_total) {
+        const int64_t base = task * (32 * EPT);
+        State z[EPT];
+        Keys ka[EPT], kr[EPT];
+        uint32_t ep_len[EPT], ret[EPT], cnt[EPT];
+        int64_t idx[EPT];
+        bool valid[EPT];
+#pragma unroll
+        for (int j = 0; j < EPT; ++j) {
+            idx[j] = base + j * 32 + lane;
+            valid[j] = idx[j] < p.n;
+            if (!valid[j]) idx[j] = p.n - 1;  // idle lanes shadow the last environment and store nothing
+            const uint32_t env = p.env_offset + (uint32_t)idx[j];
+            if (POLICY == 0) ka[j] = make_keys(p.salt_a, env);
+            kr[j] = make_keys(p.salt_r, env);
+            if (p.init_planes) {
+                z[j].x = p.init_planes[idx[j]];
+                z[j].xd = p.init_planes[p.init_stride + idx[j]];
+                z[j].th = p.init_planes[2 * p.init_stride + idx[j]];
+                z[j].thd = p.init_planes[3 * p.init_stride + idx[j]];
+            } else {
+                z[j] = start_state(kr[j], p.t0);
+            }
+            ep_len[j] = p.ep_len_io ? p.ep_len_io[idx[j]] : 0u;
+            ret[j] = 0u;
+            cnt[j] = 0u;
+        }
+
+        for (uint32_t k = 0; k < p.T; ++k) {
+            const uint32_t t = p.t0 + k;
+#pragma unroll
+            for (int j = 0; j < EPT; ++j) {
+                const uint32_t sb = policy_signbit<POLICY>(p, ka[j], t, z[j]);
+                const bool done = euler_step(z[j], force_from_signbit(sb));
+                ep_len[j] += 1u;  // reward 1 per step, the terminating step included
+                if (done) {
+                    ret[j] += ep_len[j];
+                    cnt[j] += 1u;
+                    ep_len[j] = 0u;
+                    z[j] = start_state(kr[j], t + 1u);
+                }
+                if (STREAMS) {
+                    const int64_t word = task * EPT + j;
+                    if (p.done_bits) {
+                        const uint32_t m = __ballot_sync(0xffffffffu, done && valid[j]);
+                        if (lane == 0 && word < words) p.done_bits[(int64_t)k * words + word] = m;
+                    }
+                    if (p.action_bits) {
+                        const uint32_t m = __ballot_sync(0xffffffffu, (sb != 0u) && valid[j]);
+                        if (lane == 0 && word < words) p.action_bits[(int64_t)k * words + word] = m;
+                    }
+                    if (valid[j]) {
+                        if (p.reward_stream) p.reward_stream[(int64_t)k * p.n + idx[j]] = 1.0f;
+                        if (p.trajectory) {
+                            float *tr = p.trajectory + (int64_t)k * 4 * p.n + idx[j];
+                            tr[0] = z[j].x;
+                            tr[p.n] = z[j].xd;
+                            tr[2 * p.n] = z[j].th;
+                            tr[3 * p.n] = z[j].thd;
+                        }
+                    }
+                }
+            }
+        }
+
+#pragma unroll
+        for (int j = 0; j < EPT; ++j) {
+            if (!valid[j]) continue;
+            if (p.ep_return_sum) p.ep_return_sum[idx[j]] = (float)ret[j];
+            if (p.ep_count) p.ep_count[idx[j]] = cnt[j];
+            if (p.ep_len_io) p.ep_len_io[idx[j]] = ep_len[j];
+            if (p.out_planes) {
+                p.out_planes[idx[j]] = z[j].x;
+                p.out_planes[p.out_stride + idx[j]] = z[j].xd;
+                p.out_planes[2 * p.out_stride + idx[j]] = z[j].th;
+                p.out_planes[3 * p.out_stride + idx[j]] = z[j].thd;
+            }
+            tot_ret += ret[j];
+            tot_cnt += cnt[j];
+        }
+    }
+
+    if (p.totals) {
+        for (int o = 16; o > 0; o >>= 1) {
+            tot_ret += __shfl_down_sync(0xffffffffu, tot_ret, o);
+            tot_cnt += __shfl_down_sync(0xffffffffu, tot_cnt, o);
+        }
+        if (lane == 0 && (tot_ret | tot_cnt)) {
+            atomicAdd(p.totals, tot_ret);
+            atomicAdd(p.totals + 1, tot_cnt);
+        }
+    }
+}
+
+namespace {
+
+template <int POLICY, int EPT, bool STREAMS>
+cudaError_t launch_one(RolloutParams &p, cudaStream_t s) {
+    const int block = g_tuning.rollout_block;
+    p.n_tasks = (p.n + 32 * EPT - 1) / (32 * EPT);
+    int per_sm = g_tuning.rollout_ctas_per_sm;
+    if (per_sm <= 0) {
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rollout_kernel<POLICY, EPT, STREAMS>,
+                                                                      block, 0);
+        if (e != cudaSuccess) return e;
+        if (per_sm < 1) per_sm = 1;
+    }
+    const int wpb = block / 32;
+    int64_t grid = (p.n_tasks + wpb - 1) / wpb;
+    const int64_t resident = (int64_t)per_sm * sm_count();
+    if (grid > resident) grid = resident;
+    rollout_kernel<POLICY, EPT, STREAMS><<<(unsigned)grid, block, 0, s>>>(p);
+    count_launch();
+    return cudaGetLastError();
+}
+
+template <int POLICY, bool STREAMS>
+cudaError_t launch_ept(RolloutParams &p, int ept, cudaStream_t s) {
+    switch (ept) {
+        case 1: return launch_one<POLICY, 1, STREAMS>(p, s);
+        case 2: return launch_one<POLICY, 2, STREAMS>(p, s);
+        default: return launch_one<POLICY, 4, STREAMS>(p, s);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_rollout(RolloutParams &p, int policy, bool streams, cudaStream_t s) {
+    int ept = g_tuning.rollout_ept;
+    if (ept == 0) ept = 2;
+    // Small batches: spread environments over as many warps as possible.
+    while (ept > 1 && (p.n + 32 * ept - 1) / (32 * ept) < (int64_t)sm_count() * 16) ept >>= 1;
+    switch (policy) {
+        case 0: return streams ? launch_ept<0, true>(p, ept, s) : launch_ept<0, false>(p, ept, s);
+        case 1: return streams ? launch_ept<1, true>(p, ept, s) : launch_ept<1, false>(p, ept, s);
+        default: return streams ? launch_ept<2, true>(p, ept, s) : launch_ept<2, false>(p, ept, s);
+    }
+}
+
+}  // namespace cp

@@ -1,0 +1,173 @@
+// Fused single-step kernel (paper Sec. V-C: the four state values travel as
+// separate planes and the whole update is one kernel with the state in
+// registers), plus the small generator kernels (start states, hashed actions)
+// and the sine/cosine self-test.
+//
+// HBM traffic per env-step: 16 B state in + 16 B state out + 4 B reward + 1 B
+// done (+ 1 B action when supplied). Vector form: each thread owns 4 consecutive
+// environments, i.e. one float4 per plane, so a warp moves 512 B per plane per
+// access and keeps 4 x 16 B loads in flight per thread.
+#include "cartpole_device.cuh"
+#include "cartpole_internal.h"
+
+namespace cp {
+
+// One environment: action -> dynamics -> done -> start state of the next episode.
+__device__ __forceinline__ bool step_one(State &z, uint32_t env, const StepParams &p, bool has_action,
+                                         uint8_t a_in) {
+    uint32_t sb;
+    if (has_action) {
+        sb = a_in ? 0x80000000u : 0u;
+    } else {
+        sb = action_signbit(make_keys(p.salt_a, env), p.t);
+    }
+    return euler_step(z, force_from_signbit(sb));
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(256) step_kernel(const __grid_constant__ StepParams p) {
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool has_action = p.action != nullptr;
+    if (VEC) {
+        const int64_t i0 = tid * 4;
+        if (i0 >= p.n) return;
+        const float4 vx = *reinterpret_cast<const float4 *>(p.in + i0);
+        const float4 vxd = *reinterpret_cast<const float4 *>(p.in + p.in_stride + i0);
+        const float4 vth = *reinterpret_cast<const float4 *>(p.in + 2 * p.in_stride + i0);
+        const float4 vthd = *reinterpret_cast<const float4 *>(p.in + 3 * p.in_stride + i0);
+        State z[4] = {{vx.x, vxd.x, vth.x, vthd.x},
+                      {vx.y, vxd.y, vth.y, vthd.y},
+                      {vx.z, vxd.z, vth.z, vthd.z},
+                      {vx.w, vxd.w, vth.w, vthd.w}};
+        const bool full = i0 + 3 < p.n;
+        uint8_t a_in[4] = {0, 0, 0, 0};
+        if (has_action) {
+            if (full) {
+                uchar4 av = *reinterpret_cast<const uchar4 *>(p.action + i0);
+                a_in[0] = av.x; a_in[1] = av.y; a_in[2] = av.z; a_in[3] = av.w;
+            } else {
+                for (int j = 0; j < 4; ++j)
+                    if (i0 + j < p.n) a_in[j] = p.action[i0 + j];
+            }
+        }
+        const uint32_t env0 = p.env_offset + (uint32_t)i0;
+        uint32_t dmask = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            dmask |= (step_one(z[j], env0 + j, p, has_action, a_in[j]) ? 1u : 0u) << j;
+        // Restart finished environments one per pass: almost always at most one of a
+        // thread's four environments finishes in a step, so the start-state hashes are
+        // issued once per warp instead of once per environment slot.
+        uint32_t pending = dmask;
+        while (pending) {
+            const int j = __ffs(pending) - 1;
+            pending &= pending - 1;
+            const State r = start_state(make_keys(p.salt_r, env0 + j), p.t + 1u);
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (q == j) z[q] = r;
+        }
+        *reinterpret_cast<float4 *>(p.out + i0) = make_float4(z[0].x, z[1].x, z[2].x, z[3].x);
+        *reinterpret_cast<float4 *>(p.out + p.out_stride + i0) = make_float4(z[0].xd, z[1].xd, z[2].xd, z[3].xd);
+        *reinterpret_cast<float4 *>(p.out + 2 * p.out_stride + i0) = make_float4(z[0].th, z[1].th, z[2].th, z[3].th);
+        *reinterpret_cast<float4 *>(p.out + 3 * p.out_stride + i0) = make_float4(z[0].thd, z[1].thd, z[2].thd, z[3].thd);
+        if (full) {
+            if (p.reward) *reinterpret_cast<float4 *>(p.reward + i0) = make_float4(1.0f, 1.0f, 1.0f, 1.0f);
+            if (p.done)
+                *reinterpret_cast<uchar4 *>(p.done + i0) =
+                    make_uchar4(dmask & 1u, (dmask >> 1) & 1u, (dmask >> 2) & 1u, (dmask >> 3) & 1u);
+        } else {
+            for (int j = 0; j < 4; ++j)
+                if (i0 + j < p.n) {
+                    if (p.reward) p.reward[i0 + j] = 1.0f;
+                    if (p.done) p.done[i0 + j] = (dmask >> j) & 1u;
+                }
+        }
+    } else {
+        const int64_t i = tid;
+        if (i >= p.n) return;
+        State z = {p.in[i], p.in[p.in_stride + i], p.in[2 * p.in_stride + i], p.in[3 * p.in_stride + i]};
+        const uint32_t env = p.env_offset + (uint32_t)i;
+        const bool d = step_one(z, env, p, has_action, has_action ? p.action[i] : (uint8_t)0);
+        if (d) z = start_state(make_keys(p.salt_r, env), p.t + 1u);
+        p.out[i] = z.x;
+        p.out[p.out_stride + i] = z.xd;
+        p.out[2 * p.out_stride + i] = z.th;
+        p.out[3 * p.out_stride + i] = z.thd;
+        if (p.reward) p.reward[i] = 1.0f;
+        if (p.done) p.done[i] = d ? 1 : 0;
+    }
+}
+
+cudaError_t launch_step(const StepParams &p, bool vec, cudaStream_t s) {
+    const int block = g_tuning.step_block;
+    if (vec) {
+        const int64_t threads = (p.n + 3) / 4;
+        const int64_t grid = (threads + block - 1) / block;
+        step_kernel<true><<<(unsigned)grid, block, 0, s>>>(p);
+    } else {
+        const int64_t grid = (p.n + block - 1) / block;
+        step_kernel<false><<<(unsigned)grid, block, 0, s>>>(p);
+    }
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ---- generators ----
+__global__ void fill_start_kernel(float *planes, int64_t stride, int64_t n, uint32_t env_offset, uint32_t salt_r,
+                                  uint32_t t) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const State z = start_state(make_keys(salt_r, env_offset + (uint32_t)i), t);
+    planes[i] = z.x;
+    planes[stride + i] = z.xd;
+    planes[2 * stride + i] = z.th;
+    planes[3 * stride + i] = z.thd;
+}
+
+cudaError_t launch_fill_start(float *planes, int64_t stride, int64_t n, uint32_t env_offset, uint32_t salt_r,
+                              uint32_t t, cudaStream_t s) {
+    const int block = 256;
+    fill_start_kernel<<<(unsigned)((n + block - 1) / block), block, 0, s>>>(planes, stride, n, env_offset, salt_r, t);
+    count_launch();
+    return cudaGetLastError();
+}
+
+__global__ void actions_kernel(uint8_t *out, int64_t n, uint32_t env_offset, uint32_t salt_a, uint32_t t) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    out[i] = (uint8_t)(step_hash(make_keys(salt_a, env_offset + (uint32_t)i), t) >> 31);
+}
+
+cudaError_t launch_actions(uint8_t *out, int64_t n, uint32_t env_offset, uint32_t salt_a, uint32_t t,
+                           cudaStream_t s) {
+    const int block = 256;
+    actions_kernel<<<(unsigned)((n + block - 1) / block), block, 0, s>>>(out, n, env_offset, salt_a, t);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ---- self-test: fused sine/cosine vs separate sinf and cosf ----
+__global__ void sincos_selftest_kernel(uint32_t lo, uint32_t hi, unsigned long long *mismatches) {
+    unsigned long long bad = 0;
+    const uint64_t span = (uint64_t)hi - lo + 1;
+    for (uint64_t k = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; k < span; k += (uint64_t)gridDim.x * blockDim.x) {
+        const float v = __uint_as_float(lo + (uint32_t)k);
+        float s, c;
+        sin_cos(v, s, c);
+        bad += (__float_as_uint(s) != __float_as_uint(sinf(v))) | (__float_as_uint(c) != __float_as_uint(cosf(v)));
+        sin_cos(-v, s, c);
+        bad += (__float_as_uint(s) != __float_as_uint(sinf(-v))) | (__float_as_uint(c) != __float_as_uint(cosf(-v)));
+    }
+    for (int o = 16; o > 0; o >>= 1) bad += __shfl_down_sync(0xffffffffu, bad, o);
+    if ((threadIdx.x & 31) == 0 && bad) atomicAdd(mismatches, bad);
+}
+
+cudaError_t launch_sincos_selftest(uint32_t lo_bits, uint32_t hi_bits, unsigned long long *mismatches,
+                                   cudaStream_t s) {
+    sincos_selftest_kernel<<<sm_count() * 8, 256, 0, s>>>(lo_bits, hi_bits, mismatches);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace cp

@@ -1,0 +1,423 @@
+"""GPU parity tests: the CUDA library (through its C ABI) against the CPU oracle,
+element by element on the same seeded inputs, plus GPU-internal identities
+(ladder == fused step == rollout, bit for bit)."""
+import numpy as np
+import pytest
+
+from paper_2301_13062_b200 import inputs
+from tests import gpu_helpers as H
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def cp():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2301_13062_b200 import binding
+    binding.lib()  # raises if the library is missing: there is no fallback
+    torch.cuda.set_device(0)
+    return binding
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def host(t):
+    return t.cpu().numpy()
+
+
+def alloc_planes(n, stride=None):
+    stride = stride or (n + 3) // 4 * 4
+    return torch.zeros(4, stride, dtype=torch.float32, device="cuda")
+
+
+def gpu_step(cp, z, seed, t, action=None, env_offset=0, stride=None, in_place=False, unfused=False):
+    n = z.shape[1]
+    pin = alloc_planes(n, stride)
+    pin[:, :n] = dev(z)
+    pout = pin if in_place else alloc_planes(n, stride)
+    s_in = cp.cp_wrap(pin, n, seed, t, env_offset)
+    s_out = s_in if in_place else cp.cp_wrap(pout, n, seed, 0, 0)
+    reward = torch.full((n,), -7.0, dtype=torch.float32, device="cuda")
+    done = torch.full((n,), 9, dtype=torch.uint8, device="cuda")
+    act = dev(action) if action is not None else None
+    if unfused:
+        ws = torch.empty(cp.cp_unfused_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+        cp.cp_step_unfused(s_in, act, s_out, reward, done, ws)
+    else:
+        cp.cp_step(s_in, act, s_out, reward, done)
+    torch.cuda.synchronize()
+    info = s_out.info()
+    assert info["t"] == t + 1 and info["seed"] == seed and info["env_offset"] == env_offset
+    return host(pout[:, :n]), host(reward), host(done)
+
+
+# ------------------------------------------------------------------ generators
+@pytest.mark.parametrize("n,off,t", [(1, 0, 0), (33, 0, 0), (1025, 7, 22), (70001, 1 << 20, 499)])
+def test_start_states_and_actions_bit_exact(cp, oracle, n, off, t):
+    planes = alloc_planes(n)
+    st = cp.cp_wrap(planes, n, seed=3, t=t, env_offset=off)
+    cp.cp_fill_start(st)
+    a = torch.empty(n, dtype=torch.uint8, device="cuda")
+    cp.cp_actions(n, 3, t, off, a)
+    torch.cuda.synchronize()
+    got = host(planes[:, :n])
+    m = min(n, 3000)
+    want = oracle.initial_state(m, 3, t, off)
+    assert np.array_equal(got[:, :m].view(np.uint32), want.view(np.uint32))
+    r = oracle.step(got, seed=3, t=t, env_offset=off)
+    assert np.array_equal(host(a), r["action"])
+
+
+def test_reset_allocates_and_fills(cp, oracle):
+    n = 1000
+    st = cp.cp_reset(n, 5)
+    info = st.info()
+    assert info["n_envs"] == n and info["plane_stride"] % 4 == 0 and info["t"] == 0
+    planes = alloc_planes(n)
+    out = cp.cp_wrap(planes, n, 5)
+    reward = torch.empty(n, dtype=torch.float32, device="cuda")
+    done = torch.empty(n, dtype=torch.uint8, device="cuda")
+    cp.cp_step(st, None, out, reward, done)
+    torch.cuda.synchronize()
+    z0 = oracle.initial_state(n, 5)
+    want = oracle.step(z0, seed=5, t=0, want_pre_reset=True)
+    H.assert_step_matches(want, z0, host(planes[:, :n]), host(reward), host(done))
+    assert out.info()["t"] == 1
+    cp.cp_free(st)
+
+
+# ------------------------------------------------------------------ single step vs oracle
+@pytest.mark.parametrize("spread", ["start", "live", "edge", "wide"])
+@pytest.mark.parametrize("n", [1, 3, 5, 33, 1025, 65537])
+def test_step_matches_oracle(cp, oracle, spread, n):
+    z = inputs.random_states(n, seed=n + len(spread), spread=spread)
+    for action, off, t in ((None, 0, 0), (None, 12345, 17), (inputs.random_actions(n, 3), 0, 5)):
+        want = oracle.step(z, seed=1, t=t, action_u8=action, env_offset=off, want_pre_reset=True)
+        got_state, got_reward, got_done = gpu_step(cp, z, 1, t, action, off)
+        stats = H.assert_step_matches(want, z, got_state, got_reward, got_done)
+        if spread in ("start", "live") and n >= 1025:
+            assert stats["bit_exact_fraction"] > 0.9
+
+
+def test_step_scalar_path_and_in_place_equal_vector_path(cp):
+    n = 4099
+    z = inputs.random_states(n, seed=2, spread="edge")
+    a = inputs.random_actions(n, 9)
+    base = gpu_step(cp, z, 4, 3, None, 100)
+    for kwargs in ({"stride": n}, {"stride": n + 1}, {"in_place": True}, {"stride": n, "in_place": True}):
+        other = gpu_step(cp, z, 4, 3, None, 100, **kwargs)
+        for b, o in zip(base, other):
+            assert np.array_equal(b.view(np.uint8), o.view(np.uint8)), kwargs
+    base = gpu_step(cp, z, 4, 3, a, 100)
+    other = gpu_step(cp, z, 4, 3, a, 100, stride=n)
+    for b, o in zip(base, other):
+        assert np.array_equal(b.view(np.uint8), o.view(np.uint8))
+
+
+def test_step_optional_outputs_and_misaligned_buffers(cp):
+    n = 1000
+    z = inputs.random_states(n, seed=3, spread="edge")
+    want = gpu_step(cp, z, 0, 0)
+    pin = alloc_planes(n)
+    pin[:, :n] = dev(z)
+    s = cp.cp_wrap(pin, n, 0, 0)
+    pout = alloc_planes(n)
+    o = cp.cp_wrap(pout, n, 0)
+    cp.cp_step(s, None, o, None, None)  # reward/done not wanted
+    torch.cuda.synchronize()
+    assert np.array_equal(host(pout[:, :n]), want[0])
+    # reward/done at odd offsets: scalar path, same bits
+    rbuf = torch.zeros(n + 1, dtype=torch.float32, device="cuda")
+    dbuf = torch.zeros(n + 1, dtype=torch.uint8, device="cuda")
+    cp.cp_set_time(s, 0)
+    cp.cp_step(s, None, o, rbuf[1:], dbuf[1:])
+    torch.cuda.synchronize()
+    assert np.array_equal(host(pout[:, :n]), want[0])
+    assert np.array_equal(host(rbuf[1:]), want[1]) and np.array_equal(host(dbuf[1:]), want[2])
+    assert float(rbuf[0]) == 0 and int(dbuf[0]) == 0
+
+
+def test_mirror_antisymmetry_on_gpu(cp):
+    n = 50000
+    z = inputs.random_states(n, seed=6, spread="edge")
+    a = inputs.random_actions(n, 6)
+    pin, pout = alloc_planes(n), alloc_planes(n)
+    res = []
+    for zz, aa in ((z, a), (-z, (1 - a).astype(np.uint8))):
+        pin[:, :n] = dev(zz)
+        s, o = cp.cp_wrap(pin, n, 0, 0), cp.cp_wrap(pout, n, 0)
+        done = torch.empty(n, dtype=torch.uint8, device="cuda")
+        cp.cp_step(s, dev(aa), o, None, done)
+        torch.cuda.synchronize()
+        res.append((host(pout[:, :n]), host(done)))
+    live = res[0][1] == 0
+    assert np.array_equal(res[0][1], res[1][1])
+    assert np.array_equal(-res[0][0][:, live], res[1][0][:, live])
+
+
+def test_nan_inf_states_do_not_fault(cp):
+    n = 64
+    z = inputs.random_states(n, seed=1, spread="live")
+    z[0, 0] = np.nan
+    z[2, 1] = np.nan
+    z[0, 2] = np.inf
+    z[3, 3] = -np.inf
+    state, reward, done = gpu_step(cp, z, 0, 0)
+    assert done[0] == 0 and done[1] == 0 and done[2] == 1
+    assert np.isnan(state[0, 0]) and np.isnan(state[2, 1])
+    assert np.all(reward == 1.0)
+
+
+# ------------------------------------------------------------------ ladder == fused step
+@pytest.mark.parametrize("n", [1, 33, 1025, 50001])
+def test_ladder_equals_fused_step_bitwise(cp, n):
+    before = cp.cp_launch_count()
+    for spread in ("edge", "wide", "start"):
+        z = inputs.random_states(n, seed=n, spread=spread)
+        for action in (None, inputs.random_actions(n, 4)):
+            fused = gpu_step(cp, z, 7, 11, action, 5)
+            ladder = gpu_step(cp, z, 7, 11, action, 5, unfused=True)
+            for f, l in zip(fused, ladder):
+                assert np.array_equal(f.view(np.uint8), l.view(np.uint8))
+    # 3 spreads x (46 + 45 ladder launches + 2 fused launches)
+    assert cp.cp_launch_count() - before == 3 * (46 + 45 + 2)
+
+
+def test_ladder_argument_checks(cp):
+    n = 100
+    pin, pout = alloc_planes(n), alloc_planes(n)
+    s, o = cp.cp_wrap(pin, n, 0, 0), cp.cp_wrap(pout, n, 0)
+    r = torch.empty(n, dtype=torch.float32, device="cuda")
+    d = torch.empty(n, dtype=torch.uint8, device="cuda")
+    ws = torch.empty(cp.cp_unfused_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    with pytest.raises(cp.CartpoleError) as e:
+        cp.cp_step_unfused(s, None, s, r, d, ws)
+    assert e.value.code == cp.CP_EINVAL
+    with pytest.raises(cp.CartpoleError) as e:
+        cp.cp_step_unfused(s, None, o, r, d, ws[:1024])
+    assert e.value.code == cp.CP_ENOMEM
+    with pytest.raises(cp.CartpoleError):
+        cp.cp_step_unfused(s, None, o, r, d, ws[1:])
+    odd = cp.cp_wrap(torch.zeros(4, 101, device="cuda"), 100, 0, 0)
+    with pytest.raises(cp.CartpoleError):
+        cp.cp_step_unfused(odd, None, o, r, d, ws)
+
+
+# ------------------------------------------------------------------ rollout
+def run_rollout(cp, n, T, seed, kind=0, weights=None, env_offset=0, streams=False, traj=False, final=True):
+    words = (n + 31) // 32
+    out = {
+        "ep_return_sum": torch.full((n,), -1.0, dtype=torch.float32, device="cuda"),
+        "ep_count": torch.full((n,), -1, dtype=torch.int32, device="cuda"),
+        "totals": torch.zeros(2, dtype=torch.int64, device="cuda"),
+    }
+    if final:
+        out["final_state"] = torch.zeros(4, n, dtype=torch.float32, device="cuda")
+    if streams:
+        out["reward_stream"] = torch.zeros(T, n, dtype=torch.float32, device="cuda")
+        out["done_bits"] = torch.zeros(T, words, dtype=torch.int32, device="cuda")
+        out["action_bits"] = torch.zeros(T, words, dtype=torch.int32, device="cuda")
+    if traj:
+        out["trajectory"] = torch.zeros(T, 4, n, dtype=torch.float32, device="cuda")
+    pol = cp.policy(kind, weights) if kind else None
+    cp.cp_rollout_shard(env_offset, n, T, seed, pol, **out)
+    torch.cuda.synchronize()
+    res = {k: host(v) for k, v in out.items()}
+    res["ep_count"] = res["ep_count"].view(np.uint32)
+    res["totals"] = res["totals"].view(np.uint64)
+    return res
+
+
+@pytest.mark.parametrize("n,T", [(1, 64), (33, 64), (1025, 100), (5000, 37)])
+@pytest.mark.parametrize("ept", [1, 2, 4])
+def test_rollout_equals_repeated_fused_steps_bitwise(cp, n, T, ept):
+    cp.cp_tune("rollout_ept", ept)
+    try:
+        seed, off = 2, 77
+        r = run_rollout(cp, n, T, seed, env_offset=off, streams=True, traj=True)
+    finally:
+        cp.cp_tune("rollout_ept", 0)
+    planes = alloc_planes(n)
+    st = cp.cp_wrap(planes, n, seed, 0, off)
+    cp.cp_fill_start(st)
+    done = torch.empty(n, dtype=torch.uint8, device="cuda")
+    reward = torch.empty(n, dtype=torch.float32, device="cuda")
+    act = torch.empty(n, dtype=torch.uint8, device="cuda")
+    db, ab = H.unpack_bits(r["done_bits"], n), H.unpack_bits(r["action_bits"], n)
+    ep_len = np.zeros(n, np.int64)
+    ret = np.zeros(n, np.int64)
+    cnt = np.zeros(n, np.int64)
+    for t in range(T):
+        cp.cp_actions(n, seed, t, off, act)
+        cp.cp_step(st, None, st, reward, done)
+        torch.cuda.synchronize()
+        assert np.array_equal(host(planes[:, :n]).view(np.uint32), r["trajectory"][t].view(np.uint32)), t
+        d = host(done)
+        assert np.array_equal(d, db[t]) and np.array_equal(host(act), ab[t])
+        ep_len += 1
+        m = d.astype(bool)
+        ret[m] += ep_len[m]
+        cnt[m] += 1
+        ep_len[m] = 0
+    assert np.array_equal(r["final_state"], r["trajectory"][-1])
+    assert np.array_equal(r["ep_return_sum"], ret.astype(np.float32))
+    assert np.array_equal(r["ep_count"], cnt.astype(np.uint32))
+    assert np.all(r["reward_stream"] == 1.0)
+    assert int(r["totals"][0]) == ret.sum() and int(r["totals"][1]) == cnt.sum()
+    # padding bits of the last mask word stay zero
+    if n % 32:
+        assert not np.any(r["done_bits"].view(np.uint32)[:, -1] >> (n % 32))
+
+
+def test_config1_full_trajectory_against_oracle(cp, oracle):
+    """1,024 envs x 200 steps, seed 0: every step of the GPU trajectory checked against one
+    oracle step from the GPU's own previous state (teacher-forced), then the free-running
+    comparison of returns."""
+    w = inputs.WORKLOADS["c1"]
+    n, T = w.n_envs, w.T
+    r = run_rollout(cp, n, T, w.seed, streams=True, traj=True)
+    db, ab = H.unpack_bits(r["done_bits"], n), H.unpack_bits(r["action_bits"], n)
+    z = oracle.initial_state(n, w.seed)
+    flips = band = 0
+    for t in range(T):
+        want = oracle.step(z, seed=w.seed, t=t, want_pre_reset=True)
+        st = H.assert_step_matches(want, z, r["trajectory"][t], r["reward_stream"][t], db[t], ab[t])
+        flips += st["done_flips"]
+        band += st["band"]
+        z = r["trajectory"][t]
+    o = oracle.rollout(n, T, w.seed)
+    H.assert_returns_match(r["ep_return_sum"], r["ep_count"], o["ep_return_sum"], o["ep_count"])
+    assert flips <= band
+
+
+@pytest.mark.parametrize("name", ["c3"])
+def test_full_size_random_rollout_against_oracle(cp, oracle, name):
+    """1,048,576 envs x 500 steps in the benchmark's launch configuration; the oracle runs the
+    whole workload on all host cores."""
+    import os
+    w = inputs.WORKLOADS[name]
+    r = run_rollout(cp, w.n_envs, w.T, w.seed, final=False)
+    o = oracle.rollout(w.n_envs, w.T, w.seed, nthreads=os.cpu_count() or 1)
+    s = H.assert_returns_match(r["ep_return_sum"], r["ep_count"], o["ep_return_sum"], o["ep_count"])
+    assert int(r["totals"][0]) == int(r["ep_return_sum"].astype(np.int64).sum())
+    assert int(r["totals"][1]) == int(r["ep_count"].astype(np.int64).sum())
+    assert 21.5 < s["mean_gpu"] < 22.5
+
+
+@pytest.mark.parametrize("kind,pseed,n,T", [(1, 1, 40000, 300), (2, 2, 40000, 200), (1, 5, 3001, 150), (2, 6, 3001, 150)])
+def test_policy_rollouts_against_oracle(cp, oracle, kind, pseed, n, T):
+    wts = inputs.policy_weights(kind, pseed)
+    r = run_rollout(cp, n, T, 0, kind, wts, streams=True)
+    o = oracle.rollout(n, T, 0, kind, wts, action_bits=True, done_bits=True, min_gap=True, nthreads=4)
+    excuse = o["min_gap"] < 1e-5
+    H.assert_returns_match(r["ep_return_sum"], r["ep_count"], o["ep_return_sum"], o["ep_count"], excuse)
+    # until an env's first divergence its action and done streams are identical; most never diverge
+    same_env = (r["ep_return_sum"] == o["ep_return_sum"])
+    ga, oa = H.unpack_bits(r["action_bits"], n), H.unpack_bits(o["action_bits"], n)
+    gd, od = H.unpack_bits(r["done_bits"], n), H.unpack_bits(o["done_bits"], n)
+    agree = (ga == oa).all(axis=0) & (gd == od).all(axis=0)
+    assert agree.mean() >= 0.995
+    assert np.array_equal(gd.sum(axis=0), r["ep_count"])
+
+
+def test_sampled_envs_of_large_policy_configs(cp, oracle):
+    """Configs 4 and 5 at their full env counts but fewer steps would not be the benchmark launch;
+    instead run the full launch shape on a slice of time and compare sampled env ranges."""
+    for name, T in (("c4", 64), ("c5", 48)):
+        w = inputs.WORKLOADS[name]
+        wts = inputs.policy_weights(w.policy, w.policy_seed)
+        n = w.n_envs
+        r = run_rollout(cp, n, T, w.seed, w.policy, wts, final=False)
+        for lo in (0, n // 2 - 1000, n - 4096):
+            m = 4096
+            o = oracle.rollout(m, T, w.seed, w.policy, wts, env_offset=lo, min_gap=True)
+            H.assert_returns_match(r["ep_return_sum"][lo:lo + m], r["ep_count"][lo:lo + m],
+                                   o["ep_return_sum"], o["ep_count"], o["min_gap"] < 1e-5, min_identical=0.998)
+        assert int(r["totals"][1]) == int(r["ep_count"].astype(np.int64).sum())
+
+
+def test_shards_compose(cp):
+    n, T = 10000, 80
+    whole = run_rollout(cp, n, T, 3)
+    tot = np.zeros(2, np.uint64)
+    for rank in range(3):
+        lo, hi = inputs.shard_range(n, rank, 3)
+        part = run_rollout(cp, hi - lo, T, 3, env_offset=lo)
+        assert np.array_equal(part["ep_return_sum"], whole["ep_return_sum"][lo:hi])
+        assert np.array_equal(part["final_state"], whole["final_state"][:, lo:hi])
+        tot += part["totals"]
+    assert np.array_equal(tot, whole["totals"])
+
+
+def test_chunked_rollout_from_state(cp):
+    n, seed = 3000, 8
+    whole = run_rollout(cp, n, 90, seed)
+    st = cp.cp_reset(n, seed)
+    ep_len = torch.zeros(n, dtype=torch.int32, device="cuda")
+    ret = np.zeros(n, np.float32)
+    cnt = np.zeros(n, np.uint32)
+    tot = torch.zeros(2, dtype=torch.int64, device="cuda")
+    for T in (1, 29, 60):
+        rs = torch.zeros(n, dtype=torch.float32, device="cuda")
+        ct = torch.zeros(n, dtype=torch.int32, device="cuda")
+        cp.cp_rollout_from(st, T, ep_len, None, ep_return_sum=rs, ep_count=ct, totals=tot)
+        torch.cuda.synchronize()
+        ret += host(rs)
+        cnt += host(ct).view(np.uint32)
+    assert st.info()["t"] == 90
+    assert np.array_equal(ret, whole["ep_return_sum"]) and np.array_equal(cnt, whole["ep_count"])
+    assert np.array_equal(host(tot).view(np.uint64), whole["totals"])
+    # the batch itself now holds the final state: one more fused step equals step 91 of a longer rollout
+    longer = run_rollout(cp, n, 91, seed)
+    planes = alloc_planes(n)
+    o = cp.cp_wrap(planes, n, seed)
+    cp.cp_step(st, None, o, None, None)
+    torch.cuda.synchronize()
+    assert np.array_equal(host(planes[:, :n]), longer["final_state"])
+
+
+def test_host_buffer_entry_points(cp, oracle):
+    n, T = 5000, 60
+    wts = inputs.policy_weights(1, 1)
+    for kind, w in ((0, None), (1, wts)):
+        ref = run_rollout(cp, n, T, 4, kind, w)
+        h_ret = torch.empty(n, dtype=torch.float32).pin_memory()
+        h_cnt = torch.empty(n, dtype=torch.int32).pin_memory()
+        h_tot = torch.empty(2, dtype=torch.int64).pin_memory()
+        cp.cp_rollout_host(n, T, 4, cp.policy(kind, w) if kind else None, h_ret, h_cnt, h_tot)
+        assert np.array_equal(h_ret.numpy(), ref["ep_return_sum"])
+        assert np.array_equal(h_cnt.numpy().view(np.uint32), ref["ep_count"])
+        assert np.array_equal(h_tot.numpy().view(np.uint64), ref["totals"])
+    z = inputs.random_states(n, seed=1, spread="edge")
+    a = inputs.random_actions(n, 2)
+    for action in (None, a):
+        want = gpu_step(cp, z, 9, 4, action)
+        out, rew, dn = np.empty_like(z), np.empty(n, np.float32), np.empty(n, np.uint8)
+        cp.cp_step_host(n, 9, 4, z, action, out, rew, dn)
+        assert np.array_equal(out, want[0]) and np.array_equal(rew, want[1]) and np.array_equal(dn, want[2])
+    cp.cp_shutdown()
+
+
+def test_fused_sincos_equals_separate_sin_and_cos(cp):
+    bad = torch.zeros(1, dtype=torch.int64, device="cuda")
+    f = lambda v: int(np.float32(v).view(np.uint32))
+    cp.cp_selftest_sincos(0, f(0.35), bad)           # every float the episodes can reach
+    cp.cp_selftest_sincos(f(0.35), f(200.0), bad)    # every float up to 200 rad
+    cp.cp_selftest_sincos(f(1e5), f(1.2e5), bad)     # across the switch to the large-argument path
+    cp.cp_selftest_sincos(f(1e30), f(1.0001e30), bad)
+    torch.cuda.synchronize()
+    assert int(bad[0]) == 0
+
+
+def test_stream_selection(cp):
+    n, T = 2000, 30
+    ref = run_rollout(cp, n, T, 1)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        got = run_rollout(cp, n, T, 1)
+    assert np.array_equal(ref["ep_return_sum"], got["ep_return_sum"])

@@ -1,0 +1,92 @@
+"""CPU-only checks of the C-ABI library: it loads without a GPU, exports every
+symbol the header declares, and rejects bad arguments on the host before any
+CUDA work is attempted."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "cartpole.h")
+
+
+@pytest.fixture(scope="module")
+def cp():
+    from paper_2301_13062_b200 import binding, build
+    build.build()
+    binding.lib()
+    return binding
+
+
+def _declared():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(cp_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(cp):
+    names = _declared()
+    assert len(names) >= 20
+    assert sorted(cp.EXPORTS) == names
+    L = C.CDLL(cp.LIB_PATH)
+    for n in names:
+        assert hasattr(L, n), n
+
+
+def test_version_and_counters(cp):
+    assert "sm_100a" in cp.cp_version()
+    assert cp.cp_launch_count() >= 0
+
+
+def test_host_side_argument_errors(cp):
+    L = cp.lib()
+    assert L.cp_tune(b"no_such_key", 1) == cp.CP_EINVAL
+    assert b"unknown tuning key" in L.cp_last_error()
+    assert L.cp_tune(b"rollout_block", 100) == cp.CP_EINVAL
+    assert L.cp_tune(b"rollout_ept", 3) == cp.CP_EINVAL
+    assert L.cp_tune(b"rollout_block", 256) == cp.CP_OK
+    r = cp.cp_returns()
+    assert L.cp_rollout(0, 10, 0, None, C.byref(r)) == cp.CP_EINVAL
+    assert L.cp_rollout(16, 0, 0, None, C.byref(r)) == cp.CP_EINVAL
+    assert L.cp_rollout(16, (1 << 30) + 1, 0, None, C.byref(r)) == cp.CP_EINVAL
+    assert L.cp_rollout(16, 10, 0, None, None) == cp.CP_EINVAL
+    bad = cp.cp_policy(7, None)
+    assert L.cp_rollout(16, 10, 0, C.byref(bad), C.byref(r)) == cp.CP_EINVAL
+    noweights = cp.cp_policy(cp.CP_POLICY_MLP, None)
+    assert L.cp_rollout(16, 10, 0, C.byref(noweights), C.byref(r)) == cp.CP_EINVAL
+    assert L.cp_rollout_shard(0xFFFFFFFF, 16, 10, 0, None, C.byref(r)) == cp.CP_EINVAL
+    assert not L.cp_wrap(None, 16, 16, 0, 0, 0)
+    assert not L.cp_reset(0, 0)
+    assert not L.cp_reset(-5, 0)
+    assert L.cp_step(None, None, None, None, None) == cp.CP_EINVAL
+    assert L.cp_step_unfused(None, None, None, None, None, None, 0) == cp.CP_EINVAL
+    assert L.cp_actions(0, 0, 0, 0, None) == cp.CP_EINVAL
+    assert L.cp_rollout_host(8, 10, 0, None, None, None, None) == cp.CP_EINVAL
+    assert L.cp_step_host(8, 0, 0, None, None, None, None, None) == cp.CP_EINVAL
+    assert L.cp_selftest_sincos(5, 1, None) == cp.CP_EINVAL
+    L.cp_free(None)
+    assert L.cp_unfused_workspace_bytes(0) == 0
+    assert L.cp_unfused_workspace_bytes(1024) >= 1024 * (33 * 4 + 7)
+
+
+def test_wrap_bookkeeping_needs_no_gpu(cp):
+    L = cp.lib()
+    fake = C.c_void_p(0x7000_0000_0100)  # never dereferenced on the host
+    h = L.cp_wrap(fake, 100, 128, 9, 5, 1000)
+    assert h
+    st = cp.State(h)
+    info = st.info()
+    assert info == {"n_envs": 100, "plane_stride": 128, "seed": 9, "t": 5, "env_offset": 1000,
+                    "planes": 0x7000_0000_0100}
+    cp.cp_set_time(st, 77)
+    assert st.info()["t"] == 77
+    assert not L.cp_wrap(fake, 100, 64, 0, 0, 0)  # stride < n
+    st.close()
+
+
+def test_missing_library_fails_loudly(cp, monkeypatch):
+    monkeypatch.setattr(cp, "_lib", None)
+    monkeypatch.setattr(cp, "LIB_PATH", os.path.join(ROOT, "does_not_exist.so"))
+    with pytest.raises(ImportError):
+        cp.lib()
