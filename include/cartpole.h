@@ -146,6 +146,26 @@ int cp_step_unfused(cp_state *state, const uint8_t *action, cp_state *out_state,
                     uint8_t *done, void *workspace, size_t workspace_bytes);
 size_t cp_unfused_workspace_bytes(int64_t n_envs);
 
+/* The paper has no counterpart to this call; it exists for callers that cannot allocate device
+ * memory themselves or let a library do it on their behalf: a control loop that must not hit
+ * the device-wide synchronisation an allocation can cause, a plugin living inside another
+ * application's fixed memory budget, a process whose free device memory already belongs to
+ * some other allocator. It is cp_step_unfused with the workspace taken from an array built
+ * into the library instead of from the caller: same arguments otherwise, same results bit for
+ * bit, and it calls no cudaMalloc / cudaFree or any other allocating routine.
+ *   - At most CP_NOALLOC_MAX_ENVS environments; a larger batch is refused with CP_EINVAL
+ *     (cp_last_error says so). The array (about 8.7 MiB) is resident on every GPU that loads
+ *     this library until the process exits.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current) and keeps it; make that first call before starting any stream capture.
+ *   - All calls share the one array, which still holds the previous call's intermediates.
+ *     Nothing in it needs to start at zero (each plane is fully rewritten before it is read),
+ *     but two calls whose kernels overlap on the GPU (different streams, or different threads
+ *     without ordering between them) race on it: order such calls yourself. */
+#define CP_NOALLOC_MAX_ENVS 65536
+int cp_step_unfused_noalloc(cp_state *state, const uint8_t *action, cp_state *out_state, float *reward,
+                            uint8_t *done);
+
 /* Wrap caller-owned DEVICE planes (for example a torch tensor) as a batch at global step t.
  * plane_stride >= n_envs. The handle does not own the planes. NULL on error. */
 cp_state *cp_wrap(float *planes, int64_t n_envs, int64_t plane_stride, uint32_t seed, uint32_t t,

@@ -24,8 +24,9 @@ EXPORTS = [
     "cp_reset", "cp_step", "cp_rollout", "cp_step_unfused", "cp_unfused_workspace_bytes", "cp_wrap",
     "cp_fill_start", "cp_set_time", "cp_free", "cp_state_info", "cp_actions", "cp_rollout_shard",
     "cp_rollout_from", "cp_rollout_host", "cp_step_host", "cp_shutdown", "cp_set_stream", "cp_tune",
-    "cp_launch_count", "cp_selftest_sincos", "cp_last_error", "cp_version",
+    "cp_launch_count", "cp_selftest_sincos", "cp_last_error", "cp_version", "cp_step_unfused_noalloc",
 ]
+CP_NOALLOC_MAX_ENVS = 65536
 
 
 class cp_policy(C.Structure):
@@ -61,6 +62,7 @@ def lib() -> C.CDLL:
             "cp_rollout": (i32, [i64, i64, u32, C.POINTER(cp_policy), C.POINTER(cp_returns)]),
             "cp_step_unfused": (i32, [p, p, p, p, p, p, sz]),
             "cp_unfused_workspace_bytes": (sz, [i64]),
+            "cp_step_unfused_noalloc": (i32, [p, p, p, p, p]),
             "cp_wrap": (p, [p, i64, i64, u32, u32, u32]),
             "cp_fill_start": (i32, [p]),
             "cp_set_time": (i32, [p, u32]),
@@ -228,6 +230,16 @@ def cp_step_unfused(state: State, action, out_state: State, reward, done, worksp
     _check(lib().cp_step_unfused(state.handle, _dptr(action, torch.uint8), out_state.handle,
                                  _dptr(reward, torch.float32), _dptr(done, torch.uint8), _dptr(workspace),
                                  workspace.numel() * workspace.element_size()))
+
+
+def cp_step_unfused_noalloc(state: State, action, out_state: State, reward, done) -> None:
+    """The per-op step for callers that cannot allocate device memory (no workspace argument:
+    the intermediates live in an array built into the library). At most CP_NOALLOC_MAX_ENVS
+    environments; calls that overlap on the GPU race on that shared array."""
+    import torch
+    _use_current_stream()
+    _check(lib().cp_step_unfused_noalloc(state.handle, _dptr(action, torch.uint8), out_state.handle,
+                                         _dptr(reward, torch.float32), _dptr(done, torch.uint8)))
 
 
 def cp_actions(n_envs: int, seed: int, t: int, env_offset: int, out) -> None:

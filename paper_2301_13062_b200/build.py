@@ -13,7 +13,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcartpole.so")
-SOURCES = ["capi.cu", "step_kernel.cu", "ladder_kernels.cu", "rollout_kernel.cu"]
+SOURCES = ["capi.cu", "step_kernel.cu", "ladder_kernels.cu", "rollout_kernel.cu", "ladder_noalloc.cu"]
 HEADERS = ["cartpole_device.cuh", "cartpole_internal.h", os.path.join("..", "..", "include", "cartpole.h")]
 
 NVCC_FLAGS = [

@@ -184,6 +184,13 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 }  // namespace
 
+// Accessors for entry points that live in other translation units.
+namespace cp {
+cudaStream_t thread_stream() { return tl_stream; }
+int set_error(int code, const char *text) { return fail(code, "%s", text); }
+void adopt_step(cp_state *state, cp_state *out_state, uint32_t steps) { advance(state, out_state, steps); }
+}  // namespace cp
+
 extern "C" {
 
 cp_state *cp_reset(int64_t n_envs, uint32_t seed) {

@@ -4,6 +4,8 @@
 #include <cstdint>
 #include <cuda_runtime.h>
 
+struct cp_state;
+
 namespace cp {
 
 // Parameters of one fused step launch.
@@ -64,5 +66,10 @@ cudaError_t launch_sincos_selftest(uint32_t lo_bits, uint32_t hi_bits, unsigned 
 size_t ladder_workspace_bytes(int64_t n);
 int ladder_launch_count(bool hashed_action);
 cudaError_t launch_ladder(const StepParams &p, void *workspace, cudaStream_t s);
+
+// Defined in capi.cu, for entry points that live in other translation units.
+cudaStream_t thread_stream();                    // stream chosen by cp_set_stream on this thread
+int set_error(int code, const char *text);       // records the text for cp_last_error, returns code
+void adopt_step(cp_state *state, cp_state *out_state, uint32_t steps);  // out takes seed/offset, t + steps
 
 }  // namespace cp
