@@ -42,8 +42,10 @@
  *   thacc = (g*s - c*temp) / (l*(ft - (m_pole*(c*c))/m_total))
  *   xacc  = temp - ((pml*thacc)*c)/m_total
  *   x' = x + tau*xd; xd' = xd + tau*xacc; th' = th + tau*thd; thd' = thd + tau*thacc
- *   every operation rounded once to float32 (no fused multiply-add, IEEE division,
- *   accurate sinf/cosf; no fast-math);
+ *   every operation rounded once to float32 (no fused multiply-add, IEEE division; no
+ *   fast-math). sinf/cosf: for |theta| <= 0.25 (every angle an episode can hold; the
+ *   termination threshold is 0.2095) a polynomial with measured error <= 0.53 ulp, for any
+ *   other argument the CUDA library's accurate sinf/cosf;
  *   done = x'<-x_max | x'>x_max | th'<-theta_max | th'>theta_max  (strict, on the
  *   updated state); reward = 1.0f for every step (each step starts from a live
  *   state; the terminating step counts); a finished environment continues from a
@@ -137,6 +139,11 @@ int cp_rollout(int64_t n_envs, int64_t T, uint32_t seed, const cp_policy *policy
 
 /* ---- helpers ------------------------------------------------------------------------- */
 
+/* Sec. V (the host loop over steps): k consecutive cp_step launches in place with hashed
+ * actions, issued from one call so that the host cost per step is one kernel launch. reward and
+ * done (each may be NULL) are overwritten by every step and end up holding the last step's. */
+int cp_step_repeat(cp_state *state, int64_t k, float *reward, uint8_t *done);
+
 /* Sec. V-F (eager per-op execution): the same step as cp_step computed by one kernel per
  * elementwise operation (45 launches, 46 when the action is hashed), every intermediate a
  * plane in `workspace` (DEVICE, 256-byte aligned, >= cp_unfused_workspace_bytes(n_envs)).
@@ -212,18 +219,32 @@ void cp_shutdown(void);
 /* Stream used by this thread's later calls (a cudaStream_t; NULL = legacy default stream). */
 void cp_set_stream(void *cuda_stream);
 
-/* Launch tuning, process-wide. key: "rollout_block" (threads per CTA, multiple of 32),
- * "rollout_ept" (environments per thread: 1, 2 or 4), "rollout_ctas_per_sm" (0 = from the
- * occupancy calculator), "step_block". Returns CP_EINVAL for an unknown key or value. */
+/* Launch tuning, process-wide. key: "rollout_block" (threads per CTA, 32..256, multiple of 32;
+ * default 256), "rollout_ept" (environments per thread: 1, 2 or 4; 0 = default, 2 for large
+ * batches), "rollout_ctas_per_sm" (0 = default: one 32*ept-environment task per warp and as many
+ * CTAs as that takes; k > 0 = persistent grid of k CTAs per SM looping over tasks), "step_block"
+ * (32..256, default 64). Returns CP_EINVAL for an unknown key or value. */
 int cp_tune(const char *key, int value);
 
 /* Number of kernels this library has launched in this process (all threads). */
 uint64_t cp_launch_count(void);
 
 /* Diagnostics: count float32 values v in [lo, hi] (bit patterns, both >= 0, lo <= hi, and their
- * negatives) for which the fused kernels' sine/cosine differ in any bit from the ladder's
- * separate sinf / cosf kernels. mismatches DEVICE [1] uint64, caller zeroes. */
+ * negatives) for which the fused kernels' combined sine/cosine differs in any bit from the
+ * ladder's separate sine and cosine kernels. mismatches DEVICE [1] uint64, caller zeroes. */
 int cp_selftest_sincos(uint32_t lo_bits, uint32_t hi_bits, uint64_t *mismatches);
+
+/* Diagnostics: error of the kernels' sine and cosine against float64 over the float32 values in
+ * [lo, hi] (bit patterns as above). out DEVICE [4] uint64, caller zeroes: out[0] / out[1] = largest
+ * error of sin / cos in millionths of a float32 ulp; out[2] / out[3] = number of results that are
+ * not the correctly rounded value. */
+int cp_selftest_sincos_accuracy(uint32_t lo_bits, uint32_t hi_bits, uint64_t *out);
+
+/* Diagnostics: the kernels replace x / 1.1f by a three-operation exact sequence and the start-state
+ * mapping by an equivalent two-operation one. This checks, over all 2^32 float bit patterns (2^24
+ * for the mapping), that the replacements give the bits of the operations they stand for wherever
+ * they are used. out DEVICE [4] uint64, caller zeroes; every count must come back 0. */
+int cp_selftest_arith(uint64_t *out);
 
 const char *cp_last_error(void);
 const char *cp_version(void);

@@ -13,7 +13,8 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libcartpole.so")
+# CARTPOLE_LIB selects another build of the same library (tuning experiments).
+LIB_PATH = os.environ.get("CARTPOLE_LIB") or os.path.join(_HERE, "libcartpole.so")
 
 CP_OK, CP_EINVAL, CP_ECUDA, CP_ENOMEM = 0, -1, -2, -3
 CP_POLICY_RANDOM, CP_POLICY_LINEAR, CP_POLICY_MLP = 0, 1, 2
@@ -25,6 +26,7 @@ EXPORTS = [
     "cp_fill_start", "cp_set_time", "cp_free", "cp_state_info", "cp_actions", "cp_rollout_shard",
     "cp_rollout_from", "cp_rollout_host", "cp_step_host", "cp_shutdown", "cp_set_stream", "cp_tune",
     "cp_launch_count", "cp_selftest_sincos", "cp_last_error", "cp_version", "cp_step_unfused_noalloc",
+    "cp_selftest_sincos_accuracy", "cp_selftest_arith", "cp_step_repeat",
 ]
 CP_NOALLOC_MAX_ENVS = 65536
 
@@ -60,6 +62,7 @@ def lib() -> C.CDLL:
             "cp_reset": (p, [i64, u32]),
             "cp_step": (i32, [p, p, p, p, p]),
             "cp_rollout": (i32, [i64, i64, u32, C.POINTER(cp_policy), C.POINTER(cp_returns)]),
+            "cp_step_repeat": (i32, [p, i64, p, p]),
             "cp_step_unfused": (i32, [p, p, p, p, p, p, sz]),
             "cp_unfused_workspace_bytes": (sz, [i64]),
             "cp_step_unfused_noalloc": (i32, [p, p, p, p, p]),
@@ -79,6 +82,8 @@ def lib() -> C.CDLL:
             "cp_tune": (i32, [C.c_char_p, i32]),
             "cp_launch_count": (C.c_uint64, []),
             "cp_selftest_sincos": (i32, [u32, u32, p]),
+            "cp_selftest_sincos_accuracy": (i32, [u32, u32, p]),
+            "cp_selftest_arith": (i32, [p]),
             "cp_last_error": (C.c_char_p, []),
             "cp_version": (C.c_char_p, []),
         }
@@ -220,6 +225,12 @@ def cp_step(state: State, action, out_state: State, reward, done) -> None:
                          _dptr(done, torch.uint8)))
 
 
+def cp_step_repeat(state: State, k: int, reward, done) -> None:
+    import torch
+    _use_current_stream()
+    _check(lib().cp_step_repeat(state.handle, k, _dptr(reward, torch.float32), _dptr(done, torch.uint8)))
+
+
 def cp_unfused_workspace_bytes(n_envs: int) -> int:
     return int(lib().cp_unfused_workspace_bytes(n_envs))
 
@@ -294,6 +305,18 @@ def cp_selftest_sincos(lo_bits: int, hi_bits: int, mismatches) -> None:
     import torch
     _use_current_stream()
     _check(lib().cp_selftest_sincos(lo_bits, hi_bits, _dptr(mismatches, torch.int64)))
+
+
+def cp_selftest_sincos_accuracy(lo_bits: int, hi_bits: int, out) -> None:
+    import torch
+    _use_current_stream()
+    _check(lib().cp_selftest_sincos_accuracy(lo_bits, hi_bits, _dptr(out, torch.int64)))
+
+
+def cp_selftest_arith(out) -> None:
+    import torch
+    _use_current_stream()
+    _check(lib().cp_selftest_arith(_dptr(out, torch.int64)))
 
 
 def cp_version() -> str:

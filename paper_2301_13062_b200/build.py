@@ -36,7 +36,11 @@ def _stale(target: str, deps: list[str]) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, extra: list[str] | None = None, out: str | None = None) -> str:
+    """Compile and link. `extra` adds nvcc flags (e.g. -DCP_ROLLOUT_MIN_CTAS=5) and `out` names
+    another output file; both are for tuning experiments and force a full rebuild."""
+    if extra or out:
+        return _build_variant(extra or [], out or LIB, verbose)
     hdrs = [os.path.normpath(os.path.join(CSRC, h)) for h in HEADERS] + [os.path.abspath(__file__)]
     objs = []
     for src in SOURCES:
@@ -53,6 +57,21 @@ def build(force: bool = False, verbose: bool = False) -> str:
         cmd = [_nvcc(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB, *objs]
         subprocess.run(cmd, check=True)
     return LIB
+
+
+def _build_variant(extra: list[str], out: str, verbose: bool) -> str:
+    import tempfile
+    with tempfile.TemporaryDirectory() as tmp:
+        objs = []
+        for src in SOURCES:
+            o = os.path.join(tmp, src.replace(".cu", ".o"))
+            cmd = [_nvcc(), *NVCC_FLAGS, *extra, "-c", os.path.join(CSRC, src), "-o", o]
+            if verbose:
+                cmd.insert(1, "-Xptxas=-v")
+            subprocess.run(cmd, check=True)
+            objs.append(o)
+        subprocess.run([_nvcc(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", out, *objs], check=True)
+    return out
 
 
 if __name__ == "__main__":

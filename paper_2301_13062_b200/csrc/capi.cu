@@ -296,6 +296,15 @@ int cp_step(cp_state *state, const uint8_t *action, cp_state *out_state, float *
     return CP_OK;
 }
 
+int cp_step_repeat(cp_state *state, int64_t k, float *reward, uint8_t *done) {
+    if (k < 0 || k > CP_MAX_T) return fail(CP_EINVAL, "k must be in [0, 2^30]");
+    for (int64_t i = 0; i < k; ++i) {
+        int rc = cp_step(state, nullptr, state, reward, done);
+        if (rc != CP_OK) return rc;
+    }
+    return CP_OK;
+}
+
 size_t cp_unfused_workspace_bytes(int64_t n_envs) {
     return n_envs > 0 ? cp::ladder_workspace_bytes(n_envs) : 0;
 }
@@ -430,7 +439,7 @@ int cp_tune(const char *key, int value) {
         if (value != 0 && value != 1 && value != 2 && value != 4) return fail(CP_EINVAL, "rollout_ept must be 0, 1, 2 or 4");
         cp::g_tuning.rollout_ept = value;
     } else if (!strcmp(key, "rollout_ctas_per_sm")) {
-        if (value < 0 || value > 32) return fail(CP_EINVAL, "rollout_ctas_per_sm must be 0..32");
+        if (value < 0 || value > 1024) return fail(CP_EINVAL, "rollout_ctas_per_sm must be 0..1024");
         cp::g_tuning.rollout_ctas_per_sm = value;
     } else if (!strcmp(key, "step_block")) {
         if (value < 32 || value > 256 || value % 32) return fail(CP_EINVAL, "step_block must be 32..256, multiple of 32");
@@ -448,6 +457,19 @@ int cp_selftest_sincos(uint32_t lo_bits, uint32_t hi_bits, uint64_t *mismatches)
     if (lo_bits > hi_bits || hi_bits >= 0x7F800000u) return fail(CP_EINVAL, "need lo <= hi, both finite and non-negative");
     cudaError_t e = cp::launch_sincos_selftest(lo_bits, hi_bits, reinterpret_cast<unsigned long long *>(mismatches),
                                                tl_stream);
+    return e == cudaSuccess ? CP_OK : cuda_fail(e, "self-test launch");
+}
+
+int cp_selftest_sincos_accuracy(uint32_t lo_bits, uint32_t hi_bits, uint64_t *out) {
+    if (!out || !is_aligned(out, 8)) return fail(CP_EINVAL, "out is NULL or misaligned");
+    if (lo_bits > hi_bits || hi_bits >= 0x7F800000u) return fail(CP_EINVAL, "need lo <= hi, both finite and non-negative");
+    cudaError_t e = cp::launch_sincos_accuracy(lo_bits, hi_bits, reinterpret_cast<unsigned long long *>(out), tl_stream);
+    return e == cudaSuccess ? CP_OK : cuda_fail(e, "self-test launch");
+}
+
+int cp_selftest_arith(uint64_t *out) {
+    if (!out || !is_aligned(out, 8)) return fail(CP_EINVAL, "out is NULL or misaligned");
+    cudaError_t e = cp::launch_arith_selftest(reinterpret_cast<unsigned long long *>(out), tl_stream);
     return e == cudaSuccess ? CP_OK : cuda_fail(e, "self-test launch");
 }
 

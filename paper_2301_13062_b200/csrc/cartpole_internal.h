@@ -45,8 +45,8 @@ struct RolloutParams {
 struct LaunchTuning {
     int rollout_block = 256;
     int rollout_ept = 0;          // 0: chosen per policy
-    int rollout_ctas_per_sm = 0;  // 0: occupancy calculator
-    int step_block = 256;
+    int rollout_ctas_per_sm = 0;  // 0: one task per warp (non-persistent grid)
+    int step_block = 64;
 };
 extern LaunchTuning g_tuning;
 
@@ -61,6 +61,9 @@ cudaError_t launch_actions(uint8_t *out, int64_t n, uint32_t env_offset, uint32_
 cudaError_t launch_rollout(RolloutParams &p, int policy, bool streams, cudaStream_t s);
 cudaError_t launch_sincos_selftest(uint32_t lo_bits, uint32_t hi_bits, unsigned long long *mismatches,
                                    cudaStream_t s);
+
+cudaError_t launch_sincos_accuracy(uint32_t lo_bits, uint32_t hi_bits, unsigned long long *out, cudaStream_t s);
+cudaError_t launch_arith_selftest(unsigned long long *out, cudaStream_t s);
 
 // The per-op ladder. Workspace layout is private to ladder_kernels.cu.
 size_t ladder_workspace_bytes(int64_t n);

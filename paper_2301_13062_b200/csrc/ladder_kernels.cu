@@ -129,10 +129,10 @@ struct OpForce {
     __device__ float operator()(uint8_t a) const { return a ? kF : -kF; }
 };
 struct OpSin {
-    __device__ float operator()(float x) const { return sinf(x); }
+    __device__ float operator()(float x) const { return sin_op(x); }
 };
 struct OpCos {
-    __device__ float operator()(float x) const { return cosf(x); }
+    __device__ float operator()(float x) const { return cos_op(x); }
 };
 struct OpMulC {
     float c;

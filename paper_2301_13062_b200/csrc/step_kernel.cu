@@ -24,8 +24,12 @@ __device__ __forceinline__ bool step_one(State &z, uint32_t env, const StepParam
     return euler_step(z, force_from_signbit(sb));
 }
 
+#ifndef CP_STEP_MIN_CTAS
+#define CP_STEP_MIN_CTAS 1
+#endif
+
 template <bool VEC>
-__global__ void __launch_bounds__(256) step_kernel(const __grid_constant__ StepParams p) {
+__global__ void __launch_bounds__(256, CP_STEP_MIN_CTAS) step_kernel(const __grid_constant__ StepParams p) {
     const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const bool has_action = p.action != nullptr;
     if (VEC) {
@@ -155,9 +159,9 @@ __global__ void sincos_selftest_kernel(uint32_t lo, uint32_t hi, unsigned long l
         const float v = __uint_as_float(lo + (uint32_t)k);
         float s, c;
         sin_cos(v, s, c);
-        bad += (__float_as_uint(s) != __float_as_uint(sinf(v))) | (__float_as_uint(c) != __float_as_uint(cosf(v)));
+        bad += (__float_as_uint(s) != __float_as_uint(sin_op(v))) | (__float_as_uint(c) != __float_as_uint(cos_op(v)));
         sin_cos(-v, s, c);
-        bad += (__float_as_uint(s) != __float_as_uint(sinf(-v))) | (__float_as_uint(c) != __float_as_uint(cosf(-v)));
+        bad += (__float_as_uint(s) != __float_as_uint(sin_op(-v))) | (__float_as_uint(c) != __float_as_uint(cos_op(-v)));
     }
     for (int o = 16; o > 0; o >>= 1) bad += __shfl_down_sync(0xffffffffu, bad, o);
     if ((threadIdx.x & 31) == 0 && bad) atomicAdd(mismatches, bad);
@@ -166,6 +170,95 @@ __global__ void sincos_selftest_kernel(uint32_t lo, uint32_t hi, unsigned long l
 cudaError_t launch_sincos_selftest(uint32_t lo_bits, uint32_t hi_bits, unsigned long long *mismatches,
                                    cudaStream_t s) {
     sincos_selftest_kernel<<<sm_count() * 8, 256, 0, s>>>(lo_bits, hi_bits, mismatches);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ---- self-test: error of the kernels' sine/cosine against float64, in millionths of an ulp ----
+// out[0], out[1] = max error of sin, cos; out[2], out[3] = how many results are not the
+// correctly rounded float32 value.
+__device__ __forceinline__ unsigned long long micro_ulps(float got, double exact) {
+    const float near = (float)exact;
+    // ulp of the exact value's binade
+    const float up = __uint_as_float(__float_as_uint(fabsf(near)) + 1u);
+    const double ulp = (double)up - (double)fabsf(near);
+    const double e = fabs((double)got - exact) / ulp;
+    return (unsigned long long)(e * 1e6);
+}
+
+__global__ void sincos_accuracy_kernel(uint32_t lo, uint32_t hi, unsigned long long *out) {
+    unsigned long long ms = 0, mc = 0, ns = 0, nc = 0;
+    const uint64_t span = (uint64_t)hi - lo + 1;
+    for (uint64_t k = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; k < span; k += (uint64_t)gridDim.x * blockDim.x) {
+        const float v = __uint_as_float(lo + (uint32_t)k);
+        float s, c;
+        sin_cos(v, s, c);
+        const double es = sin((double)v), ec = cos((double)v);
+        const unsigned long long a = micro_ulps(s, es), b = micro_ulps(c, ec);
+        ms = a > ms ? a : ms;
+        mc = b > mc ? b : mc;
+        ns += __float_as_uint(s) != __float_as_uint((float)es);
+        nc += __float_as_uint(c) != __float_as_uint((float)ec);
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long a = __shfl_down_sync(0xffffffffu, ms, o), b = __shfl_down_sync(0xffffffffu, mc, o);
+        ms = a > ms ? a : ms;
+        mc = b > mc ? b : mc;
+        ns += __shfl_down_sync(0xffffffffu, ns, o);
+        nc += __shfl_down_sync(0xffffffffu, nc, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        atomicMax(out, ms);
+        atomicMax(out + 1, mc);
+        if (ns) atomicAdd(out + 2, ns);
+        if (nc) atomicAdd(out + 3, nc);
+    }
+}
+
+cudaError_t launch_sincos_accuracy(uint32_t lo_bits, uint32_t hi_bits, unsigned long long *out, cudaStream_t s) {
+    sincos_accuracy_kernel<<<sm_count() * 8, 256, 0, s>>>(lo_bits, hi_bits, out);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ---- self-test: the exact shortcuts against the operations they replace ----
+// out[0]: bit patterns x (all 2^32) where div_mtot(x) != __fdiv_rn(x, 1.1f)
+// out[1]: patterns inside div_mtot_not_tiny's domain (+0, NaN, Inf, |x| >= 2^-100) where it differs
+// out[2]: patterns inside div_mtot_normal's domain (+0, NaN, 2^-100 <= |x| <= FLT_MAX) where it differs
+// out[3]: 24-bit inputs where start_from_bits differs from the three-operation definition
+__global__ void arith_selftest_kernel(unsigned long long *out) {
+    unsigned long long b0 = 0, b1 = 0, b2 = 0, b3 = 0;
+    for (uint64_t k = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; k < (1ull << 32);
+         k += (uint64_t)gridDim.x * blockDim.x) {
+        const uint32_t bits = (uint32_t)k;
+        const float x = __uint_as_float(bits);
+        const uint32_t want = __float_as_uint(__fdiv_rn(x, kMTot));
+        const float ax = fabsf(x);
+        const bool is_nan = x != x;
+        const bool pos_zero = bits == 0u;
+        b0 += __float_as_uint(div_mtot(x)) != want;
+        if (pos_zero || is_nan || ax >= 7.888609052e-31f) b1 += __float_as_uint(div_mtot_not_tiny(x)) != want;
+        if (pos_zero || is_nan || (ax >= 7.888609052e-31f && ax <= 3.402823466e+38f))
+            b2 += __float_as_uint(div_mtot_normal(x)) != want;
+        if (bits < (1u << 24))
+            b3 += __float_as_uint(start_from_bits(bits)) != __float_as_uint(start_from_bits_reference(bits));
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        b0 += __shfl_down_sync(0xffffffffu, b0, o);
+        b1 += __shfl_down_sync(0xffffffffu, b1, o);
+        b2 += __shfl_down_sync(0xffffffffu, b2, o);
+        b3 += __shfl_down_sync(0xffffffffu, b3, o);
+    }
+    if ((threadIdx.x & 31) == 0 && (b0 | b1 | b2 | b3)) {
+        atomicAdd(out, b0);
+        atomicAdd(out + 1, b1);
+        atomicAdd(out + 2, b2);
+        atomicAdd(out + 3, b3);
+    }
+}
+
+cudaError_t launch_arith_selftest(unsigned long long *out, cudaStream_t s) {
+    arith_selftest_kernel<<<sm_count() * 8, 256, 0, s>>>(out);
     count_launch();
     return cudaGetLastError();
 }
