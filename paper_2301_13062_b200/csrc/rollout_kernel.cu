@@ -32,7 +32,7 @@ __device__ __forceinline__ uint32_t policy_signbit(const RolloutParams &p, const
 #define CP_ROLLOUT_MIN_CTAS 1
 #endif
 
-template <int POLICY, int EPT, bool STREAMS>
+template <int POLICY, int EPT, int STREAMS>
 __global__ void __launch_bounds__(256, CP_ROLLOUT_MIN_CTAS) rollout_kernel(const __grid_constant__ RolloutParams p) {
     const uint32_t lane = threadIdx.x & 31u;
     const int64_t warps_total = (int64_t)gridDim.x * (blockDim.x >> 5);
@@ -70,6 +70,25 @@ __global__ void __launch_bounds__(256, CP_ROLLOUT_MIN_CTAS) rollout_kernel(const
             last[j] = p.t0;
         }
 
+        // Per-step stream outputs advance by one row per step: keep running pointers / offsets
+        // instead of recomputing row * width + column with 64-bit multiplies every step.
+        // STREAMS == 1: exactly the reward plane and the done bitmask are written (no run-time
+        // tests in the loop); STREAMS == 2: any combination, tested per step.
+        float *rew_ptr[EPT];
+        uint32_t *done_ptr[EPT];
+        int64_t env_off[EPT], word_off[EPT];  // into [T][n] planes and [T][words] bit planes
+        bool word_ok[EPT];
+#pragma unroll
+        for (int j = 0; j < EPT; ++j) {
+            env_off[j] = idx[j];
+            word_off[j] = task * EPT + j;
+            word_ok[j] = lane == 0 && word_off[j] < words;
+            rew_ptr[j] = STREAMS == 1 ? p.reward_stream + idx[j] : nullptr;
+            done_ptr[j] = STREAMS == 1 ? p.done_bits + (word_ok[j] ? word_off[j] : 0) : nullptr;
+        }
+        const bool want_done = STREAMS == 2 && p.done_bits, want_act = STREAMS == 2 && p.action_bits;
+        const bool want_rew = STREAMS == 2 && p.reward_stream, want_traj = STREAMS == 2 && p.trajectory;
+
         const uint32_t t_end = p.t0 + p.T;
         for (uint32_t t = p.t0; t != t_end; ++t) {
 #pragma unroll
@@ -81,27 +100,34 @@ __global__ void __launch_bounds__(256, CP_ROLLOUT_MIN_CTAS) rollout_kernel(const
                     last[j] = t + 1u;
                     z[j] = start_state(kr[j], t + 1u);
                 }
-                if (STREAMS) {
-                    const uint32_t k = t - p.t0;
-                    const int64_t word = task * EPT + j;
-                    if (p.done_bits) {
+                if (STREAMS == 1) {
+                    const uint32_t m = __ballot_sync(0xffffffffu, done && valid[j]);
+                    if (word_ok[j]) *done_ptr[j] = m;
+                    if (valid[j]) *rew_ptr[j] = 1.0f;
+                    done_ptr[j] += words;
+                    rew_ptr[j] += p.n;
+                }
+                if (STREAMS == 2) {
+                    if (want_done) {
                         const uint32_t m = __ballot_sync(0xffffffffu, done && valid[j]);
-                        if (lane == 0 && word < words) p.done_bits[(int64_t)k * words + word] = m;
+                        if (word_ok[j]) p.done_bits[word_off[j]] = m;
                     }
-                    if (p.action_bits) {
+                    if (want_act) {
                         const uint32_t m = __ballot_sync(0xffffffffu, (sb != 0u) && valid[j]);
-                        if (lane == 0 && word < words) p.action_bits[(int64_t)k * words + word] = m;
+                        if (word_ok[j]) p.action_bits[word_off[j]] = m;
                     }
                     if (valid[j]) {
-                        if (p.reward_stream) p.reward_stream[(int64_t)k * p.n + idx[j]] = 1.0f;
-                        if (p.trajectory) {
-                            float *tr = p.trajectory + (int64_t)k * 4 * p.n + idx[j];
+                        if (want_rew) p.reward_stream[env_off[j]] = 1.0f;
+                        if (want_traj) {
+                            float *tr = p.trajectory + 4 * env_off[j] - 3 * idx[j];  // row 4k, column idx
                             tr[0] = z[j].x;
                             tr[p.n] = z[j].xd;
                             tr[2 * p.n] = z[j].th;
                             tr[3 * p.n] = z[j].thd;
                         }
                     }
+                    env_off[j] += p.n;
+                    word_off[j] += words;
                 }
             }
         }
@@ -140,7 +166,7 @@ __global__ void __launch_bounds__(256, CP_ROLLOUT_MIN_CTAS) rollout_kernel(const
 
 namespace {
 
-template <int POLICY, int EPT, bool STREAMS>
+template <int POLICY, int EPT, int STREAMS>
 cudaError_t launch_one(RolloutParams &p, cudaStream_t s) {
     const int block = g_tuning.rollout_block;
     p.n_tasks = (p.n + 32 * EPT - 1) / (32 * EPT);
@@ -162,7 +188,7 @@ cudaError_t launch_one(RolloutParams &p, cudaStream_t s) {
     return cudaGetLastError();
 }
 
-template <int POLICY, bool STREAMS>
+template <int POLICY, int STREAMS>
 cudaError_t launch_ept(RolloutParams &p, int ept, cudaStream_t s) {
     switch (ept) {
         case 1: return launch_one<POLICY, 1, STREAMS>(p, s);
@@ -178,10 +204,18 @@ cudaError_t launch_rollout(RolloutParams &p, int policy, bool streams, cudaStrea
     if (ept == 0) ept = 2;
     // Small batches: spread environments over as many warps as possible.
     while (ept > 1 && (p.n + 32 * ept - 1) / (32 * ept) < (int64_t)sm_count() * 16) ept >>= 1;
-    switch (policy) {
-        case 0: return streams ? launch_ept<0, true>(p, ept, s) : launch_ept<0, false>(p, ept, s);
-        case 1: return streams ? launch_ept<1, true>(p, ept, s) : launch_ept<1, false>(p, ept, s);
-        default: return streams ? launch_ept<2, true>(p, ept, s) : launch_ept<2, false>(p, ept, s);
+    // 0: no per-step output; 1: reward plane + done bitmask only; 2: any other combination
+    const int mode = !streams ? 0 : (p.reward_stream && p.done_bits && !p.action_bits && !p.trajectory) ? 1 : 2;
+    switch (policy * 3 + mode) {
+        case 0: return launch_ept<0, 0>(p, ept, s);
+        case 1: return launch_ept<0, 1>(p, ept, s);
+        case 2: return launch_ept<0, 2>(p, ept, s);
+        case 3: return launch_ept<1, 0>(p, ept, s);
+        case 4: return launch_ept<1, 1>(p, ept, s);
+        case 5: return launch_ept<1, 2>(p, ept, s);
+        case 6: return launch_ept<2, 0>(p, ept, s);
+        case 7: return launch_ept<2, 1>(p, ept, s);
+        default: return launch_ept<2, 2>(p, ept, s);
     }
 }
 

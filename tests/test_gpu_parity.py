@@ -221,7 +221,8 @@ def run_rollout(cp, n, T, seed, kind=0, weights=None, env_offset=0, streams=Fals
     if streams:
         out["reward_stream"] = torch.zeros(T, n, dtype=torch.float32, device="cuda")
         out["done_bits"] = torch.zeros(T, words, dtype=torch.int32, device="cuda")
-        out["action_bits"] = torch.zeros(T, words, dtype=torch.int32, device="cuda")
+        if streams != "reward+done":
+            out["action_bits"] = torch.zeros(T, words, dtype=torch.int32, device="cuda")
     if traj:
         out["trajectory"] = torch.zeros(T, 4, n, dtype=torch.float32, device="cuda")
     pol = cp.policy(kind, weights) if kind else None
@@ -339,6 +340,23 @@ def test_sampled_envs_of_large_policy_configs(cp, oracle):
             H.assert_returns_match(r["ep_return_sum"][lo:lo + m], r["ep_count"][lo:lo + m],
                                    o["ep_return_sum"], o["ep_count"], o["min_gap"] < 1e-5, min_identical=0.998)
         assert int(r["totals"][1]) == int(r["ep_count"].astype(np.int64).sum())
+
+
+@pytest.mark.parametrize("ept", [1, 2, 4])
+def test_reward_and_done_only_streams_equal_the_general_stream_kernel(cp, ept):
+    """The reward-plane + done-bitmask combination has a kernel of its own."""
+    cp.cp_tune("rollout_ept", ept)
+    try:
+        for n, T, kind in ((5001, 60, 0), (40000, 40, 1), (33, 20, 2)):
+            w = inputs.policy_weights(kind, 3) if kind else None
+            a = run_rollout(cp, n, T, 2, kind, w, env_offset=9, streams=True)
+            b = run_rollout(cp, n, T, 2, kind, w, env_offset=9, streams="reward+done")
+            for k in ("ep_return_sum", "ep_count", "totals", "final_state", "reward_stream", "done_bits"):
+                assert np.array_equal(a[k], b[k]), (k, n, kind)
+            assert np.all(b["reward_stream"] == 1.0)
+            assert np.array_equal(H.unpack_bits(b["done_bits"], n).sum(axis=0), b["ep_count"])
+    finally:
+        cp.cp_tune("rollout_ept", 0)
 
 
 def test_shards_compose(cp):
