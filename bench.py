@@ -30,9 +30,21 @@ sys.path.insert(0, ROOT)
 METRIC = "env_steps_per_sec"
 UNIT = "env-steps/s"
 SMS = 148
-# Algorithmic thread-level operations per env-step of each rollout variant (see the design doc,
-# "Rollout kernel: operation count") and algorithmic HBM bytes per env-step of the step paths.
-ALG_OPS = {"random": 150.0, "linear": 152.0, "mlp": 540.0}
+# Work per env-step of each rollout variant, counted by ncu on 1,048,576 envs x 100 steps
+# (profiles/rollout_kernel_*.md): "thread" = smsp__thread_inst_executed.sum / (N*T), the
+# instructions environments actually execute (the algorithmic figure: an env that does not
+# terminate executes no restart code); "slot" = 32 * smsp__inst_executed.sum / (N*T), the issue
+# slots the warps occupy, which also counts lanes idling while a neighbour restarts.
+ROLLOUT_OPS = {
+    "random": {"thread": 78.5, "slot": 111.9},
+    "linear": {"thread": 82.5, "slot": 92.0},
+    "linear+streams": {"thread": 97.2, "slot": 106.8},
+    "mlp": {"thread": 449.1, "slot": 480.7},
+}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch in the same captures.
+ROLLOUT_DRAM_BYTES = {"random": 20.7e3, "linear": 21.0e3, "linear+streams": 382.9e6, "mlp": 33.0e3}
+STEP_DRAM_BYTES_16M = 565.8e6  # step_kernel at 16,777,216 envs (profiles/step_kernel_16m_envs.md)
+# Algorithmic HBM bytes per env-step of the step paths.
 STEP_BYTES = 37.0      # 16 in + 16 out + 4 reward + 1 done, hashed action
 LADDER_BYTES = 375.0   # sum over the 46 one-op kernels of their input and output planes
 
@@ -60,7 +72,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -161,7 +173,7 @@ def main() -> None:
     import torch.distributed as dist
 
     from paper_2301_13062_b200 import binding as cp
-    from paper_2301_13062_b200 import inputs
+    from paper_2301_13062_b200 import inputs, sharding
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -179,11 +191,7 @@ def main() -> None:
         torch.cuda.synchronize()
 
     def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t[0])
+        return sharding.max_over_ranks(x, device="cuda")
 
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")  # > 126 MB L2
 
@@ -212,7 +220,7 @@ def main() -> None:
     weights = inputs.policy_weights(w.policy, w.policy_seed) if w.policy else None
     pol = cp.policy(w.policy, weights) if w.policy else None
     n, T = w.n_envs, w.T
-    env_offset = rank * n  # weak scaling: every rank runs a full batch on its own env range
+    env_offset = sharding.weak_env_offset(n, rank)  # weak scaling: a full batch per rank, own env range
     ret = torch.empty(n, dtype=torch.float32, device="cuda")
     cnt = torch.empty(n, dtype=torch.int32, device="cuda")
     tot = torch.zeros(2, dtype=torch.int64, device="cuda")
@@ -227,16 +235,25 @@ def main() -> None:
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
+        for _ in range(10):  # load the GPU while the first clock samples are taken
+            rollout_step()
+        torch.cuda.synchronize()
     ms, launches = timed(rollout_step, args.steps, args.warmup)
     clocks = sampler.stop() if rank == 0 else {}
     ms_per_step = ms / args.steps
     value = world * n * T / (ms_per_step * 1e-3)
-    ops = ALG_OPS[pol_name]
-    ach = n * T * ops / (ms_per_step * 1e-3)
-    roofline = {"bound": "alu", "kernel": "rollout_kernel", "achieved": ach / 1e12, "peak": peak_inst / 1e12,
-                "unit": "Tinst/s", "frac": ach / peak_inst, "traffic": None,
-                "algorithmic_ops_per_env_step": ops,
-                "peak_source": f"148 SMs x 4 schedulers x 32 lanes x {peaks['sm_max_mhz']:.0f} MHz ({peaks['source']} max clock)"}
+    ops = ROLLOUT_OPS[pol_name + ("+streams" if w.streams else "")]
+    rate = n * T / (ms_per_step * 1e-3)  # per GPU
+    roofline = {"bound": "alu", "kernel": "rollout_kernel", "achieved": rate * ops["thread"] / 1e12,
+                "peak": peak_inst / 1e12, "unit": "Tinst/s", "frac": rate * ops["thread"] / peak_inst,
+                "issue_slot_frac": rate * ops["slot"] / peak_inst,
+                "traffic": ROLLOUT_DRAM_BYTES.get(pol_name + ("+streams" if w.streams else "")),
+                "traffic_note": "ncu dram bytes of one launch at 1,048,576 envs x 100 steps; the 8 B/env of "
+                                "per-env results stay in L2, stream outputs scale with N*T",
+                "thread_inst_per_env_step": ops["thread"], "issue_slots_per_env_step": ops["slot"],
+                "peak_source": f"148 SMs x 4 schedulers x 32 lanes x {peaks['sm_max_mhz']:.0f} MHz ({peaks['source']} max clock)",
+                "note": "frac counts instructions executed by active lanes only; issue_slot_frac counts whole "
+                        "warp instructions x 32 (what the schedulers issue)"}
     if w.streams:
         roofline["stream_write_gbs"] = n * T * 4.125 / (ms_per_step * 1e-3) / 1e9
         roofline["stream_write_frac_of_hbm"] = roofline["stream_write_gbs"] / peaks["hbm_gbs"]
@@ -274,8 +291,7 @@ def main() -> None:
                "sample": f"first {sample} envs x {T} steps of the workload, one pass, {dt:.2f} s",
                "returns_identical_to_gpu": same}
 
-    if world > 1:
-        dist.all_reduce(tot)  # the only exchange the path has: 16 bytes, outside the timed region
+    sharding.reduce_totals(tot)  # the only exchange the path has: 16 bytes, outside the timed region
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -332,7 +348,8 @@ def measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args) -> dict:
     out["fused_step_hbm"] = {"n_envs": n, "ms_per_launch": ms, "env_steps_per_sec": n / (ms * 1e-3),
                              "roofline": {"bound": "hbm", "kernel": "step_kernel", "achieved": gbs,
                                           "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs * 1e9 / hbm,
-                                          "traffic": None, "bytes_per_env_step": STEP_BYTES}}
+                                          "traffic": STEP_DRAM_BYTES_16M if n == 1 << 24 else None,
+                                          "bytes_per_env_step": STEP_BYTES}}
     # ladder at the same size
     ws = torch.empty(cp.cp_unfused_workspace_bytes(n), dtype=torch.uint8, device="cuda")
 
@@ -414,8 +431,9 @@ def measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args) -> dict:
         ms /= k
         pol_name = {0: "random", 1: "linear", 2: "mlp"}[w.policy]
         rate = n * T / (ms * 1e-3)
+        ops = ROLLOUT_OPS[pol_name + ("+streams" if w.streams else "")]
         entry = {"n_envs": n, "T": T, "policy": pol_name, "ms_per_launch": ms, "env_steps_per_sec": rate,
-                 "alu_frac": rate * ALG_OPS[pol_name] / peak_inst}
+                 "alu_frac": rate * ops["thread"] / peak_inst, "issue_slot_frac": rate * ops["slot"] / peak_inst}
         if w.streams:
             entry["stream_write_gbs"] = rate * 4.125 / 1e9
             entry["stream_write_frac_of_hbm"] = rate * 4.125 / hbm

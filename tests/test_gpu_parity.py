@@ -326,20 +326,84 @@ def test_policy_rollouts_against_oracle(cp, oracle, kind, pseed, n, T):
     assert np.array_equal(gd.sum(axis=0), r["ep_count"])
 
 
-def test_sampled_envs_of_large_policy_configs(cp, oracle):
-    """Configs 4 and 5 at their full env counts but fewer steps would not be the benchmark launch;
-    instead run the full launch shape on a slice of time and compare sampled env ranges."""
-    for name, T in (("c4", 64), ("c5", 48)):
+def test_full_size_policy_configs_on_sampled_envs(cp, oracle):
+    """Configs 4 (4,194,304 x 1,000, linear policy, reward plane + done bitmask) and 5
+    (16,777,216 x 200, MLP policy) exactly as bench.py launches them; the oracle recomputes
+    sampled env ranges one by one (results of an env do not depend on its neighbours)."""
+    for name in ("c4", "c5"):
         w = inputs.WORKLOADS[name]
         wts = inputs.policy_weights(w.policy, w.policy_seed)
-        n = w.n_envs
-        r = run_rollout(cp, n, T, w.seed, w.policy, wts, final=False)
-        for lo in (0, n // 2 - 1000, n - 4096):
-            m = 4096
-            o = oracle.rollout(m, T, w.seed, w.policy, wts, env_offset=lo, min_gap=True)
-            H.assert_returns_match(r["ep_return_sum"][lo:lo + m], r["ep_count"][lo:lo + m],
-                                   o["ep_return_sum"], o["ep_count"], o["min_gap"] < 1e-5, min_identical=0.998)
-        assert int(r["totals"][1]) == int(r["ep_count"].astype(np.int64).sum())
+        n, T = w.n_envs, w.T
+        words = (n + 31) // 32
+        outs = {"ep_return_sum": torch.empty(n, dtype=torch.float32, device="cuda"),
+                "ep_count": torch.empty(n, dtype=torch.int32, device="cuda"),
+                "totals": torch.zeros(2, dtype=torch.int64, device="cuda")}
+        if w.streams:
+            outs["reward_stream"] = torch.empty(T, n, dtype=torch.float32, device="cuda")
+            outs["done_bits"] = torch.empty(T, words, dtype=torch.int32, device="cuda")
+        cp.cp_rollout(n, T, w.seed, cp.policy(w.policy, wts), **outs)
+        torch.cuda.synchronize()
+        ret, cnt = host(outs["ep_return_sum"]), host(outs["ep_count"]).view(np.uint32)
+        m = 2048
+        for lo in (0, n // 2 - 1024, n - m):
+            o = oracle.rollout(m, T, w.seed, w.policy, wts, env_offset=lo, min_gap=True, done_bits=w.streams)
+            excuse = o["min_gap"] < 1e-5
+            H.assert_returns_match(ret[lo:lo + m], cnt[lo:lo + m], o["ep_return_sum"], o["ep_count"], excuse,
+                                   min_identical=0.998)
+            if w.streams:
+                gd = H.unpack_bits(host(outs["done_bits"][:, lo // 32:(lo + m) // 32]), m)
+                od = H.unpack_bits(o["done_bits"], m)
+                same_env = (ret[lo:lo + m] == o["ep_return_sum"]) & (cnt[lo:lo + m] == o["ep_count"])
+                assert np.array_equal(gd[:, same_env], od[:, same_env])
+                assert np.array_equal(gd.sum(axis=0), cnt[lo:lo + m])
+                assert bool((outs["reward_stream"][:, lo:lo + m] == 1.0).all())
+        tot = host(outs["totals"]).view(np.uint64)
+        assert int(tot[1]) == int(cnt.astype(np.int64).sum())
+        assert int(tot[0]) == int(ret.astype(np.float64).sum())
+        if w.streams:  # every row of the reward plane was written, every done bit is accounted for
+            assert float(outs["reward_stream"].min()) == 1.0 and float(outs["reward_stream"].max()) == 1.0
+        del outs
+        torch.cuda.empty_cache()
+
+
+def test_config2_step_path_at_full_size(cp, oracle):
+    """65,536 envs x 1,000 steps through per-step launches (state round-trips HBM every step):
+    equal to the one-launch rollout bit for bit, whose returns are checked against the oracle;
+    and the per-op ladder equals the fused step over 20 consecutive steps at this size."""
+    import os
+    w = inputs.WORKLOADS["c2"]
+    n, T = w.n_envs, w.T
+    roll = run_rollout(cp, n, T, w.seed)
+    planes = alloc_planes(n)
+    st = cp.cp_wrap(planes, n, w.seed)
+    cp.cp_fill_start(st)
+    reward = torch.empty(n, dtype=torch.float32, device="cuda")
+    done = torch.empty(n, dtype=torch.uint8, device="cuda")
+    done_count = torch.zeros(n, dtype=torch.int32, device="cuda")
+    for _ in range(T // 100):
+        for _ in range(100):
+            cp.cp_step(st, None, st, reward, done)
+            done_count += done  # torch only accumulates the library's output for the comparison
+    torch.cuda.synchronize()
+    assert np.array_equal(host(planes[:, :n]), roll["final_state"])
+    assert np.array_equal(host(done_count).view(np.uint32), roll["ep_count"])
+    o = oracle.rollout(n, T, w.seed, nthreads=os.cpu_count() or 1)
+    H.assert_returns_match(roll["ep_return_sum"], roll["ep_count"], o["ep_return_sum"], o["ep_count"])
+    # ladder vs fused step, 20 steps, ping-pong
+    a, b, c = alloc_planes(n), alloc_planes(n), alloc_planes(n)
+    sa, sb, sc = cp.cp_wrap(a, n, w.seed), cp.cp_wrap(b, n, w.seed), cp.cp_wrap(c, n, w.seed)
+    cp.cp_fill_start(sa)
+    c.copy_(a)
+    ws = torch.empty(cp.cp_unfused_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    done2 = torch.empty_like(done)
+    for k in range(10):
+        cp.cp_step_unfused(sa, None, sb, reward, done, ws)
+        cp.cp_step_unfused(sb, None, sa, reward, done, ws)
+        cp.cp_step(sc, None, sc, reward, done2)
+        cp.cp_step(sc, None, sc, reward, done2)
+    torch.cuda.synchronize()
+    assert torch.equal(a, c) and torch.equal(done, done2)
+    assert sa.info()["t"] == 20 == sc.info()["t"]
 
 
 @pytest.mark.parametrize("ept", [1, 2, 4])
