@@ -110,6 +110,12 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def workload_name(w) -> str:
+    pol = {0: "random", 1: "linear", 2: "mlp"}[w.policy]
+    return (f"{w.name}: {w.n_envs} envs x {w.T} steps per GPU, fused rollout, policy={pol}, seed={w.seed}"
+            + (", reward+done streams" if w.streams else ""))
+
+
 def host_cores() -> int:
     try:
         return len(os.sched_getaffinity(0))
@@ -141,8 +147,8 @@ def run_reference(args) -> None:
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{w.name}: {w.n_envs} envs x {w.T} steps, fused rollout, policy={w.policy}",
-                   "sample": f"first {sample} envs x {w.T} steps per step"},
+        "config": {"workload": workload_name(w), "envs_per_gpu": w.n_envs, "T": w.T,
+                   "sample": f"each step = the first {sample} envs x {w.T} steps on the host cores"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": f"first {sample} envs x {w.T} steps, {args.steps} repeats"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -235,8 +241,9 @@ def main() -> None:
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-        for _ in range(10):  # load the GPU while the first clock samples are taken
-            rollout_step()
+    t_load = time.perf_counter()
+    while time.perf_counter() - t_load < 1.5:  # keep the GPU loaded while nvidia-smi starts sampling
+        rollout_step()
         torch.cuda.synchronize()
     ms, launches = timed(rollout_step, args.steps, args.warmup)
     clocks = sampler.stop() if rank == 0 else {}
@@ -297,8 +304,7 @@ def main() -> None:
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": f"{w.name}: {n} envs x {T} steps per GPU, fused rollout, policy={pol_name}, "
-                                   f"seed={w.seed}" + (", reward+done streams" if w.streams else ""),
+            "config": {"workload": workload_name(w),
                        "l2": "flushed between iterations (256 MiB fill outside the timed events)",
                        "envs_per_gpu": n, "T": T},
             "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "roofline": roofline,

@@ -206,7 +206,10 @@ int cp_rollout_from(cp_state *state, int64_t T, uint32_t *ep_len, const cp_polic
 /* End-to-end forms with HOST buffers (pinned memory recommended): device staging buffers
  * are owned by the library (grown on demand, released by cp_shutdown); the calls copy in,
  * launch, copy out and SYNCHRONISE the stream before returning.
- * cp_rollout_host: h_ep_return_sum [n_envs], h_ep_count [n_envs], h_totals [2] (overwritten). */
+ * cp_rollout_host: h_ep_return_sum [n_envs], h_ep_count [n_envs], h_totals [2] (overwritten).
+ * When the two per-env buffers are page-locked (cudaHostAlloc / cudaHostRegister, e.g. torch
+ * pinned tensors) the kernel stores into them directly over PCIe while it runs, so the transfer
+ * overlaps the computation; pageable buffers are filled by copies after the kernel. */
 int cp_rollout_host(int64_t n_envs, int64_t T, uint32_t seed, const cp_policy *policy,
                     float *h_ep_return_sum, uint32_t *h_ep_count, uint64_t *h_totals);
 /* cp_step_host: h_planes_in/out [4][n_envs] (stride n_envs), h_action [n_envs] or NULL,
@@ -223,7 +226,9 @@ void cp_set_stream(void *cuda_stream);
  * default 256), "rollout_ept" (environments per thread: 1, 2 or 4; 0 = default, 2 for large
  * batches), "rollout_ctas_per_sm" (0 = default: one 32*ept-environment task per warp and as many
  * CTAs as that takes; k > 0 = persistent grid of k CTAs per SM looping over tasks), "step_block"
- * (32..256, default 64). Returns CP_EINVAL for an unknown key or value. */
+ * (32..256, default 64), "step_vec_min_envs" (batches smaller than this use the one-env-per-thread
+ * step kernel even when the four-envs-per-thread vector form is possible; default 262144).
+ * Returns CP_EINVAL for an unknown key or value. */
 int cp_tune(const char *key, int value);
 
 /* Number of kernels this library has launched in this process (all threads). */

@@ -182,6 +182,23 @@ int staging_reserve(size_t bytes, void **out) {
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Device-side address of a page-locked host range [p, p + bytes), or nullptr if the range is
+// pageable (or not wholly inside one registered allocation).
+void *device_view_of_pinned(void *p, size_t bytes) {
+    cudaPointerAttributes a0, a1;
+    if (cudaPointerGetAttributes(&a0, p) != cudaSuccess || a0.type != cudaMemoryTypeHost || !a0.devicePointer) {
+        (void)cudaGetLastError();
+        return nullptr;
+    }
+    if (cudaPointerGetAttributes(&a1, static_cast<char *>(p) + bytes - 1) != cudaSuccess ||
+        a1.type != cudaMemoryTypeHost || !a1.devicePointer ||
+        static_cast<char *>(a1.devicePointer) - static_cast<char *>(a0.devicePointer) != (ptrdiff_t)(bytes - 1)) {
+        (void)cudaGetLastError();
+        return nullptr;
+    }
+    return a0.devicePointer;
+}
+
 }  // namespace
 
 // Accessors for entry points that live in other translation units.
@@ -288,8 +305,9 @@ int cp_step(cp_state *state, const uint8_t *action, cp_state *out_state, float *
     if (reward && !is_aligned(reward, 4)) return fail(CP_EINVAL, "reward is not float-aligned");
     cp::StepParams p;
     fill_step_params(p, state, out_state, action, reward, done);
-    const bool vec = state_vec_ok(state) && state_vec_ok(out_state) && (!reward || is_aligned(reward, 16)) &&
-                     (!done || is_aligned(done, 4)) && (!action || is_aligned(action, 4));
+    const bool vec = state->n >= cp::g_tuning.step_vec_min_envs && state_vec_ok(state) && state_vec_ok(out_state) &&
+                     (!reward || is_aligned(reward, 16)) && (!done || is_aligned(done, 4)) &&
+                     (!action || is_aligned(action, 4));
     cudaError_t e = cp::launch_step(p, vec, tl_stream);
     if (e != cudaSuccess) return cuda_fail(e, "step launch");
     advance(state, out_state, 1);
@@ -366,21 +384,30 @@ int cp_rollout_host(int64_t n_envs, int64_t T, uint32_t seed, const cp_policy *p
     if (rc != CP_OK) return rc;
     if (!h_ep_return_sum || !h_ep_count || !h_totals) return fail(CP_EINVAL, "a host output pointer is NULL");
     std::lock_guard<std::mutex> lock(g_staging.mu);
-    const size_t per = round_up((size_t)n_envs * 4, 256);
+    // Page-locked host buffers are addressable from the device: the kernel then stores each env's
+    // two results straight into host memory as its warp finishes (8 B/env spread over the whole
+    // launch), instead of a device buffer plus a copy after the kernel. Pageable buffers take the
+    // staged route.
+    float *d_ret = static_cast<float *>(device_view_of_pinned(h_ep_return_sum, (size_t)n_envs * 4));
+    uint32_t *d_cnt = static_cast<uint32_t *>(device_view_of_pinned(h_ep_count, (size_t)n_envs * 4));
+    const bool direct = d_ret && d_cnt;
+    const size_t per = direct ? 0 : round_up((size_t)n_envs * 4, 256);
     void *buf;
     if ((rc = staging_reserve(2 * per + 256, &buf)) != CP_OK) return rc;
     char *base = static_cast<char *>(buf);
     cp_returns r;
     memset(&r, 0, sizeof r);
-    r.ep_return_sum = reinterpret_cast<float *>(base);
-    r.ep_count = reinterpret_cast<uint32_t *>(base + per);
+    r.ep_return_sum = direct ? d_ret : reinterpret_cast<float *>(base);
+    r.ep_count = direct ? d_cnt : reinterpret_cast<uint32_t *>(base + per);
     r.totals = reinterpret_cast<uint64_t *>(base + 2 * per);
     cudaError_t e = cudaMemsetAsync(r.totals, 0, 16, tl_stream);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
     if ((rc = rollout_impl(0, n_envs, T, seed, 0, policy, &r, nullptr, 0, nullptr, 0, nullptr)) != CP_OK) return rc;
-    e = cudaMemcpyAsync(h_ep_return_sum, r.ep_return_sum, (size_t)n_envs * 4, cudaMemcpyDeviceToHost, tl_stream);
-    if (e == cudaSuccess)
-        e = cudaMemcpyAsync(h_ep_count, r.ep_count, (size_t)n_envs * 4, cudaMemcpyDeviceToHost, tl_stream);
+    if (!direct) {
+        e = cudaMemcpyAsync(h_ep_return_sum, r.ep_return_sum, (size_t)n_envs * 4, cudaMemcpyDeviceToHost, tl_stream);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(h_ep_count, r.ep_count, (size_t)n_envs * 4, cudaMemcpyDeviceToHost, tl_stream);
+    }
     if (e == cudaSuccess) e = cudaMemcpyAsync(h_totals, r.totals, 16, cudaMemcpyDeviceToHost, tl_stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(tl_stream);
     return e == cudaSuccess ? CP_OK : cuda_fail(e, "rollout copy-out");
@@ -444,6 +471,9 @@ int cp_tune(const char *key, int value) {
     } else if (!strcmp(key, "step_block")) {
         if (value < 32 || value > 256 || value % 32) return fail(CP_EINVAL, "step_block must be 32..256, multiple of 32");
         cp::g_tuning.step_block = value;
+    } else if (!strcmp(key, "step_vec_min_envs")) {
+        if (value < 0) return fail(CP_EINVAL, "step_vec_min_envs must be >= 0");
+        cp::g_tuning.step_vec_min_envs = value;
     } else {
         return fail(CP_EINVAL, "unknown tuning key '%s'", key);
     }

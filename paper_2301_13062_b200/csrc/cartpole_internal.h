@@ -47,6 +47,10 @@ struct LaunchTuning {
     int rollout_ept = 0;          // 0: chosen per policy
     int rollout_ctas_per_sm = 0;  // 0: one task per warp (non-persistent grid)
     int step_block = 64;
+    // Below this many envs the one-env-per-thread kernel is used: a small batch is latency-bound,
+    // and four envs in sequence per thread take longer than four times as many threads
+    // (65,536 envs, graph replay: 1.9 us vs 2.5 us per launch; equal at 262,144; slower above).
+    int step_vec_min_envs = 262144;
 };
 extern LaunchTuning g_tuning;
 

@@ -22,6 +22,9 @@ def cp():
     return binding
 
 
+VEC_MIN_DEFAULT = 262144  # library default of "step_vec_min_envs"
+
+
 def dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
@@ -98,18 +101,28 @@ def test_step_matches_oracle(cp, oracle, spread, n):
     z = inputs.random_states(n, seed=n + len(spread), spread=spread)
     for action, off, t in ((None, 0, 0), (None, 12345, 17), (inputs.random_actions(n, 3), 0, 5)):
         want = oracle.step(z, seed=1, t=t, action_u8=action, env_offset=off, want_pre_reset=True)
-        got_state, got_reward, got_done = gpu_step(cp, z, 1, t, action, off)
-        stats = H.assert_step_matches(want, z, got_state, got_reward, got_done)
-        if spread in ("start", "live") and n >= 1025:
-            assert stats["bit_exact_fraction"] > 0.8
+        for vec_min in (0, 1 << 30):  # four-envs-per-thread vector kernel, one-env-per-thread kernel
+            cp.cp_tune("step_vec_min_envs", vec_min)
+            try:
+                got_state, got_reward, got_done = gpu_step(cp, z, 1, t, action, off)
+            finally:
+                cp.cp_tune("step_vec_min_envs", VEC_MIN_DEFAULT)
+            stats = H.assert_step_matches(want, z, got_state, got_reward, got_done)
+            if spread in ("start", "live") and n >= 1025:
+                assert stats["bit_exact_fraction"] > 0.8
 
 
 def test_step_scalar_path_and_in_place_equal_vector_path(cp):
     n = 4099
     z = inputs.random_states(n, seed=2, spread="edge")
     a = inputs.random_actions(n, 9)
-    base = gpu_step(cp, z, 4, 3, None, 100)
-    for kwargs in ({"stride": n}, {"stride": n + 1}, {"in_place": True}, {"stride": n, "in_place": True}):
+    cp.cp_tune("step_vec_min_envs", 0)  # vector kernel for the aligned layout
+    try:
+        base = gpu_step(cp, z, 4, 3, None, 100)
+        assert all(np.array_equal(b, o) for b, o in zip(base, gpu_step(cp, z, 4, 3, None, 100, in_place=True)))
+    finally:
+        cp.cp_tune("step_vec_min_envs", VEC_MIN_DEFAULT)
+    for kwargs in ({}, {"stride": n}, {"stride": n + 1}, {"in_place": True}, {"stride": n, "in_place": True}):
         other = gpu_step(cp, z, 4, 3, None, 100, **kwargs)
         for b, o in zip(base, other):
             assert np.array_equal(b.view(np.uint8), o.view(np.uint8)), kwargs
@@ -176,6 +189,7 @@ def test_nan_inf_states_do_not_fault(cp):
 # ------------------------------------------------------------------ ladder == fused step
 @pytest.mark.parametrize("n", [1, 33, 1025, 50001])
 def test_ladder_equals_fused_step_bitwise(cp, n):
+    cp.cp_tune("step_vec_min_envs", 0 if n % 2 else VEC_MIN_DEFAULT)  # both fused kernels get compared
     before = cp.cp_launch_count()
     for spread in ("edge", "wide", "start"):
         z = inputs.random_states(n, seed=n, spread=spread)
@@ -184,6 +198,7 @@ def test_ladder_equals_fused_step_bitwise(cp, n):
             ladder = gpu_step(cp, z, 7, 11, action, 5, unfused=True)
             for f, l in zip(fused, ladder):
                 assert np.array_equal(f.view(np.uint8), l.view(np.uint8))
+    cp.cp_tune("step_vec_min_envs", VEC_MIN_DEFAULT)
     # 3 spreads x (46 + 45 ladder launches + 2 fused launches)
     assert cp.cp_launch_count() - before == 3 * (46 + 45 + 2)
 
@@ -501,13 +516,17 @@ def test_host_buffer_entry_points(cp, oracle):
     wts = inputs.policy_weights(1, 1)
     for kind, w in ((0, None), (1, wts)):
         ref = run_rollout(cp, n, T, 4, kind, w)
-        h_ret = torch.empty(n, dtype=torch.float32).pin_memory()
-        h_cnt = torch.empty(n, dtype=torch.int32).pin_memory()
-        h_tot = torch.empty(2, dtype=torch.int64).pin_memory()
-        cp.cp_rollout_host(n, T, 4, cp.policy(kind, w) if kind else None, h_ret, h_cnt, h_tot)
-        assert np.array_equal(h_ret.numpy(), ref["ep_return_sum"])
-        assert np.array_equal(h_cnt.numpy().view(np.uint32), ref["ep_count"])
-        assert np.array_equal(h_tot.numpy().view(np.uint64), ref["totals"])
+        # page-locked buffers (written by the kernel directly) and pageable ones (staged copy)
+        for pin in (True, False):
+            h_ret = torch.full((n,), -1.0, dtype=torch.float32)
+            h_cnt = torch.full((n,), -1, dtype=torch.int32)
+            h_tot = torch.full((2,), -1, dtype=torch.int64)
+            if pin:
+                h_ret, h_cnt, h_tot = h_ret.pin_memory(), h_cnt.pin_memory(), h_tot.pin_memory()
+            cp.cp_rollout_host(n, T, 4, cp.policy(kind, w) if kind else None, h_ret, h_cnt, h_tot)
+            assert np.array_equal(h_ret.numpy(), ref["ep_return_sum"])
+            assert np.array_equal(h_cnt.numpy().view(np.uint32), ref["ep_count"])
+            assert np.array_equal(h_tot.numpy().view(np.uint64), ref["totals"])
     z = inputs.random_states(n, seed=1, spread="edge")
     a = inputs.random_actions(n, 2)
     for action in (None, a):
