@@ -201,12 +201,14 @@ def main() -> None:
 
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")  # > 126 MB L2
 
-    def timed(fn, steps, warmup, flush=True):
+    def timed(fn, steps, warmup, flush=True, all_ranks=True):
         """Sum of per-iteration CUDA-event times on the launching stream (ms), L2 flushed
-        between iterations outside the timed events; max over ranks."""
+        between iterations outside the timed events; barrier on both sides and max over ranks
+        (all_ranks=False: a measurement only rank 0 makes, no collective)."""
+        sync = barrier if all_ranks else torch.cuda.synchronize
         for _ in range(warmup):
             fn()
-        barrier()
+        sync()
         evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
         launches0 = cp.cp_launch_count()
         for a, b in evs:
@@ -215,10 +217,10 @@ def main() -> None:
             a.record()
             fn()
             b.record()
-        barrier()
+        sync()
         launches = cp.cp_launch_count() - launches0
         ms = sum(a.elapsed_time(b) for a, b in evs)
-        return max_over_ranks(ms), launches
+        return (max_over_ranks(ms) if all_ranks else ms), launches
 
     # ---- headline: fused rollout ----
     w = inputs.WORKLOADS[args.workload]
@@ -278,12 +280,13 @@ def main() -> None:
     e2e = {"value": world * n * T / (e2e_ms * 1e-3), "unit": UNIT,
            "h2d_bytes_per_step": int(4 * inputs.N_WEIGHTS[w.policy]) + 24, "d2h_bytes_per_step": 8 * n + 16,
            "ms_per_step": e2e_ms,
-           "note": "cp_rollout_host: host scalars (n_envs, T, seed) and policy weights in, per-env returns and "
-                   "counts copied to pinned host memory, stream synchronised, every step"}
+           "note": "cp_rollout_host: host scalars (n_envs, T, seed) and policy weights in; per-env returns and "
+                   "counts land in pinned host memory (stored there by the kernel over PCIe while it runs), "
+                   "totals copied back, stream synchronised, every step"}
 
     paths = {}
     if not args.no_paths and rank == 0:
-        paths = measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args)
+        paths = measure_paths(cp, inputs, torch, lambda *a, **k: timed(*a, all_ranks=False, **k), peaks, peak_inst, args)
 
     cpu = None
     if not args.no_cpu and rank == 0:

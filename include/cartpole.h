@@ -251,6 +251,15 @@ int cp_selftest_sincos_accuracy(uint32_t lo_bits, uint32_t hi_bits, uint64_t *ou
  * they are used. out DEVICE [4] uint64, caller zeroes; every count must come back 0. */
 int cp_selftest_arith(uint64_t *out);
 
+/* Diagnostics: for states inside the range episodes visit (|theta| <= 0.25, |theta_dot| <= 20) the
+ * kernels compute the angular acceleration's quotient with the hardware reciprocal plus one exact
+ * correction instead of the general division. This compares the two over the whole operand domain
+ * of such states: every den_step-th float32 denominator in [0.6210, 0.6242] (53,688 values at
+ * den_step = 1) times every float32 numerator of magnitude in [2, 32), both signs (about two
+ * seconds of GPU time at den_step = 1). out DEVICE [2] uint64, caller zeroes:
+ * out[0] += mismatching quotients (must stay 0), out[1] += (denominator, |numerator|) pairs tested. */
+int cp_selftest_tame_div(uint32_t den_step, uint64_t *out);
+
 const char *cp_last_error(void);
 const char *cp_version(void);
 

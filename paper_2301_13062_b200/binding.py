@@ -26,7 +26,7 @@ EXPORTS = [
     "cp_fill_start", "cp_set_time", "cp_free", "cp_state_info", "cp_actions", "cp_rollout_shard",
     "cp_rollout_from", "cp_rollout_host", "cp_step_host", "cp_shutdown", "cp_set_stream", "cp_tune",
     "cp_launch_count", "cp_selftest_sincos", "cp_last_error", "cp_version", "cp_step_unfused_noalloc",
-    "cp_selftest_sincos_accuracy", "cp_selftest_arith", "cp_step_repeat",
+    "cp_selftest_sincos_accuracy", "cp_selftest_arith", "cp_step_repeat", "cp_selftest_tame_div",
 ]
 CP_NOALLOC_MAX_ENVS = 65536
 
@@ -84,6 +84,7 @@ def lib() -> C.CDLL:
             "cp_selftest_sincos": (i32, [u32, u32, p]),
             "cp_selftest_sincos_accuracy": (i32, [u32, u32, p]),
             "cp_selftest_arith": (i32, [p]),
+            "cp_selftest_tame_div": (i32, [u32, p]),
             "cp_last_error": (C.c_char_p, []),
             "cp_version": (C.c_char_p, []),
         }
@@ -317,6 +318,12 @@ def cp_selftest_arith(out) -> None:
     import torch
     _use_current_stream()
     _check(lib().cp_selftest_arith(_dptr(out, torch.int64)))
+
+
+def cp_selftest_tame_div(den_step: int, out) -> None:
+    import torch
+    _use_current_stream()
+    _check(lib().cp_selftest_tame_div(den_step, _dptr(out, torch.int64)))
 
 
 def cp_version() -> str:

@@ -503,6 +503,13 @@ int cp_selftest_arith(uint64_t *out) {
     return e == cudaSuccess ? CP_OK : cuda_fail(e, "self-test launch");
 }
 
+int cp_selftest_tame_div(uint32_t den_step, uint64_t *out) {
+    if (!out || !is_aligned(out, 8)) return fail(CP_EINVAL, "out is NULL or misaligned");
+    if (den_step == 0) return fail(CP_EINVAL, "den_step must be >= 1");
+    cudaError_t e = cp::launch_tame_div_selftest(den_step, reinterpret_cast<unsigned long long *>(out), tl_stream);
+    return e == cudaSuccess ? CP_OK : cuda_fail(e, "self-test launch");
+}
+
 const char *cp_last_error(void) { return tl_error; }
 const char *cp_version(void) { return "cartpole-b200 0.1 (sm_100a)"; }
 

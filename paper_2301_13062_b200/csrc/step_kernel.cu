@@ -7,6 +7,8 @@
 // done (+ 1 B action when supplied). Vector form: each thread owns 4 consecutive
 // environments, i.e. one float4 per plane, so a warp moves 512 B per plane per
 // access and keeps 4 x 16 B loads in flight per thread.
+#include <cstring>
+
 #include "cartpole_device.cuh"
 #include "cartpole_internal.h"
 
@@ -255,6 +257,43 @@ __global__ void arith_selftest_kernel(unsigned long long *out) {
         atomicAdd(out + 2, b2);
         atomicAdd(out + 3, b3);
     }
+}
+
+// ---- self-test: the tame-state division against IEEE division over its whole operand domain ----
+// den: every den_step-th float in [kTameDenLo, kTameDenHi]; num: every float in [2, 32) (the
+// sequence is odd in num, so negative numerators need no separate pass).
+// out[0] += mismatches, out[1] += pairs tested.
+__global__ void tame_div_selftest_kernel(uint32_t den_lo, uint32_t den_hi, uint32_t den_step,
+                                         unsigned long long *out) {
+    unsigned long long bad = 0, pairs = 0;
+    for (uint64_t db = (uint64_t)den_lo + (uint64_t)blockIdx.y * den_step; db <= den_hi;
+         db += (uint64_t)gridDim.y * den_step) {
+        const float den = __uint_as_float((uint32_t)db);
+        for (uint32_t nb = 0x40000000u + blockIdx.x * blockDim.x + threadIdx.x; nb < 0x42000000u;
+             nb += gridDim.x * blockDim.x) {
+            const float num = __uint_as_float(nb);
+            bad += __float_as_uint(div_tame(num, den)) != __float_as_uint(__fdiv_rn(num, den));
+            bad += __float_as_uint(div_tame(-num, den)) != (__float_as_uint(__fdiv_rn(num, den)) ^ 0x80000000u);
+            pairs += 1;
+        }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        bad += __shfl_down_sync(0xffffffffu, bad, o);
+        pairs += __shfl_down_sync(0xffffffffu, pairs, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        if (bad) atomicAdd(out, bad);
+        atomicAdd(out + 1, pairs);
+    }
+}
+
+cudaError_t launch_tame_div_selftest(uint32_t den_step, unsigned long long *out, cudaStream_t s) {
+    uint32_t lo, hi;
+    memcpy(&lo, &kTameDenLo, 4);
+    memcpy(&hi, &kTameDenHi, 4);
+    tame_div_selftest_kernel<<<dim3(sm_count() * 2, 64), 256, 0, s>>>(lo, hi, den_step, out);
+    count_launch();
+    return cudaGetLastError();
 }
 
 cudaError_t launch_arith_selftest(unsigned long long *out, cudaStream_t s) {

@@ -572,6 +572,23 @@ def test_exact_shortcuts_equal_the_operations_they_replace(cp):
     assert [int(v) for v in out.cpu()] == [0, 0, 0, 0]
 
 
+def test_tame_state_division_equals_ieee_division_on_its_whole_domain(cp):
+    """53,688 denominators x 33,554,432 numerators x both signs, every pair (about 2 s)."""
+    out = torch.zeros(2, dtype=torch.int64, device="cuda")
+    cp.cp_selftest_tame_div(1, out)
+    torch.cuda.synchronize()
+    bad, pairs = (int(v) for v in out.cpu())
+    lo, hi = (int(np.float32(v).view(np.uint32)) for v in (0.6210, 0.6242))
+    assert pairs == (hi - lo + 1) * (1 << 25)
+    assert bad == 0
+    # the domain really contains what a tame state produces: den at c = 1 and c = cos(0.25), |num| bounds
+    m, ft = np.float32(1.1), np.float32(4.0 / 3.0)
+    for c in (np.float32(1.0), np.float32(np.cos(0.25)) - np.float32(1e-6)):
+        den = np.float32(0.5) * (ft - (np.float32(0.1) * (c * c)) / m)
+        assert 0.6210 < float(den) < 0.6242
+    assert 0.9689 * 5.05 / 1.1 - 9.8 * 0.2475 > 2.0 and 9.8 * 0.2475 + 14.95 / 1.1 < 32.0
+
+
 def test_stream_selection(cp):
     n, T = 2000, 30
     ref = run_rollout(cp, n, T, 1)
