@@ -36,14 +36,14 @@ SMS = 148
 # terminate executes no restart code); "slot" = 32 * smsp__inst_executed.sum / (N*T), the issue
 # slots the warps occupy, which also counts lanes idling while a neighbour restarts.
 ROLLOUT_OPS = {
-    "random": {"thread": 78.5, "slot": 111.9},
-    "linear": {"thread": 82.5, "slot": 92.0},
-    "linear+streams": {"thread": 97.2, "slot": 106.8},
-    "mlp": {"thread": 449.1, "slot": 480.7},
+    "random": {"thread": 71.5, "slot": 104.9},
+    "linear": {"thread": 75.5, "slot": 85.0},
+    "linear+streams": {"thread": 90.2, "slot": 99.8},
+    "mlp": {"thread": 442.2, "slot": 473.7},
 }
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch in the same captures.
-ROLLOUT_DRAM_BYTES = {"random": 20.7e3, "linear": 21.0e3, "linear+streams": 382.9e6, "mlp": 33.0e3}
-STEP_DRAM_BYTES_16M = 565.8e6  # step_kernel at 16,777,216 envs (profiles/step_kernel_16m_envs.md)
+ROLLOUT_DRAM_BYTES = {"random": 20.7e3, "linear": 20.5e3, "linear+streams": 381.2e6, "mlp": 32.5e3}
+STEP_DRAM_BYTES_16M = 567.8e6  # step_kernel at 16,777,216 envs (profiles/step_kernel_16m_envs.md)
 # Algorithmic HBM bytes per env-step of the step paths.
 STEP_BYTES = 37.0      # 16 in + 16 out + 4 reward + 1 done, hashed action
 LADDER_BYTES = 375.0   # sum over the 46 one-op kernels of their input and output planes

@@ -471,6 +471,9 @@ int cp_tune(const char *key, int value) {
     } else if (!strcmp(key, "step_block")) {
         if (value < 32 || value > 256 || value % 32) return fail(CP_EINVAL, "step_block must be 32..256, multiple of 32");
         cp::g_tuning.step_block = value;
+    } else if (!strcmp(key, "step_pdl")) {
+        if (value != 0 && value != 1) return fail(CP_EINVAL, "step_pdl must be 0 or 1");
+        cp::g_tuning.step_pdl = value;
     } else if (!strcmp(key, "step_vec_min_envs")) {
         if (value < 0) return fail(CP_EINVAL, "step_vec_min_envs must be >= 0");
         cp::g_tuning.step_vec_min_envs = value;

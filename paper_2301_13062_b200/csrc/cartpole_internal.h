@@ -51,6 +51,10 @@ struct LaunchTuning {
     // and four envs in sequence per thread take longer than four times as many threads
     // (65,536 envs, graph replay: 1.9 us vs 2.5 us per launch; equal at 262,144; slower above).
     int step_vec_min_envs = 262144;
+    // 1: launch the step kernel with programmatic stream serialization, so that a launch's
+    // memory-independent preamble overlaps the tail of the launch before it (same stream).
+    // Measured per launch, 65,536 envs: 4.10 -> 2.38 us issued eagerly, 2.01 -> 1.46 us from a graph.
+    int step_pdl = 1;
 };
 extern LaunchTuning g_tuning;
 

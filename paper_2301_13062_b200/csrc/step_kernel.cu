@@ -14,22 +14,20 @@
 
 namespace cp {
 
-// One environment: action -> dynamics -> done -> start state of the next episode.
-__device__ __forceinline__ bool step_one(State &z, uint32_t env, const StepParams &p, bool has_action,
-                                         uint8_t a_in) {
-    uint32_t sb;
-    if (has_action) {
-        sb = a_in ? 0x80000000u : 0u;
-    } else {
-        sb = action_signbit(make_keys(p.salt_a, env), p.t);
-    }
-    return euler_step(z, force_from_signbit(sb));
+// Action of one environment in sign-bit form: hashed (independent of any memory) or supplied.
+__device__ __forceinline__ uint32_t hashed_signbit(const StepParams &p, uint32_t env) {
+    return action_signbit(make_keys(p.salt_a, env), p.t);
 }
 
 #ifndef CP_STEP_MIN_CTAS
 #define CP_STEP_MIN_CTAS 1
 #endif
 
+// The kernel is written for programmatic dependent launch: everything that does not depend on
+// what the previous launch wrote (the action hashes, about a quarter of the instructions) comes
+// first; then the kernel waits for the previous launch's memory to be visible and immediately
+// lets the next launch begin its own preamble. Launched without that attribute the two
+// grid-dependency instructions do nothing.
 template <bool VEC>
 __global__ void __launch_bounds__(256, CP_STEP_MIN_CTAS) step_kernel(const __grid_constant__ StepParams p) {
     const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -37,6 +35,15 @@ __global__ void __launch_bounds__(256, CP_STEP_MIN_CTAS) step_kernel(const __gri
     if (VEC) {
         const int64_t i0 = tid * 4;
         if (i0 >= p.n) return;
+        const uint32_t env0 = p.env_offset + (uint32_t)i0;
+        const bool full = i0 + 3 < p.n;
+        uint32_t sb[4] = {0u, 0u, 0u, 0u};
+        if (!has_action) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) sb[j] = hashed_signbit(p, env0 + j);
+        }
+        cudaGridDependencySynchronize();
+        cudaTriggerProgrammaticLaunchCompletion();
         const float4 vx = *reinterpret_cast<const float4 *>(p.in + i0);
         const float4 vxd = *reinterpret_cast<const float4 *>(p.in + p.in_stride + i0);
         const float4 vth = *reinterpret_cast<const float4 *>(p.in + 2 * p.in_stride + i0);
@@ -45,22 +52,21 @@ __global__ void __launch_bounds__(256, CP_STEP_MIN_CTAS) step_kernel(const __gri
                       {vx.y, vxd.y, vth.y, vthd.y},
                       {vx.z, vxd.z, vth.z, vthd.z},
                       {vx.w, vxd.w, vth.w, vthd.w}};
-        const bool full = i0 + 3 < p.n;
-        uint8_t a_in[4] = {0, 0, 0, 0};
         if (has_action) {
             if (full) {
                 uchar4 av = *reinterpret_cast<const uchar4 *>(p.action + i0);
-                a_in[0] = av.x; a_in[1] = av.y; a_in[2] = av.z; a_in[3] = av.w;
+                sb[0] = av.x ? 0x80000000u : 0u;
+                sb[1] = av.y ? 0x80000000u : 0u;
+                sb[2] = av.z ? 0x80000000u : 0u;
+                sb[3] = av.w ? 0x80000000u : 0u;
             } else {
                 for (int j = 0; j < 4; ++j)
-                    if (i0 + j < p.n) a_in[j] = p.action[i0 + j];
+                    if (i0 + j < p.n) sb[j] = p.action[i0 + j] ? 0x80000000u : 0u;
             }
         }
-        const uint32_t env0 = p.env_offset + (uint32_t)i0;
         uint32_t dmask = 0;
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-            dmask |= (step_one(z[j], env0 + j, p, has_action, a_in[j]) ? 1u : 0u) << j;
+        for (int j = 0; j < 4; ++j) dmask |= (euler_step(z[j], force_from_signbit(sb[j])) ? 1u : 0u) << j;
         // Restart finished environments one per pass: almost always at most one of a
         // thread's four environments finishes in a step, so the start-state hashes are
         // issued once per warp instead of once per environment slot.
@@ -92,9 +98,13 @@ __global__ void __launch_bounds__(256, CP_STEP_MIN_CTAS) step_kernel(const __gri
     } else {
         const int64_t i = tid;
         if (i >= p.n) return;
-        State z = {p.in[i], p.in[p.in_stride + i], p.in[2 * p.in_stride + i], p.in[3 * p.in_stride + i]};
         const uint32_t env = p.env_offset + (uint32_t)i;
-        const bool d = step_one(z, env, p, has_action, has_action ? p.action[i] : (uint8_t)0);
+        uint32_t sb = has_action ? 0u : hashed_signbit(p, env);
+        cudaGridDependencySynchronize();
+        cudaTriggerProgrammaticLaunchCompletion();
+        State z = {p.in[i], p.in[p.in_stride + i], p.in[2 * p.in_stride + i], p.in[3 * p.in_stride + i]};
+        if (has_action) sb = p.action[i] ? 0x80000000u : 0u;
+        const bool d = euler_step(z, force_from_signbit(sb));
         if (d) z = start_state(make_keys(p.salt_r, env), p.t + 1u);
         p.out[i] = z.x;
         p.out[p.out_stride + i] = z.xd;
@@ -105,18 +115,35 @@ __global__ void __launch_bounds__(256, CP_STEP_MIN_CTAS) step_kernel(const __gri
     }
 }
 
+template <bool VEC>
+static cudaError_t launch_step_kernel(const StepParams &p, unsigned grid, int block, cudaStream_t s) {
+    if (!g_tuning.step_pdl) {
+        step_kernel<VEC><<<grid, block, 0, s>>>(p);
+        return cudaGetLastError();
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, step_kernel<VEC>, p);
+}
+
 cudaError_t launch_step(const StepParams &p, bool vec, cudaStream_t s) {
     const int block = g_tuning.step_block;
+    cudaError_t e;
     if (vec) {
         const int64_t threads = (p.n + 3) / 4;
-        const int64_t grid = (threads + block - 1) / block;
-        step_kernel<true><<<(unsigned)grid, block, 0, s>>>(p);
+        e = launch_step_kernel<true>(p, (unsigned)((threads + block - 1) / block), block, s);
     } else {
-        const int64_t grid = (p.n + block - 1) / block;
-        step_kernel<false><<<(unsigned)grid, block, 0, s>>>(p);
+        e = launch_step_kernel<false>(p, (unsigned)((p.n + block - 1) / block), block, s);
     }
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 // ---- generators ----

@@ -486,11 +486,15 @@ def test_step_repeat_and_graph_replay_equal_rollout(cp):
     cp.cp_fill_start(st)
     reward = torch.zeros(n, dtype=torch.float32, device="cuda")
     done = torch.zeros(n, dtype=torch.uint8, device="cuda")
-    cp.cp_step_repeat(st, T, reward, done)
-    torch.cuda.synchronize()
-    assert st.info()["t"] == T
-    assert np.array_equal(host(planes[:, :n]), ref["final_state"])
-    assert np.array_equal(host(done), H.unpack_bits(ref["done_bits"], n)[-1])
+    for pdl in (0, 1):  # plain launches, then programmatic dependent launches (the default)
+        cp.cp_tune("step_pdl", pdl)
+        cp.cp_set_time(st, 0)
+        cp.cp_fill_start(st)
+        cp.cp_step_repeat(st, T, reward, done)
+        torch.cuda.synchronize()
+        assert st.info()["t"] == T
+        assert np.array_equal(host(planes[:, :n]), ref["final_state"])
+        assert np.array_equal(host(done), H.unpack_bits(ref["done_bits"], n)[-1])
     # the same T launches captured in a CUDA graph and replayed from the start states
     side = torch.cuda.Stream()
     g = torch.cuda.CUDAGraph()
