@@ -31,7 +31,7 @@ METRIC = "env_steps_per_sec"
 UNIT = "env-steps/s"
 SMS = 148
 # Work per env-step of each rollout variant, counted by ncu on 1,048,576 envs x 100 steps
-# (profiles/rollout_kernel_*.md): "thread" = smsp__thread_inst_executed.sum / (N*T), the
+# (summaries under profiles/): "thread" = smsp__thread_inst_executed.sum / (N*T), the
 # instructions environments actually execute (the algorithmic figure: an env that does not
 # terminate executes no restart code); "slot" = 32 * smsp__inst_executed.sum / (N*T), the issue
 # slots the warps occupy, which also counts lanes idling while a neighbour restarts.
@@ -43,7 +43,7 @@ ROLLOUT_OPS = {
 }
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch in the same captures.
 ROLLOUT_DRAM_BYTES = {"random": 20.7e3, "linear": 20.5e3, "linear+streams": 381.2e6, "mlp": 32.5e3}
-STEP_DRAM_BYTES_16M = 567.8e6  # step_kernel at 16,777,216 envs (profiles/step_kernel_16m_envs.md)
+STEP_DRAM_BYTES_16M = 567.8e6  # step_kernel at 16,777,216 envs, same kind of capture
 # Algorithmic HBM bytes per env-step of the step paths.
 STEP_BYTES = 37.0      # 16 in + 16 out + 4 reward + 1 done, hashed action
 LADDER_BYTES = 375.0   # sum over the 46 one-op kernels of their input and output planes

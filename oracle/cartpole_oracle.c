@@ -307,6 +307,8 @@ typedef struct {
     float *final_state;      /* [4][n] or NULL */
     float *trajectory;       /* [T][4][n] or NULL: state after step t (after any reset) */
     float *min_gap;          /* [n] or NULL: smallest |logit1-logit0| seen */
+    uint32_t max_steps;      /* episode step limit (CartPole-v1 uses 500); 0 = none */
+    const uint32_t *action_bits_in; /* [T][ceil(n/32)] supplied actions (bit i%32 of word i/32) or NULL */
     int64_t lo, hi;          /* env sub-range handled by this worker */
     uint64_t tot_ret, tot_cnt;
 } co_rollout_job;
@@ -332,10 +334,19 @@ static void co_rollout_range(co_rollout_job *J)
         for (int64_t k = 0; k < T; ++k) {
             uint32_t t = J->t0 + (uint32_t)k;
             float gap;
-            int a = co_policy_action(J->kind, J->w, ka0, ka1, t, z, &gap);
+            int a;
+            if (J->action_bits_in) {
+                a = (int)((J->action_bits_in[k * words + i / 32] >> (i % 32)) & 1u);
+                gap = INFINITY;
+            } else {
+                a = co_policy_action(J->kind, J->w, ka0, ka1, t, z, &gap);
+            }
             if (gap < min_gap) min_gap = gap;
             int d = co_dynamics_f32(z, a, zn);
             ep_len += 1u; /* reward 1 per step, terminating step included */
+            /* an episode that has lasted max_steps steps is cut off: it counts as finished
+             * (done = 1, its return is its length) and the env restarts like after a fall */
+            if (J->max_steps && ep_len >= J->max_steps) d = 1;
             if (d) {
                 ret_sum += ep_len;
                 ep_cnt += 1u;
@@ -373,11 +384,11 @@ static void *co_rollout_thread(void *arg)
 /* totals[0] += sum over envs of ep_return_sum (as integer), totals[1] +=
  * sum of ep_count. nthreads > 1 splits the env range statically; worker
  * ranges are multiples of 32 envs so bit-stream words are never shared. */
-void co_rollout(uint32_t env_offset, int64_t n, int64_t T, uint32_t seed, uint32_t t0, int kind,
-                const float *weights, const float *init_state, uint32_t *ep_len_io,
-                float *ep_return_sum, uint32_t *ep_count, uint64_t *totals, float *reward_stream,
-                uint32_t *done_bits, uint32_t *action_bits, float *final_state, float *trajectory,
-                float *min_gap, int nthreads)
+void co_rollout_ex(uint32_t env_offset, int64_t n, int64_t T, uint32_t seed, uint32_t t0, int kind,
+                   const float *weights, const float *init_state, uint32_t *ep_len_io,
+                   float *ep_return_sum, uint32_t *ep_count, uint64_t *totals, float *reward_stream,
+                   uint32_t *done_bits, uint32_t *action_bits, float *final_state, float *trajectory,
+                   float *min_gap, int nthreads, uint32_t max_steps, const uint32_t *action_bits_in)
 {
     if (nthreads < 1) nthreads = 1;
     if (nthreads > 256) nthreads = 256;
@@ -392,7 +403,7 @@ void co_rollout(uint32_t env_offset, int64_t n, int64_t T, uint32_t seed, uint32
         if (hi > n) hi = n;
         co_rollout_job J = {env_offset, n, T, seed, t0, kind, weights, init_state, ep_len_io,
                             ep_return_sum, ep_count, reward_stream, done_bits, action_bits,
-                            final_state, trajectory, min_gap, lo, hi, 0, 0};
+                            final_state, trajectory, min_gap, max_steps, action_bits_in, lo, hi, 0, 0};
         jobs[used++] = J;
     }
     if (used == 1) {
@@ -408,4 +419,43 @@ void co_rollout(uint32_t env_offset, int64_t n, int64_t T, uint32_t seed, uint32
             totals[0] += jobs[w].tot_ret;
             totals[1] += jobs[w].tot_cnt;
         }
+}
+
+/* The basic contract: no episode step limit, actions from the policy. */
+void co_rollout(uint32_t env_offset, int64_t n, int64_t T, uint32_t seed, uint32_t t0, int kind,
+                const float *weights, const float *init_state, uint32_t *ep_len_io,
+                float *ep_return_sum, uint32_t *ep_count, uint64_t *totals, float *reward_stream,
+                uint32_t *done_bits, uint32_t *action_bits, float *final_state, float *trajectory,
+                float *min_gap, int nthreads)
+{
+    co_rollout_ex(env_offset, n, T, seed, t0, kind, weights, init_state, ep_len_io, ep_return_sum, ep_count,
+                  totals, reward_stream, done_bits, action_bits, final_state, trajectory, min_gap, nthreads,
+                  0u, NULL);
+}
+
+/* co_step with an episode step limit: ep_len [n] holds the steps already taken in each
+ * running episode, in and out (0 after a restart). max_steps = 0 means no limit. */
+void co_step_limited(uint32_t env_offset, int64_t n, int64_t stride_in, int64_t stride_out, uint32_t seed,
+                     uint32_t t, const float *planes_in, const uint8_t *action, float *planes_out,
+                     float *reward, uint8_t *done, uint32_t *ep_len, uint32_t max_steps)
+{
+    for (int64_t i = 0; i < n; ++i) {
+        uint32_t env = env_offset + (uint32_t)i;
+        float z[4], zn[4];
+        for (int p = 0; p < 4; ++p)
+            z[p] = planes_in[p * stride_in + i];
+        int a = action ? (action[i] != 0) : (int)co_action(seed, env, t);
+        int d = co_dynamics_f32(z, a, zn);
+        uint32_t len = ep_len[i] + 1u;
+        if (max_steps && len >= max_steps) d = 1;
+        if (d) {
+            co_reset_state(seed, env, t + 1u, zn);
+            len = 0u;
+        }
+        ep_len[i] = len;
+        for (int p = 0; p < 4; ++p)
+            planes_out[p * stride_out + i] = zn[p];
+        if (reward) reward[i] = 1.0f;
+        if (done) done[i] = (uint8_t)d;
+    }
 }

@@ -67,6 +67,10 @@ def lib() -> C.CDLL:
         L.co_step.argtypes = [u32, i64, i64, i64, u32, u32, p, p, p, p, p, p, p]
         L.co_rollout.restype = None
         L.co_rollout.argtypes = [u32, i64, i64, u32, u32, i32, p, p, p, p, p, p, p, p, p, p, p, p, i32]
+        L.co_rollout_ex.restype = None
+        L.co_rollout_ex.argtypes = [u32, i64, i64, u32, u32, i32, p, p, p, p, p, p, p, p, p, p, p, p, i32, u32, p]
+        L.co_step_limited.restype = None
+        L.co_step_limited.argtypes = [u32, i64, i64, i64, u32, u32, p, p, p, p, p, p, u32]
         _lib = L
     return _lib
 
@@ -183,8 +187,12 @@ def rollout(n: int, T: int, seed: int, policy_kind: int = POLICY_RANDOM, weights
             ep_len: np.ndarray | None = None, per_env: bool = True,
             reward_stream: bool = False, done_bits: bool = False,
             action_bits: bool = False, final_state: bool = False, trajectory: bool = False,
-            min_gap: bool = False, nthreads: int = 1) -> dict:
-    """Rollout of n envs for T steps. Returns a dict of the requested outputs."""
+            min_gap: bool = False, nthreads: int = 1, max_episode_steps: int = 0,
+            action_bits_in: np.ndarray | None = None) -> dict:
+    """Rollout of n envs for T steps. Returns a dict of the requested outputs.
+
+    max_episode_steps > 0 cuts episodes off at that length; action_bits_in ([T, ceil(n/32)]
+    uint32, bit i%32 of word i//32) supplies the actions instead of the policy."""
     w = None
     if policy_kind != POLICY_RANDOM:
         w = np.ascontiguousarray(weights, np.float32).ravel()
@@ -208,9 +216,28 @@ def rollout(n: int, T: int, seed: int, policy_kind: int = POLICY_RANDOM, weights
         ep_len = np.ascontiguousarray(ep_len, np.uint32).copy()
         assert ep_len.size == n
         res["ep_len"] = ep_len
-    lib().co_rollout(env_offset, n, T, seed, t0, policy_kind, _ptr(w), _ptr(init_state), _ptr(ep_len),
-                     _ptr(res["ep_return_sum"]), _ptr(res["ep_count"]), _ptr(res["totals"]),
-                     _ptr(res["reward_stream"]), _ptr(res["done_bits"]), _ptr(res["action_bits"]),
-                     _ptr(res["final_state"]), _ptr(res["trajectory"]), _ptr(res["min_gap"]),
-                     int(nthreads))
+    if action_bits_in is not None:
+        action_bits_in = np.ascontiguousarray(action_bits_in).view(np.uint32)
+        assert action_bits_in.shape == (T, words)
+    lib().co_rollout_ex(env_offset, n, T, seed, t0, policy_kind, _ptr(w), _ptr(init_state), _ptr(ep_len),
+                        _ptr(res["ep_return_sum"]), _ptr(res["ep_count"]), _ptr(res["totals"]),
+                        _ptr(res["reward_stream"]), _ptr(res["done_bits"]), _ptr(res["action_bits"]),
+                        _ptr(res["final_state"]), _ptr(res["trajectory"]), _ptr(res["min_gap"]),
+                        int(nthreads), int(max_episode_steps), _ptr(action_bits_in))
     return res
+
+
+def step_limited(planes: np.ndarray, seed: int, t: int, ep_len: np.ndarray, max_episode_steps: int,
+                 action_u8: np.ndarray | None = None, env_offset: int = 0) -> dict:
+    """One batched step with an episode step limit; ep_len (uint32 [n]) is carried in and out."""
+    planes = np.ascontiguousarray(planes, np.float32)
+    n = planes.shape[1]
+    out = np.empty((4, n), np.float32)
+    reward = np.empty(n, np.float32)
+    done = np.empty(n, np.uint8)
+    ep_len = np.ascontiguousarray(ep_len, np.uint32).copy()
+    if action_u8 is not None:
+        action_u8 = np.ascontiguousarray(action_u8, np.uint8)
+    lib().co_step_limited(env_offset, n, n, n, seed, t, _ptr(planes), _ptr(action_u8), _ptr(out), _ptr(reward),
+                          _ptr(done), _ptr(ep_len), int(max_episode_steps))
+    return {"state": out, "reward": reward, "done": done, "ep_len": ep_len}

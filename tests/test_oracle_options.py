@@ -1,0 +1,150 @@
+"""Pins for the oracle's optional behaviours (CPU only): the episode step limit of
+CartPole-v1 (an episode is cut off after a fixed number of steps and the environment restarts
+as after a fall) and actions supplied as a packed bit stream instead of drawn by the policy.
+Both are checked by brute force against per-environment scalar calls composed in Python and
+by the invariants the definitions imply."""
+import numpy as np
+import pytest
+
+from paper_2301_13062_b200 import inputs
+
+
+def pack_bits(bits: np.ndarray) -> np.ndarray:
+    """[T, n] 0/1 -> [T, ceil(n/32)] uint32, bit i%32 of word i//32."""
+    T, n = bits.shape
+    words = (n + 31) // 32
+    padded = np.zeros((T, words * 32), np.uint8)
+    padded[:, :n] = bits
+    return np.packbits(padded, axis=1, bitorder="little").view(np.uint32).reshape(T, words)
+
+
+def unpack_bits(words: np.ndarray, n: int) -> np.ndarray:
+    return np.unpackbits(np.ascontiguousarray(words).view(np.uint8), axis=-1, bitorder="little")[..., :n]
+
+
+def brute_rollout(oracle, n, T, seed, limit=0, actions=None, env_offset=0):
+    """Scalar composition: dynamics_f32 / action / reset_state per env and step."""
+    ret = np.zeros(n, np.int64)
+    cnt = np.zeros(n, np.int64)
+    done = np.zeros((T, n), np.uint8)
+    final = np.zeros((4, n), np.float32)
+    for i in range(n):
+        e = env_offset + i
+        z = oracle.reset_state(seed, e, 0)
+        ep_len = 0
+        for t in range(T):
+            a = int(actions[t, i]) if actions is not None else oracle.action(seed, e, t)
+            z, d = oracle.dynamics_f32(z, a)
+            ep_len += 1
+            if limit and ep_len >= limit:
+                d = True
+            if d:
+                ret[i] += ep_len
+                cnt[i] += 1
+                ep_len = 0
+                z = oracle.reset_state(seed, e, t + 1)
+            done[t, i] = d
+        final[:, i] = z
+    return ret, cnt, done, final
+
+
+@pytest.mark.parametrize("limit", [1, 3, 7, 25])
+def test_step_limit_matches_brute_force(oracle, limit):
+    n, T, seed = 37, 60, 4
+    r = oracle.rollout(n, T, seed, max_episode_steps=limit, done_bits=True, final_state=True, env_offset=5)
+    ret, cnt, done, final = brute_rollout(oracle, n, T, seed, limit, env_offset=5)
+    assert np.array_equal(r["ep_return_sum"], ret.astype(np.float32))
+    assert np.array_equal(r["ep_count"], cnt.astype(np.uint32))
+    assert np.array_equal(unpack_bits(r["done_bits"], n), done)
+    assert np.array_equal(r["final_state"], final)
+
+
+def test_step_limit_invariants(oracle):
+    n, T, seed = 300, 200, 1
+    free = oracle.rollout(n, T, seed, done_bits=True)
+    # a limit of 1 ends an episode at every step
+    one = oracle.rollout(n, T, seed, max_episode_steps=1)
+    assert np.all(one["ep_count"] == T) and np.all(one["ep_return_sum"] == T)
+    # a limit nothing reaches changes nothing
+    big = oracle.rollout(n, T, seed, max_episode_steps=T + 1, done_bits=True)
+    assert np.array_equal(big["done_bits"], free["done_bits"])
+    # with a limit, no gap between consecutive done flags exceeds it, and every cut-off shows up
+    lim = 12
+    r = oracle.rollout(n, T, seed, max_episode_steps=lim, done_bits=True)
+    d = unpack_bits(r["done_bits"], n)
+    for i in range(n):
+        times = np.concatenate(([-1], np.nonzero(d[:, i])[0]))
+        gaps = np.diff(times)
+        assert gaps.size == 0 or gaps.max() <= lim
+        assert T - 1 - times[-1] < lim  # the running episode is shorter than the limit
+        assert r["ep_return_sum"][i] == times[-1] + 1
+    assert r["totals"][1] > free["totals"][1]
+    # until an env's first cut-off its done stream equals the unlimited one
+    df = unpack_bits(free["done_bits"], n)
+    for i in range(0, n, 7):
+        gaps = np.diff(np.concatenate(([-1], np.nonzero(df[:, i])[0])))
+        first_long = np.nonzero(gaps > lim)[0]
+        upto = T if first_long.size == 0 else (np.concatenate(([-1], np.nonzero(df[:, i])[0]))[first_long[0]] + lim)
+        assert np.array_equal(d[:upto, i], df[:upto, i])
+
+
+def test_step_limited_equals_limited_rollout(oracle):
+    n, T, seed, lim = 50, 40, 2, 9
+    r = oracle.rollout(n, T, seed, max_episode_steps=lim, trajectory=True, done_bits=True)
+    z = oracle.initial_state(n, seed)
+    ep_len = np.zeros(n, np.uint32)
+    d = unpack_bits(r["done_bits"], n)
+    for t in range(T):
+        s = oracle.step_limited(z, seed, t, ep_len, lim)
+        z, ep_len = s["state"], s["ep_len"]
+        assert np.array_equal(z, r["trajectory"][t]) and np.array_equal(s["done"], d[t])
+        assert np.all(s["reward"] == 1.0) and ep_len.max() < lim
+    # no limit: step_limited is the plain step plus a length counter
+    z0 = inputs.random_states(200, seed=3, spread="edge")
+    a = oracle.step(z0, seed, 5)
+    b = oracle.step_limited(z0, seed, 5, np.full(200, 7, np.uint32), 0)
+    assert np.array_equal(a["state"], b["state"]) and np.array_equal(a["done"], b["done"])
+    assert np.array_equal(b["ep_len"], np.where(a["done"] == 1, 0, 8))
+
+
+def test_chunked_limited_rollout_resumes_exactly(oracle):
+    n, seed, lim = 100, 3, 15
+    whole = oracle.rollout(n, 70, seed, max_episode_steps=lim, final_state=True)
+    a = oracle.rollout(n, 33, seed, max_episode_steps=lim, final_state=True, ep_len=np.zeros(n, np.uint32))
+    b = oracle.rollout(n, 37, seed, t0=33, init_state=a["final_state"], ep_len=a["ep_len"], max_episode_steps=lim,
+                       final_state=True)
+    assert np.array_equal(whole["final_state"], b["final_state"])
+    assert np.array_equal(whole["ep_return_sum"], a["ep_return_sum"] + b["ep_return_sum"])
+    assert np.array_equal(whole["ep_count"], a["ep_count"] + b["ep_count"])
+
+
+def test_supplied_action_stream(oracle):
+    n, T, seed = 45, 50, 6
+    rng = np.random.default_rng(0)
+    acts = rng.integers(0, 2, (T, n)).astype(np.uint8)
+    r = oracle.rollout(n, T, seed, action_bits_in=pack_bits(acts), done_bits=True, action_bits=True,
+                       final_state=True, min_gap=True)
+    ret, cnt, done, final = brute_rollout(oracle, n, T, seed, actions=acts)
+    assert np.array_equal(r["ep_return_sum"], ret.astype(np.float32))
+    assert np.array_equal(r["ep_count"], cnt.astype(np.uint32))
+    assert np.array_equal(unpack_bits(r["done_bits"], n), done)
+    assert np.array_equal(unpack_bits(r["action_bits"], n), acts)  # echoed back unchanged
+    assert np.array_equal(r["final_state"], final) and np.all(np.isinf(r["min_gap"]))
+    # feeding the hashed actions back in reproduces the random-policy rollout
+    h = oracle.rollout(n, T, seed, action_bits=True, final_state=True)
+    g = oracle.rollout(n, T, seed, action_bits_in=h["action_bits"], final_state=True)
+    for k in ("ep_return_sum", "ep_count", "final_state", "totals"):
+        assert np.array_equal(h[k], g[k])
+    # a supplied stream overrides a policy; padding bits beyond n are ignored
+    w = inputs.policy_weights(inputs.POLICY_LINEAR, 1)
+    p = oracle.rollout(n, T, seed, inputs.POLICY_LINEAR, w, action_bits_in=pack_bits(acts))
+    assert np.array_equal(p["ep_return_sum"], r["ep_return_sum"])
+    full = pack_bits(acts).copy()
+    full[:, -1] |= np.uint32((0xFFFFFFFF << (n % 32)) & 0xFFFFFFFF)
+    q = oracle.rollout(n, T, seed, action_bits_in=full)
+    assert np.array_equal(q["ep_return_sum"], r["ep_return_sum"])
+    # constant push right from the start states: the pole falls to the negative side quickly
+    ones = np.ones((20, 8), np.uint8)
+    c = oracle.rollout(8, 20, seed, action_bits_in=pack_bits(ones), done_bits=True)
+    first = np.argmax(unpack_bits(c["done_bits"], 8), axis=0)
+    assert np.all((first >= 6) & (first <= 12))
