@@ -203,6 +203,40 @@ int cp_rollout_shard(uint32_t env_offset, int64_t n_envs, int64_t T, uint32_t se
 int cp_rollout_from(cp_state *state, int64_t T, uint32_t *ep_len, const cp_policy *policy,
                     const cp_returns *returns);
 
+/* The general rollout call: everything cp_rollout / cp_rollout_shard / cp_rollout_from do, plus
+ *   - an episode step limit (CartPole-v1 cuts an episode off after 500 steps): an episode that has
+ *     lasted max_episode_steps steps ends on that step exactly like a fall — done = 1, reward 1, its
+ *     length added to ep_return_sum, counted in ep_count — and the environment restarts;
+ *   - actions given as data instead of drawn by a policy (the paper's baseline, Sec. V-A, feeds
+ *     precomputed random values): action_bits_in DEVICE [T][ceil(n_envs/32)], bit (i%32) of word
+ *     (i/32) of row k = action of env i at the k-th step of this call; overrides `policy`.
+ * struct_size must be sizeof(cp_rollout_args) (guards against a caller built for another layout).
+ * state == NULL: start states of global time t0, env range [env_offset, env_offset + n_envs);
+ * state != NULL: that batch is advanced in place from its own time (n_envs, seed, env_offset, t0 of
+ * the struct are ignored, returns->final_state too) and state->t grows by T.
+ * ep_len: DEVICE [n_envs] steps already taken in each running episode, read and rewritten, or NULL
+ * (all episodes start at this call; nothing written). t0 + T <= CP_MAX_T. */
+typedef struct cp_rollout_args {
+    uint32_t struct_size;
+    uint32_t env_offset;
+    int64_t n_envs, T;
+    uint32_t seed, t0;
+    const cp_policy *policy;       /* HOST, or NULL = hashed random actions */
+    const cp_returns *returns;     /* HOST struct of DEVICE pointers, not NULL */
+    cp_state *state;               /* or NULL */
+    uint32_t *ep_len;              /* DEVICE or NULL */
+    uint32_t max_episode_steps;    /* 0 = no limit */
+    const uint32_t *action_bits_in; /* DEVICE or NULL */
+} cp_rollout_args;
+int cp_rollout_ex(const cp_rollout_args *args);
+
+/* cp_step with per-environment episode-length counters and the same optional step limit:
+ * ep_len DEVICE [n_envs] (16-byte aligned for the vector kernel) is incremented, compared with
+ * max_episode_steps (0 = no limit; an env reaching it reports done = 1 and restarts) and reset to
+ * 0 for finished environments. ep_len == NULL makes this cp_step (and then the limit must be 0). */
+int cp_step_ex(cp_state *state, const uint8_t *action, cp_state *out_state, float *reward, uint8_t *done,
+               uint32_t *ep_len, uint32_t max_episode_steps);
+
 /* End-to-end forms with HOST buffers (pinned memory recommended): device staging buffers
  * are owned by the library (grown on demand, released by cp_shutdown); the calls copy in,
  * launch, copy out and SYNCHRONISE the stream before returning.
@@ -223,7 +257,7 @@ void cp_shutdown(void);
 void cp_set_stream(void *cuda_stream);
 
 /* Launch tuning, process-wide. key: "rollout_block" (threads per CTA, 32..256, multiple of 32;
- * default 256), "rollout_ept" (environments per thread: 1, 2 or 4; 0 = default, 2 for large
+ * default 256), "rollout_ept" (environments per thread: 1 or 2; 0 = default, 2 for large
  * batches), "rollout_ctas_per_sm" (0 = default: one 32*ept-environment task per warp and as many
  * CTAs as that takes; k > 0 = persistent grid of k CTAs per SM looping over tasks), "step_block"
  * (32..256, default 64), "step_vec_min_envs" (batches smaller than this use the one-env-per-thread

@@ -27,6 +27,7 @@ EXPORTS = [
     "cp_rollout_from", "cp_rollout_host", "cp_step_host", "cp_shutdown", "cp_set_stream", "cp_tune",
     "cp_launch_count", "cp_selftest_sincos", "cp_last_error", "cp_version", "cp_step_unfused_noalloc",
     "cp_selftest_sincos_accuracy", "cp_selftest_arith", "cp_step_repeat", "cp_selftest_tame_div",
+    "cp_rollout_ex", "cp_step_ex",
 ]
 CP_NOALLOC_MAX_ENVS = 65536
 
@@ -38,6 +39,13 @@ class cp_policy(C.Structure):
 class cp_returns(C.Structure):
     _fields_ = [(k, C.c_void_p) for k in ("ep_return_sum", "ep_count", "totals", "reward_stream", "done_bits",
                                           "action_bits", "final_state", "trajectory")]
+
+
+class cp_rollout_args(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("env_offset", C.c_uint32), ("n_envs", C.c_int64), ("T", C.c_int64),
+                ("seed", C.c_uint32), ("t0", C.c_uint32), ("policy", C.POINTER(cp_policy)),
+                ("returns", C.POINTER(cp_returns)), ("state", C.c_void_p), ("ep_len", C.c_void_p),
+                ("max_episode_steps", C.c_uint32), ("action_bits_in", C.c_void_p)]
 
 
 class CartpoleError(RuntimeError):
@@ -63,6 +71,8 @@ def lib() -> C.CDLL:
             "cp_step": (i32, [p, p, p, p, p]),
             "cp_rollout": (i32, [i64, i64, u32, C.POINTER(cp_policy), C.POINTER(cp_returns)]),
             "cp_step_repeat": (i32, [p, i64, p, p]),
+            "cp_rollout_ex": (i32, [C.POINTER(cp_rollout_args)]),
+            "cp_step_ex": (i32, [p, p, p, p, p, p, u32]),
             "cp_step_unfused": (i32, [p, p, p, p, p, p, sz]),
             "cp_unfused_workspace_bytes": (sz, [i64]),
             "cp_step_unfused_noalloc": (i32, [p, p, p, p, p]),
@@ -276,6 +286,33 @@ def cp_rollout_from(state: State, T: int, ep_len=None, policy: _Policy | None = 
     r = _returns_struct(**returns)
     _check(lib().cp_rollout_from(state.handle, T, _dptr(ep_len, torch.int32), policy.ref() if policy else None,
                                  C.byref(r)))
+
+
+def cp_rollout_ex(*, n_envs: int = 0, T: int, seed: int = 0, t0: int = 0, env_offset: int = 0,
+                  policy: _Policy | None = None, state: State | None = None, ep_len=None,
+                  max_episode_steps: int = 0, action_bits_in=None, **returns) -> None:
+    """General rollout: optional episode step limit, optional supplied action bit stream, either
+    from start states (n_envs, seed, t0, env_offset) or advancing `state` in place."""
+    import torch
+    _use_current_stream()
+    r = _returns_struct(**returns)
+    a = cp_rollout_args()
+    a.struct_size = C.sizeof(cp_rollout_args)
+    a.env_offset, a.n_envs, a.T, a.seed, a.t0 = env_offset, n_envs, T, seed, t0
+    a.policy = C.pointer(policy.struct) if policy else None
+    a.returns = C.pointer(r)
+    a.state = state.handle if state is not None else None
+    a.ep_len = _dptr(ep_len, torch.int32)
+    a.max_episode_steps = max_episode_steps
+    a.action_bits_in = _dptr(action_bits_in, torch.int32)
+    _check(lib().cp_rollout_ex(C.byref(a)))
+
+
+def cp_step_ex(state: State, action, out_state: State, reward, done, ep_len, max_episode_steps: int = 0) -> None:
+    import torch
+    _use_current_stream()
+    _check(lib().cp_step_ex(state.handle, _dptr(action, torch.uint8), out_state.handle, _dptr(reward, torch.float32),
+                            _dptr(done, torch.uint8), _dptr(ep_len, torch.int32), max_episode_steps))
 
 
 def cp_rollout_host(n_envs: int, T: int, seed: int, policy: _Policy | None, h_ep_return_sum, h_ep_count, h_totals) -> None:

@@ -96,6 +96,8 @@ void fill_step_params(cp::StepParams &p, const cp_state *in, cp_state *out, cons
     p.action = action;
     p.reward = reward;
     p.done = done;
+    p.ep_len = nullptr;
+    p.max_steps = 0;
 }
 
 int check_step_args(cp_state *state, cp_state *out_state) {
@@ -117,7 +119,8 @@ void advance(cp_state *state, cp_state *out_state, uint32_t steps) {
 // Rollout shared by cp_rollout / cp_rollout_shard / cp_rollout_from / cp_rollout_host.
 int rollout_impl(uint32_t env_offset, int64_t n_envs, int64_t T, uint32_t seed, uint32_t t0, const cp_policy *policy,
                  const cp_returns *ret, const float *init_planes, int64_t init_stride, float *out_planes,
-                 int64_t out_stride, uint32_t *ep_len) {
+                 int64_t out_stride, uint32_t *ep_len, uint32_t max_steps = 0,
+                 const uint32_t *action_bits_in = nullptr) {
     int kind, rc;
     if ((rc = check_range(n_envs, env_offset)) != CP_OK) return rc;
     if (T <= 0 || T > CP_MAX_T || (int64_t)t0 + T > CP_MAX_T)
@@ -145,6 +148,8 @@ int rollout_impl(uint32_t env_offset, int64_t n_envs, int64_t T, uint32_t seed, 
     p.done_bits = ret->done_bits;
     p.action_bits = ret->action_bits;
     p.trajectory = ret->trajectory;
+    p.max_steps = max_steps;
+    p.action_bits_in = action_bits_in;
     if (kind == CP_POLICY_LINEAR) memcpy(p.w, policy->weights, 10 * sizeof(float));
     if (kind == CP_POLICY_MLP) memcpy(p.w, policy->weights, 114 * sizeof(float));
     const bool streams = p.reward_stream || p.done_bits || p.action_bits || p.trajectory;
@@ -299,19 +304,33 @@ int cp_state_info(const cp_state *state, int64_t *n_envs, int64_t *plane_stride,
     return CP_OK;
 }
 
-int cp_step(cp_state *state, const uint8_t *action, cp_state *out_state, float *reward, uint8_t *done) {
+static int step_impl(cp_state *state, const uint8_t *action, cp_state *out_state, float *reward, uint8_t *done,
+                     uint32_t *ep_len, uint32_t max_steps) {
     int rc = check_step_args(state, out_state);
     if (rc != CP_OK) return rc;
     if (reward && !is_aligned(reward, 4)) return fail(CP_EINVAL, "reward is not float-aligned");
+    if (ep_len && !is_aligned(ep_len, 4)) return fail(CP_EINVAL, "ep_len is not 4-byte aligned");
+    if (max_steps && !ep_len) return fail(CP_EINVAL, "an episode step limit needs the ep_len counters");
     cp::StepParams p;
     fill_step_params(p, state, out_state, action, reward, done);
+    p.ep_len = ep_len;
+    p.max_steps = max_steps;
     const bool vec = state->n >= cp::g_tuning.step_vec_min_envs && state_vec_ok(state) && state_vec_ok(out_state) &&
                      (!reward || is_aligned(reward, 16)) && (!done || is_aligned(done, 4)) &&
-                     (!action || is_aligned(action, 4));
+                     (!action || is_aligned(action, 4)) && (!ep_len || is_aligned(ep_len, 16));
     cudaError_t e = cp::launch_step(p, vec, tl_stream);
     if (e != cudaSuccess) return cuda_fail(e, "step launch");
     advance(state, out_state, 1);
     return CP_OK;
+}
+
+int cp_step(cp_state *state, const uint8_t *action, cp_state *out_state, float *reward, uint8_t *done) {
+    return step_impl(state, action, out_state, reward, done, nullptr, 0);
+}
+
+int cp_step_ex(cp_state *state, const uint8_t *action, cp_state *out_state, float *reward, uint8_t *done,
+               uint32_t *ep_len, uint32_t max_episode_steps) {
+    return step_impl(state, action, out_state, reward, done, ep_len, max_episode_steps);
 }
 
 int cp_step_repeat(cp_state *state, int64_t k, float *reward, uint8_t *done) {
@@ -376,6 +395,26 @@ int cp_rollout_from(cp_state *state, int64_t T, uint32_t *ep_len, const cp_polic
     if (rc != CP_OK) return rc;
     state->t += (uint32_t)T;
     return CP_OK;
+}
+
+int cp_rollout_ex(const cp_rollout_args *a) {
+    if (!a) return fail(CP_EINVAL, "args is NULL");
+    if (a->struct_size != sizeof(cp_rollout_args))
+        return fail(CP_EINVAL, "struct_size is %u, this library expects %zu", a->struct_size, sizeof(cp_rollout_args));
+    if (!a->returns) return fail(CP_EINVAL, "returns is NULL");
+    if (a->action_bits_in && !is_aligned(a->action_bits_in, 4)) return fail(CP_EINVAL, "action_bits_in is misaligned");
+    if (a->state) {
+        int rc = check_state(a->state, "state");
+        if (rc != CP_OK) return rc;
+        cp_state *st = a->state;
+        rc = rollout_impl(st->env_offset, st->n, a->T, st->seed, st->t, a->policy, a->returns, st->planes, st->stride,
+                          st->planes, st->stride, a->ep_len, a->max_episode_steps, a->action_bits_in);
+        if (rc != CP_OK) return rc;
+        st->t += (uint32_t)a->T;
+        return CP_OK;
+    }
+    return rollout_impl(a->env_offset, a->n_envs, a->T, a->seed, a->t0, a->policy, a->returns, nullptr, 0,
+                        a->returns->final_state, a->n_envs, a->ep_len, a->max_episode_steps, a->action_bits_in);
 }
 
 int cp_rollout_host(int64_t n_envs, int64_t T, uint32_t seed, const cp_policy *policy, float *h_ep_return_sum,
@@ -463,7 +502,7 @@ int cp_tune(const char *key, int value) {
         if (value < 32 || value > 256 || value % 32) return fail(CP_EINVAL, "rollout_block must be 32..256, multiple of 32");
         cp::g_tuning.rollout_block = value;
     } else if (!strcmp(key, "rollout_ept")) {
-        if (value != 0 && value != 1 && value != 2 && value != 4) return fail(CP_EINVAL, "rollout_ept must be 0, 1, 2 or 4");
+        if (value != 0 && value != 1 && value != 2) return fail(CP_EINVAL, "rollout_ept must be 0, 1 or 2");
         cp::g_tuning.rollout_ept = value;
     } else if (!strcmp(key, "rollout_ctas_per_sm")) {
         if (value < 0 || value > 1024) return fail(CP_EINVAL, "rollout_ctas_per_sm must be 0..1024");

@@ -19,6 +19,8 @@ struct StepParams {
     const uint8_t *action;  // or nullptr: hashed
     float *reward;          // or nullptr
     uint8_t *done;          // or nullptr
+    uint32_t *ep_len;       // or nullptr: steps taken in each running episode, in/out
+    uint32_t max_steps;     // episode step limit (needs ep_len), 0 = none
 };
 
 // Parameters of one rollout launch. Weights travel in the launch parameters
@@ -39,6 +41,8 @@ struct RolloutParams {
     uint32_t *done_bits;
     uint32_t *action_bits;
     float *trajectory;
+    uint32_t max_steps;              // episode step limit, 0 = none
+    const uint32_t *action_bits_in;  // [T][words] supplied actions or nullptr
     float w[114];
 };
 

@@ -95,6 +95,8 @@ extern "C" int cp_step_unfused_noalloc(cp_state *state, const uint8_t *action, c
     p.action = action;
     p.reward = reward;
     p.done = done;
+    p.ep_len = nullptr;
+    p.max_steps = 0;
     // Every intermediate plane is fully written by the kernel that produces it before any
     // kernel reads it, so nothing in the scratch needs clearing between calls.
     cudaError_t e = cp::launch_ladder(p, scratch, cp::thread_stream());

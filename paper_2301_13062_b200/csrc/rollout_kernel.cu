@@ -7,8 +7,9 @@
 // Work decomposition: a "warp task" is 32*EPT consecutive environments; lane l
 // owns environments base + j*32 + l (j < EPT), so that per-step stream stores
 // are one contiguous 128-byte line per j and a done/action bitmask word is one
-// warp ballot. Tasks are dealt round-robin to the resident warps (persistent
-// grid, sized from the occupancy calculator times the SM count).
+// warp ballot. By default every warp gets exactly one task and the hardware
+// hands out CTAs as others retire; a persistent grid looping over tasks is
+// available for tuning.
 //
 // The kernel has no shared memory, no inter-warp synchronisation and no waits.
 #include "cartpole_device.cuh"
@@ -16,6 +17,7 @@
 
 namespace cp {
 
+// POLICY: 0 hashed random action, 1 linear, 2 MLP, 3 action bits supplied by the caller.
 template <int POLICY>
 __device__ __forceinline__ uint32_t policy_signbit(const RolloutParams &p, const Keys &ka, uint32_t t,
                                                    const State &z) {
@@ -32,7 +34,10 @@ __device__ __forceinline__ uint32_t policy_signbit(const RolloutParams &p, const
 #define CP_ROLLOUT_MIN_CTAS 1
 #endif
 
-template <int POLICY, int EPT, int STREAMS>
+// STREAMS: 0 no per-step output; 1 exactly the reward plane and the done bitmask (no run-time
+// tests in the loop); 2 any combination, tested per step.
+// LIMIT: episodes are cut off after p.max_steps steps.
+template <int POLICY, int EPT, int STREAMS, bool LIMIT>
 __global__ void __launch_bounds__(256, CP_ROLLOUT_MIN_CTAS) rollout_kernel(const __grid_constant__ RolloutParams p) {
     const uint32_t lane = threadIdx.x & 31u;
     const int64_t warps_total = (int64_t)gridDim.x * (blockDim.x >> 5);
@@ -45,9 +50,11 @@ __global__ void __launch_bounds__(256, CP_ROLLOUT_MIN_CTAS) rollout_kernel(const
         State z[EPT];
         Keys ka[EPT], kr[EPT];
         // Episode bookkeeping: every step earns reward 1, so the returns of the episodes completed
-        // in this launch add up to (steps carried in) + (time of the last termination), and only
-        // the count and the time of the last termination need to live in the loop.
-        uint32_t cnt[EPT], last[EPT];  // last: global time just after the last done (t0 = none yet)
+        // in this launch add up to (time of the last termination) - (time the first of them began),
+        // and only the count and the start time of the running episode need to live in the loop.
+        // begin[j]: global time at which env j's running episode began (before t0 if steps were
+        // carried in; unsigned wrap-around is harmless, only differences are used).
+        uint32_t cnt[EPT], begin[EPT];
         int64_t idx[EPT];
         bool valid[EPT];
 #pragma unroll
@@ -67,24 +74,25 @@ __global__ void __launch_bounds__(256, CP_ROLLOUT_MIN_CTAS) rollout_kernel(const
                 z[j] = start_state(kr[j], p.t0);
             }
             cnt[j] = 0u;
-            last[j] = p.t0;
+            begin[j] = p.t0 - (p.ep_len_io ? p.ep_len_io[idx[j]] : 0u);
         }
 
         // Per-step stream outputs advance by one row per step: keep running pointers / offsets
         // instead of recomputing row * width + column with 64-bit multiplies every step.
-        // STREAMS == 1: exactly the reward plane and the done bitmask are written (no run-time
-        // tests in the loop); STREAMS == 2: any combination, tested per step.
         float *rew_ptr[EPT];
         uint32_t *done_ptr[EPT];
+        const uint32_t *act_ptr[EPT];
         int64_t env_off[EPT], word_off[EPT];  // into [T][n] planes and [T][words] bit planes
         bool word_ok[EPT];
 #pragma unroll
         for (int j = 0; j < EPT; ++j) {
             env_off[j] = idx[j];
             word_off[j] = task * EPT + j;
-            word_ok[j] = lane == 0 && word_off[j] < words;
+            const bool in_range = word_off[j] < words;
+            word_ok[j] = lane == 0 && in_range;
             rew_ptr[j] = STREAMS == 1 ? p.reward_stream + idx[j] : nullptr;
             done_ptr[j] = STREAMS == 1 ? p.done_bits + (word_ok[j] ? word_off[j] : 0) : nullptr;
+            act_ptr[j] = POLICY == 3 ? p.action_bits_in + (in_range ? word_off[j] : 0) : nullptr;
         }
         const bool want_done = STREAMS == 2 && p.done_bits, want_act = STREAMS == 2 && p.action_bits;
         const bool want_rew = STREAMS == 2 && p.reward_stream, want_traj = STREAMS == 2 && p.trajectory;
@@ -93,11 +101,18 @@ __global__ void __launch_bounds__(256, CP_ROLLOUT_MIN_CTAS) rollout_kernel(const
         for (uint32_t t = p.t0; t != t_end; ++t) {
 #pragma unroll
             for (int j = 0; j < EPT; ++j) {
-                const uint32_t sb = policy_signbit<POLICY>(p, ka[j], t, z[j]);
-                const bool done = euler_step(z[j], force_from_signbit(sb));
+                uint32_t sb;
+                if (POLICY == 3) {
+                    sb = (__ldg(act_ptr[j]) << (31u - lane)) & 0x80000000u;  // one word per warp, broadcast
+                    act_ptr[j] += words;
+                } else {
+                    sb = policy_signbit<POLICY>(p, ka[j], t, z[j]);
+                }
+                bool done = euler_step(z[j], force_from_signbit(sb));
+                if (LIMIT) done |= (t + 1u - begin[j]) >= p.max_steps;
                 if (done) {
                     cnt[j] += 1u;
-                    last[j] = t + 1u;
+                    begin[j] = t + 1u;
                     z[j] = start_state(kr[j], t + 1u);
                 }
                 if (STREAMS == 1) {
@@ -135,12 +150,12 @@ __global__ void __launch_bounds__(256, CP_ROLLOUT_MIN_CTAS) rollout_kernel(const
 #pragma unroll
         for (int j = 0; j < EPT; ++j) {
             if (!valid[j]) continue;
-            const uint32_t carried = p.ep_len_io ? p.ep_len_io[idx[j]] : 0u;
-            const bool any = last[j] != p.t0;
-            const uint32_t ret = any ? carried + (last[j] - p.t0) : 0u;
+            // sum of the returns of the completed episodes = last termination time - time the first began
+            const uint32_t first_begin = p.t0 - (p.ep_len_io ? p.ep_len_io[idx[j]] : 0u);
+            const uint32_t ret = cnt[j] ? begin[j] - first_begin : 0u;
             if (p.ep_return_sum) p.ep_return_sum[idx[j]] = (float)ret;
             if (p.ep_count) p.ep_count[idx[j]] = cnt[j];
-            if (p.ep_len_io) p.ep_len_io[idx[j]] = any ? t_end - last[j] : carried + p.T;
+            if (p.ep_len_io) p.ep_len_io[idx[j]] = t_end - begin[j];
             if (p.out_planes) {
                 p.out_planes[idx[j]] = z[j].x;
                 p.out_planes[p.out_stride + idx[j]] = z[j].xd;
@@ -166,7 +181,7 @@ __global__ void __launch_bounds__(256, CP_ROLLOUT_MIN_CTAS) rollout_kernel(const
 
 namespace {
 
-template <int POLICY, int EPT, int STREAMS>
+template <int POLICY, int EPT, int STREAMS, bool LIMIT>
 cudaError_t launch_one(RolloutParams &p, cudaStream_t s) {
     const int block = g_tuning.rollout_block;
     p.n_tasks = (p.n + 32 * EPT - 1) / (32 * EPT);
@@ -183,17 +198,27 @@ cudaError_t launch_one(RolloutParams &p, cudaStream_t s) {
         if (grid > resident) grid = resident;
     }
     if (grid > 0x7fffffffLL) grid = 0x7fffffffLL;
-    rollout_kernel<POLICY, EPT, STREAMS><<<(unsigned)grid, block, 0, s>>>(p);
+    rollout_kernel<POLICY, EPT, STREAMS, LIMIT><<<(unsigned)grid, block, 0, s>>>(p);
     count_launch();
     return cudaGetLastError();
 }
 
-template <int POLICY, int STREAMS>
+template <int POLICY, int STREAMS, bool LIMIT>
 cudaError_t launch_ept(RolloutParams &p, int ept, cudaStream_t s) {
-    switch (ept) {
-        case 1: return launch_one<POLICY, 1, STREAMS>(p, s);
-        case 2: return launch_one<POLICY, 2, STREAMS>(p, s);
-        default: return launch_one<POLICY, 4, STREAMS>(p, s);
+    return ept == 1 ? launch_one<POLICY, 1, STREAMS, LIMIT>(p, s) : launch_one<POLICY, 2, STREAMS, LIMIT>(p, s);
+}
+
+template <int POLICY, int STREAMS>
+cudaError_t launch_limit(RolloutParams &p, int ept, cudaStream_t s) {
+    return p.max_steps ? launch_ept<POLICY, STREAMS, true>(p, ept, s) : launch_ept<POLICY, STREAMS, false>(p, ept, s);
+}
+
+template <int POLICY>
+cudaError_t launch_mode(RolloutParams &p, int mode, int ept, cudaStream_t s) {
+    switch (mode) {
+        case 0: return launch_limit<POLICY, 0>(p, ept, s);
+        case 1: return launch_limit<POLICY, 1>(p, ept, s);
+        default: return launch_limit<POLICY, 2>(p, ept, s);
     }
 }
 
@@ -201,21 +226,19 @@ cudaError_t launch_ept(RolloutParams &p, int ept, cudaStream_t s) {
 
 cudaError_t launch_rollout(RolloutParams &p, int policy, bool streams, cudaStream_t s) {
     int ept = g_tuning.rollout_ept;
-    if (ept == 0) ept = 2;
-    // Small batches: spread environments over as many warps as possible.
-    while (ept > 1 && (p.n + 32 * ept - 1) / (32 * ept) < (int64_t)sm_count() * 16) ept >>= 1;
+    if (ept == 0) {
+        // Two envs per thread (two independent dependency chains) unless the batch is so small
+        // that spreading it over twice as many warps matters more.
+        ept = (p.n + 63) / 64 < (int64_t)sm_count() * 16 ? 1 : 2;
+    }
     // 0: no per-step output; 1: reward plane + done bitmask only; 2: any other combination
     const int mode = !streams ? 0 : (p.reward_stream && p.done_bits && !p.action_bits && !p.trajectory) ? 1 : 2;
-    switch (policy * 3 + mode) {
-        case 0: return launch_ept<0, 0>(p, ept, s);
-        case 1: return launch_ept<0, 1>(p, ept, s);
-        case 2: return launch_ept<0, 2>(p, ept, s);
-        case 3: return launch_ept<1, 0>(p, ept, s);
-        case 4: return launch_ept<1, 1>(p, ept, s);
-        case 5: return launch_ept<1, 2>(p, ept, s);
-        case 6: return launch_ept<2, 0>(p, ept, s);
-        case 7: return launch_ept<2, 1>(p, ept, s);
-        default: return launch_ept<2, 2>(p, ept, s);
+    if (p.action_bits_in) policy = 3;
+    switch (policy) {
+        case 0: return launch_mode<0>(p, mode, ept, s);
+        case 1: return launch_mode<1>(p, mode, ept, s);
+        case 2: return launch_mode<2>(p, mode, ept, s);
+        default: return launch_mode<3>(p, mode, ept, s);
     }
 }
 

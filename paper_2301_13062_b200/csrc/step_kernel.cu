@@ -67,6 +67,28 @@ __global__ void __launch_bounds__(256, CP_STEP_MIN_CTAS) step_kernel(const __gri
         uint32_t dmask = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) dmask |= (euler_step(z[j], force_from_signbit(sb[j])) ? 1u : 0u) << j;
+        if (p.ep_len) {  // optional episode-length counters and step limit
+            uint32_t len[4] = {0u, 0u, 0u, 0u};
+            if (full) {
+                const uint4 v = *reinterpret_cast<const uint4 *>(p.ep_len + i0);
+                len[0] = v.x; len[1] = v.y; len[2] = v.z; len[3] = v.w;
+            } else {
+                for (int j = 0; j < 4; ++j)
+                    if (i0 + j < p.n) len[j] = p.ep_len[i0 + j];
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                len[j] += 1u;
+                if (p.max_steps && len[j] >= p.max_steps) dmask |= 1u << j;
+                if ((dmask >> j) & 1u) len[j] = 0u;
+            }
+            if (full) {
+                *reinterpret_cast<uint4 *>(p.ep_len + i0) = make_uint4(len[0], len[1], len[2], len[3]);
+            } else {
+                for (int j = 0; j < 4; ++j)
+                    if (i0 + j < p.n) p.ep_len[i0 + j] = len[j];
+            }
+        }
         // Restart finished environments one per pass: almost always at most one of a
         // thread's four environments finishes in a step, so the start-state hashes are
         // issued once per warp instead of once per environment slot.
@@ -104,7 +126,12 @@ __global__ void __launch_bounds__(256, CP_STEP_MIN_CTAS) step_kernel(const __gri
         cudaTriggerProgrammaticLaunchCompletion();
         State z = {p.in[i], p.in[p.in_stride + i], p.in[2 * p.in_stride + i], p.in[3 * p.in_stride + i]};
         if (has_action) sb = p.action[i] ? 0x80000000u : 0u;
-        const bool d = euler_step(z, force_from_signbit(sb));
+        bool d = euler_step(z, force_from_signbit(sb));
+        if (p.ep_len) {
+            uint32_t len = p.ep_len[i] + 1u;
+            if (p.max_steps && len >= p.max_steps) d = true;
+            p.ep_len[i] = d ? 0u : len;
+        }
         if (d) z = start_state(make_keys(p.salt_r, env), p.t + 1u);
         p.out[i] = z.x;
         p.out[p.out_stride + i] = z.xd;

@@ -1,0 +1,206 @@
+"""GPU parity tests of the optional behaviours of the general rollout / step calls: the
+episode step limit and actions supplied as a packed bit stream, against the CPU oracle and
+against the library's own basic paths."""
+import ctypes as C
+
+import numpy as np
+import pytest
+
+from paper_2301_13062_b200 import inputs
+from tests import gpu_helpers as H
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def cp():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2301_13062_b200 import binding
+    binding.lib()
+    torch.cuda.set_device(0)
+    return binding
+
+
+def host(t):
+    return t.cpu().numpy()
+
+
+def outputs(n, T, streams=True, final=True):
+    words = (n + 31) // 32
+    out = {"ep_return_sum": torch.full((n,), -1.0, dtype=torch.float32, device="cuda"),
+           "ep_count": torch.full((n,), -1, dtype=torch.int32, device="cuda"),
+           "totals": torch.zeros(2, dtype=torch.int64, device="cuda")}
+    if final:
+        out["final_state"] = torch.zeros(4, n, dtype=torch.float32, device="cuda")
+    if streams:
+        out["done_bits"] = torch.zeros(T, words, dtype=torch.int32, device="cuda")
+        out["action_bits"] = torch.zeros(T, words, dtype=torch.int32, device="cuda")
+    return out
+
+
+def fetch(out):
+    torch.cuda.synchronize()
+    r = {k: host(v) for k, v in out.items()}
+    r["ep_count"] = r["ep_count"].view(np.uint32)
+    r["totals"] = r["totals"].view(np.uint64)
+    return r
+
+
+def pack_bits(bits):
+    T, n = bits.shape
+    words = (n + 31) // 32
+    padded = np.zeros((T, words * 32), np.uint8)
+    padded[:, :n] = bits
+    return np.packbits(padded, axis=1, bitorder="little").view(np.uint32).reshape(T, words)
+
+
+@pytest.mark.parametrize("limit", [1, 7, 50])
+@pytest.mark.parametrize("kind", [0, 1])
+def test_limited_rollout_against_oracle(cp, oracle, limit, kind):
+    n, T, seed, off = 5003, 120, 3, 64
+    w = inputs.policy_weights(kind, 4) if kind else None
+    out = outputs(n, T)
+    cp.cp_rollout_ex(n_envs=n, T=T, seed=seed, env_offset=off, policy=cp.policy(kind, w) if kind else None,
+                     max_episode_steps=limit, **out)
+    r = fetch(out)
+    o = oracle.rollout(n, T, seed, kind, w, env_offset=off, max_episode_steps=limit, done_bits=True,
+                       min_gap=True, nthreads=4)
+    H.assert_returns_match(r["ep_return_sum"], r["ep_count"], o["ep_return_sum"], o["ep_count"],
+                           o["min_gap"] < 1e-5)
+    gd, od = H.unpack_bits(r["done_bits"], n), H.unpack_bits(o["done_bits"], n)
+    same = r["ep_return_sum"] == o["ep_return_sum"]
+    assert same.mean() > 0.999
+    assert np.array_equal(gd[:, same], od[:, same])
+    # no episode outlives the limit
+    for i in range(0, n, 97):
+        times = np.concatenate(([-1], np.nonzero(gd[:, i])[0]))
+        assert np.diff(times).max(initial=0) <= limit and T - 1 - times[-1] < limit
+    if limit == 1:
+        assert np.all(r["ep_count"] == T) and np.all(r["ep_return_sum"] == T)
+    assert int(r["totals"][1]) == int(r["ep_count"].astype(np.int64).sum())
+
+
+def test_limit_that_is_never_reached_changes_nothing(cp):
+    n, T = 4000, 80
+    a, b = outputs(n, T), outputs(n, T)
+    cp.cp_rollout(n, T, 5, None, **a)
+    cp.cp_rollout_ex(n_envs=n, T=T, seed=5, max_episode_steps=T + 1, **b)
+    ra, rb = fetch(a), fetch(b)
+    for k in ra:
+        assert np.array_equal(ra[k], rb[k]), k
+
+
+def test_step_ex_equals_limited_rollout_and_chunks_resume(cp, oracle):
+    n, T, seed, limit = 3001, 60, 2, 9
+    whole = outputs(n, T)
+    cp.cp_rollout_ex(n_envs=n, T=T, seed=seed, max_episode_steps=limit, **whole)
+    rw = fetch(whole)
+    gd = H.unpack_bits(rw["done_bits"], n)
+    for vec_min in (0, 1 << 30):  # vector and scalar step kernels
+        cp.cp_tune("step_vec_min_envs", vec_min)
+        try:
+            planes = torch.zeros(4, (n + 3) // 4 * 4, device="cuda")
+            st = cp.cp_wrap(planes, n, seed)
+            cp.cp_fill_start(st)
+            ep_len = torch.zeros(n, dtype=torch.int32, device="cuda")
+            reward = torch.empty(n, device="cuda")
+            done = torch.empty(n, dtype=torch.uint8, device="cuda")
+            for t in range(T):
+                cp.cp_step_ex(st, None, st, reward, done, ep_len, limit)
+                torch.cuda.synchronize()
+                assert np.array_equal(host(done), gd[t]), t
+                assert int(ep_len.max()) < limit
+            assert np.array_equal(host(planes[:, :n]), rw["final_state"])
+        finally:
+            cp.cp_tune("step_vec_min_envs", 262144)
+    # the same rollout in three chunks on a batch, episode lengths carried between chunks
+    st = cp.cp_reset(n, seed)
+    ep_len = torch.zeros(n, dtype=torch.int32, device="cuda")
+    ret = np.zeros(n, np.float32)
+    cnt = np.zeros(n, np.uint32)
+    for chunk in (13, 1, 46):
+        o = outputs(n, chunk, streams=False, final=False)
+        cp.cp_rollout_ex(T=chunk, state=st, ep_len=ep_len, max_episode_steps=limit, **o)
+        r = fetch(o)
+        ret += r["ep_return_sum"]
+        cnt += r["ep_count"]
+    assert st.info()["t"] == T
+    assert np.array_equal(ret, rw["ep_return_sum"]) and np.array_equal(cnt, rw["ep_count"])
+    # one oracle step from the GPU's last state agrees with the GPU's next limited step
+    z = rw["final_state"]
+    tail = np.array([T - 1 - np.max(np.nonzero(gd[:, i])[0], initial=-1) for i in range(n)], np.uint32)
+    assert np.array_equal(host(ep_len).view(np.uint32), tail)
+    want = oracle.step_limited(z, seed, T, tail, limit)
+    planes = torch.zeros(4, (n + 3) // 4 * 4, device="cuda")
+    out_state = cp.cp_wrap(planes, n, seed)
+    done = torch.empty(n, dtype=torch.uint8, device="cuda")
+    cp.cp_step_ex(st, None, out_state, None, done, ep_len, limit)
+    torch.cuda.synchronize()
+    agree = host(done) == want["done"]
+    assert agree.mean() > 0.999
+    assert np.array_equal(host(ep_len).view(np.uint32)[agree], want["ep_len"][agree])
+    assert np.allclose(host(planes[:, :n])[:, agree], want["state"][:, agree], rtol=0, atol=2e-6)
+
+
+def test_supplied_action_stream(cp, oracle):
+    n, T, seed, off = 4099, 70, 8, 32
+    rng = np.random.default_rng(1)
+    acts = rng.integers(0, 2, (T, n)).astype(np.uint8)
+    bits = pack_bits(acts)
+    bits[:, -1] |= np.uint32((0xFFFFFFFF << (n % 32)) & 0xFFFFFFFF)  # garbage in the padding bits
+    d_bits = torch.from_numpy(bits.view(np.int32)).cuda()
+    for ept in (1, 2):
+        cp.cp_tune("rollout_ept", ept)
+        try:
+            out = outputs(n, T)
+            cp.cp_rollout_ex(n_envs=n, T=T, seed=seed, env_offset=off, action_bits_in=d_bits, **out)
+            r = fetch(out)
+        finally:
+            cp.cp_tune("rollout_ept", 0)
+        o = oracle.rollout(n, T, seed, env_offset=off, action_bits_in=pack_bits(acts), done_bits=True, nthreads=4)
+        H.assert_returns_match(r["ep_return_sum"], r["ep_count"], o["ep_return_sum"], o["ep_count"])
+        assert np.array_equal(H.unpack_bits(r["action_bits"], n), acts)  # echoed, padding masked off
+        same = r["ep_return_sum"] == o["ep_return_sum"]
+        assert np.array_equal(H.unpack_bits(r["done_bits"], n)[:, same], H.unpack_bits(o["done_bits"], n)[:, same])
+    # a supplied stream overrides a policy
+    w = inputs.policy_weights(1, 1)
+    out2 = outputs(n, T)
+    cp.cp_rollout_ex(n_envs=n, T=T, seed=seed, env_offset=off, policy=cp.policy(1, w), action_bits_in=d_bits, **out2)
+    r2 = fetch(out2)
+    assert np.array_equal(r2["ep_return_sum"], r["ep_return_sum"]) and np.array_equal(r2["final_state"], r["final_state"])
+    # feeding the hashed actions back in reproduces the random-policy rollout bit for bit
+    a = outputs(n, T)
+    cp.cp_rollout_shard(off, n, T, seed, None, **a)
+    ra = fetch(a)
+    b = outputs(n, T)
+    cp.cp_rollout_ex(n_envs=n, T=T, seed=seed, env_offset=off, action_bits_in=a["action_bits"], **b)
+    rb = fetch(b)
+    for k in ra:
+        assert np.array_equal(ra[k], rb[k]), k
+
+
+def test_general_call_argument_checks(cp):
+    L = cp.lib()
+    r = cp.cp_returns()
+    a = cp.cp_rollout_args()
+    a.struct_size = C.sizeof(cp.cp_rollout_args) - 8
+    a.n_envs, a.T = 64, 10
+    a.returns = C.pointer(r)
+    assert L.cp_rollout_ex(C.byref(a)) == cp.CP_EINVAL and b"struct_size" in L.cp_last_error()
+    a.struct_size = C.sizeof(cp.cp_rollout_args)
+    a.returns = None
+    assert L.cp_rollout_ex(C.byref(a)) == cp.CP_EINVAL
+    assert L.cp_rollout_ex(None) == cp.CP_EINVAL
+    n = 100
+    planes = torch.zeros(4, n, device="cuda")
+    st = cp.cp_wrap(planes, n, 0)
+    with pytest.raises(cp.CartpoleError) as e:
+        cp.cp_step_ex(st, None, st, None, None, None, 5)
+    assert e.value.code == cp.CP_EINVAL
+    before = cp.cp_launch_count()
+    with pytest.raises(cp.CartpoleError):
+        cp.cp_rollout_ex(n_envs=n, T=(1 << 30), seed=0, t0=5, totals=torch.zeros(2, dtype=torch.int64, device="cuda"))
+    assert cp.cp_launch_count() == before
