@@ -418,6 +418,25 @@ def measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args) -> dict:
                      "fused_step_over_ladder_hbm": out["fused_step_hbm"]["env_steps_per_sec"] / out["ladder_hbm"]["env_steps_per_sec"]}
     del a, b, sa, sb, reward, done, ws
 
+    # options of the general rollout call on the headline shape: CartPole-v1's 500-step episode
+    # limit, and actions supplied as a packed bit stream (here: the hashed ones, written by a
+    # first rollout) instead of drawn in the kernel
+    w3 = inputs.WORKLOADS["c3"]
+    n, T = w3.n_envs, w3.T
+    outs = {"ep_return_sum": torch.empty(n, device="cuda"), "ep_count": torch.empty(n, dtype=torch.int32, device="cuda"),
+            "totals": torch.zeros(2, dtype=torch.int64, device="cuda")}
+    act = torch.empty(T, (n + 31) // 32, dtype=torch.int32, device="cuda")
+    cp.cp_rollout(n, T, w3.seed, None, action_bits=act, **outs)
+    for key, kwargs in (("c3_rollout_step_limit_500", {"max_episode_steps": 500}),
+                        ("c3_rollout_supplied_actions", {"action_bits_in": act})):
+        def fn():
+            cp.cp_rollout_ex(n_envs=n, T=T, seed=w3.seed, **kwargs, **outs)
+        ms, _ = timed(fn, 10, 3)
+        ms /= 10
+        out[key] = {"n_envs": n, "T": T, "ms_per_launch": ms, "env_steps_per_sec": n * T / (ms * 1e-3)}
+    del outs, act
+    torch.cuda.empty_cache()
+
     # the other rollout configurations
     for name in ("c1", "c3", "c4", "c5", "paper"):
         w = inputs.WORKLOADS[name]

@@ -129,19 +129,22 @@ def test_step_ex_equals_limited_rollout_and_chunks_resume(cp, oracle):
         cnt += r["ep_count"]
     assert st.info()["t"] == T
     assert np.array_equal(ret, rw["ep_return_sum"]) and np.array_equal(cnt, rw["ep_count"])
-    # one oracle step from the GPU's last state agrees with the GPU's next limited step
-    z = rw["final_state"]
     tail = np.array([T - 1 - np.max(np.nonzero(gd[:, i])[0], initial=-1) for i in range(n)], np.uint32)
     assert np.array_equal(host(ep_len).view(np.uint32), tail)
-    want = oracle.step_limited(z, seed, T, tail, limit)
-    planes = torch.zeros(4, (n + 3) // 4 * 4, device="cuda")
-    out_state = cp.cp_wrap(planes, n, seed)
+    # one more limited step from the ORACLE's state and counters: GPU step vs oracle step
+    o = oracle.rollout(n, T, seed, max_episode_steps=limit, final_state=True, ep_len=np.zeros(n, np.uint32))
+    want = oracle.step_limited(o["final_state"], seed, T, o["ep_len"], limit)
+    planes_in = torch.zeros(4, (n + 3) // 4 * 4, device="cuda")
+    planes_in[:, :n] = torch.from_numpy(o["final_state"]).cuda()
+    planes = torch.zeros_like(planes_in)
+    s_in, out_state = cp.cp_wrap(planes_in, n, seed, T), cp.cp_wrap(planes, n, seed)
+    d_len = torch.from_numpy(o["ep_len"].view(np.int32)).cuda()
     done = torch.empty(n, dtype=torch.uint8, device="cuda")
-    cp.cp_step_ex(st, None, out_state, None, done, ep_len, limit)
+    cp.cp_step_ex(s_in, None, out_state, None, done, d_len, limit)
     torch.cuda.synchronize()
     agree = host(done) == want["done"]
     assert agree.mean() > 0.999
-    assert np.array_equal(host(ep_len).view(np.uint32)[agree], want["ep_len"][agree])
+    assert np.array_equal(host(d_len).view(np.uint32)[agree], want["ep_len"][agree])
     assert np.allclose(host(planes[:, :n])[:, agree], want["state"][:, agree], rtol=0, atol=2e-6)
 
 
