@@ -235,6 +235,29 @@ void co_mlp_logits(const float *w, const float z[4], float logits[2])
     }
 }
 
+/* The same network with H hidden units (kinds 4 and 5: H = 32 and 64):
+ * W1[H][4], b1[H], W2[2][H], b2[2] (7H + 2 floats), same chain order. */
+#define CO_POLICY_MLP32 4
+#define CO_POLICY_MLP64 5
+void co_mlp_logits_wide(const float *w, int H, const float z[4], float logits[2])
+{
+    const float *w1 = w;
+    const float *b1 = w + 4 * H;
+    const float *w2 = w + 5 * H;
+    const float *b2 = w + 7 * H;
+    float acc0 = b2[0], acc1 = b2[1];
+    for (int j = 0; j < H; ++j) {
+        float acc = b1[j];
+        for (int i = 0; i < 4; ++i)
+            acc = fmaf(w1[4 * j + i], z[i], acc);
+        float h = tanhf(acc);
+        acc0 = fmaf(w2[j], h, acc0);
+        acc1 = fmaf(w2[H + j], h, acc1);
+    }
+    logits[0] = acc0;
+    logits[1] = acc1;
+}
+
 /* Action for one environment; *gap (optional) receives |logit1 - logit0|
  * (infinity for the random policy) so tests can excuse argmax near-ties. */
 static int co_policy_action(int kind, const float *w, uint32_t ka0, uint32_t ka1, uint32_t t,
@@ -247,8 +270,10 @@ static int co_policy_action(int kind, const float *w, uint32_t ka0, uint32_t ka1
     }
     if (kind == CO_POLICY_LINEAR)
         co_linear_logits(w, z, logits);
-    else
+    else if (kind == CO_POLICY_MLP)
         co_mlp_logits(w, z, logits);
+    else
+        co_mlp_logits_wide(w, kind == CO_POLICY_MLP32 ? 32 : 64, z, logits);
     if (gap) *gap = fabsf(logits[1] - logits[0]);
     return logits[1] > logits[0];
 }

@@ -17,9 +17,10 @@ from dataclasses import dataclass
 
 import numpy as np
 
-POLICY_RANDOM, POLICY_LINEAR, POLICY_MLP = 0, 1, 2
-N_WEIGHTS = {POLICY_RANDOM: 0, POLICY_LINEAR: 10, POLICY_MLP: 114}
+POLICY_RANDOM, POLICY_LINEAR, POLICY_MLP, POLICY_MLP32, POLICY_MLP64 = 0, 1, 2, 4, 5
+N_WEIGHTS = {POLICY_RANDOM: 0, POLICY_LINEAR: 10, POLICY_MLP: 114, POLICY_MLP32: 226, POLICY_MLP64: 450}
 MLP_HIDDEN = 16
+HIDDEN_OF = {POLICY_MLP: 16, POLICY_MLP32: 32, POLICY_MLP64: 64}
 
 
 @dataclass(frozen=True)
@@ -58,9 +59,10 @@ def policy_weights(kind: int, seed: int) -> np.ndarray:
         return np.zeros(0, np.float32)
     if kind == POLICY_LINEAR:
         return (0.5 * rng.standard_normal(10)).astype(np.float32)
-    if kind == POLICY_MLP:
-        l1 = 0.5 * rng.standard_normal(4 * MLP_HIDDEN + MLP_HIDDEN)
-        l2 = 0.25 * rng.standard_normal(2 * MLP_HIDDEN + 2)
+    if kind in HIDDEN_OF:  # W1[H][4], b1[H] with std 1/sqrt(4); W2[2][H], b2[2] with std 1/sqrt(H)
+        h = HIDDEN_OF[kind]
+        l1 = 0.5 * rng.standard_normal(4 * h + h)
+        l2 = (1.0 / np.sqrt(h)) * rng.standard_normal(2 * h + 2)
         return np.concatenate([l1, l2]).astype(np.float32)
     raise ValueError(f"unknown policy kind {kind}")
 

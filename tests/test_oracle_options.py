@@ -148,3 +148,49 @@ def test_supplied_action_stream(oracle):
     c = oracle.rollout(8, 20, seed, action_bits_in=pack_bits(ones), done_bits=True)
     first = np.argmax(unpack_bits(c["done_bits"], 8), axis=0)
     assert np.all((first >= 6) & (first <= 12))
+
+
+@pytest.mark.parametrize("kind,hidden", [(inputs.POLICY_MLP32, 32), (inputs.POLICY_MLP64, 64)])
+def test_wider_mlp_policies(oracle, kind, hidden):
+    w = inputs.policy_weights(kind, 7)
+    assert w.size == 7 * hidden + 2
+    zs = inputs.random_states(100, seed=5, spread="live")
+    w1 = w[:4 * hidden].reshape(hidden, 4).astype(np.float64)
+    b1 = w[4 * hidden:5 * hidden].astype(np.float64)
+    w2 = w[5 * hidden:7 * hidden].reshape(2, hidden).astype(np.float64)
+    b2 = w[7 * hidden:].astype(np.float64)
+    for i in range(zs.shape[1]):
+        z = zs[:, i]
+        want = w2 @ np.tanh(w1 @ z.astype(np.float64) + b1) + b2
+        got = oracle.mlp_logits_wide(w, hidden, z)
+        assert np.all(np.abs(got - want) < 4e-6)
+    # one-hot probe isolates unit j, input 1 and both output rows
+    for j in (0, hidden // 2, hidden - 1):
+        probe = np.zeros(7 * hidden + 2, np.float32)
+        probe[4 * j + 1] = 2.0
+        probe[5 * hidden + j] = 1.0
+        probe[6 * hidden + j] = -3.0
+        probe[7 * hidden:] = (0.5, 0.25)
+        got = oracle.mlp_logits_wide(probe, hidden, [9, 0.1, 9, 9])
+        t = np.tanh(0.2)
+        assert abs(got[0] - (0.5 + t)) < 1e-6 and abs(got[1] - (0.25 - 3 * t)) < 1e-6
+    # rollouts use the pre-step observation and the tie rule
+    n, T = 32, 25
+    r = oracle.rollout(n, T, 0, kind, w, trajectory=True, action_bits=True, min_gap=True)
+    z = oracle.initial_state(n, 0)
+    for t in range(T):
+        ab = unpack_bits(r["action_bits"][t], n)
+        for i in range(n):
+            lg = oracle.mlp_logits_wide(w, hidden, z[:, i])
+            assert ab[i] == int(lg[1] > lg[0])
+        z = r["trajectory"][t]
+    assert np.all(np.isfinite(r["min_gap"]))
+
+
+def test_wide_mlp_routine_reduces_to_the_16_unit_network(oracle):
+    w = inputs.policy_weights(inputs.POLICY_MLP, 2)
+    zs = inputs.random_states(300, seed=6, spread="wide")
+    for i in range(zs.shape[1]):
+        a = oracle.mlp_logits(w, zs[:, i])
+        b = oracle.mlp_logits_wide(w, 16, zs[:, i])
+        assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
