@@ -437,6 +437,23 @@ def measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args) -> dict:
     del outs, act
     torch.cuda.empty_cache()
 
+    # wider in-kernel policies on config 5's shape (16,777,216 envs x 200 steps)
+    w5 = inputs.WORKLOADS["c5"]
+    n, T = w5.n_envs, w5.T
+    outs = {"ep_return_sum": torch.empty(n, device="cuda"), "ep_count": torch.empty(n, dtype=torch.int32, device="cuda"),
+            "totals": torch.zeros(2, dtype=torch.int64, device="cuda")}
+    for key, kind in (("c5_rollout_mlp32", inputs.POLICY_MLP32), ("c5_rollout_mlp64", inputs.POLICY_MLP64)):
+        pol = cp.policy(kind, inputs.policy_weights(kind, 3))
+
+        def fn():
+            cp.cp_rollout(n, T, w5.seed, pol, **outs)
+        ms, _ = timed(fn, 2, 3)
+        ms /= 2
+        out[key] = {"n_envs": n, "T": T, "hidden": inputs.HIDDEN_OF[kind], "ms_per_launch": ms,
+                    "env_steps_per_sec": n * T / (ms * 1e-3)}
+    del outs
+    torch.cuda.empty_cache()
+
     # the other rollout configurations
     for name in ("c1", "c3", "c4", "c5", "paper"):
         w = inputs.WORKLOADS[name]

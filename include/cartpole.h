@@ -82,6 +82,8 @@ extern "C" {
 #define CP_POLICY_LINEAR 1 /* argmax(W obs + b), W 2x4 */
 #define CP_POLICY_MLP 2    /* argmax(W2 tanh(W1 obs + b1) + b2), 4 -> 16 -> 2 */
 #define CP_MLP_HIDDEN 16
+#define CP_POLICY_MLP32 4  /* the same network with 32 hidden units (226 floats) */
+#define CP_POLICY_MLP64 5  /* ... with 64 hidden units (450 floats); kind 3 is not a policy */
 #define CP_MAX_T (1LL << 30)
 
 /* Opaque HOST handle of a batch: n_envs, plane_stride, seed, global step t,
@@ -92,7 +94,7 @@ typedef struct cp_state cp_state;
  * simulation with neural network inference", the paper's future work, Sec. VI).
  * weights is a HOST pointer, copied into the launch parameters by the call:
  *   linear: W[2][4] row-major, b[2]                         (10 floats)
- *   MLP:    W1[16][4], b1[16], W2[2][16], b2[2]             (114 floats)
+ *   MLP:    W1[H][4], b1[H], W2[2][H], b2[2], H = 16 / 32 / 64   (7H + 2 = 114 / 226 / 450 floats)
  * Each logit is a left-to-right chain acc = fmaf(w_i, v_i, acc) starting from the
  * bias; hidden units use accurate tanhf; action = (logit[1] > logit[0]), so a tie
  * pushes left. */

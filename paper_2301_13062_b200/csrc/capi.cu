@@ -70,7 +70,9 @@ int check_state(const cp_state *s, const char *name) {
 
 int check_policy(const cp_policy *policy, int *kind) {
     *kind = policy ? policy->kind : CP_POLICY_RANDOM;
-    if (*kind < CP_POLICY_RANDOM || *kind > CP_POLICY_MLP) return fail(CP_EINVAL, "unknown policy kind %d", *kind);
+    if (*kind != CP_POLICY_RANDOM && *kind != CP_POLICY_LINEAR && *kind != CP_POLICY_MLP &&
+        *kind != CP_POLICY_MLP32 && *kind != CP_POLICY_MLP64)
+        return fail(CP_EINVAL, "unknown policy kind %d", *kind);
     if (*kind != CP_POLICY_RANDOM && !policy->weights) return fail(CP_EINVAL, "policy weights are NULL");
     return CP_OK;
 }
@@ -152,6 +154,8 @@ int rollout_impl(uint32_t env_offset, int64_t n_envs, int64_t T, uint32_t seed, 
     p.action_bits_in = action_bits_in;
     if (kind == CP_POLICY_LINEAR) memcpy(p.w, policy->weights, 10 * sizeof(float));
     if (kind == CP_POLICY_MLP) memcpy(p.w, policy->weights, 114 * sizeof(float));
+    if (kind == CP_POLICY_MLP32) memcpy(p.w, policy->weights, 226 * sizeof(float));
+    if (kind == CP_POLICY_MLP64) memcpy(p.w, policy->weights, 450 * sizeof(float));
     const bool streams = p.reward_stream || p.done_bits || p.action_bits || p.trajectory;
     cudaError_t e = cp::launch_rollout(p, kind, streams, tl_stream);
     if (e != cudaSuccess) return cuda_fail(e, "rollout launch");

@@ -256,12 +256,14 @@ struct LinearW {
     float w[2][4];
     float b[2];
 };
-struct MlpW {
-    float w1[16][4];
-    float b1[16];
-    float w2[2][16];
+template <int H>
+struct MlpWT {  // 4 -> H (tanh) -> 2
+    float w1[H][4];
+    float b1[H];
+    float w2[2][H];
     float b2[2];
 };
+using MlpW = MlpWT<16>;
 
 // Returns the action in sign-bit form (0x80000000 = push right).
 __device__ __forceinline__ uint32_t linear_action(const LinearW &p, const State &z) {
@@ -277,10 +279,13 @@ __device__ __forceinline__ uint32_t linear_action(const LinearW &p, const State 
     return (l1 > l0) ? 0x80000000u : 0u;
 }
 
-__device__ __forceinline__ uint32_t mlp_action(const MlpW &p, const State &z) {
+// Hidden activations are consumed as they are produced (two running logits), so no array of
+// H values is ever live; every weight is an immediate operand from the launch parameters.
+template <int H>
+__device__ __forceinline__ uint32_t mlp_action(const MlpWT<H> &p, const State &z) {
     float l0 = p.b2[0], l1 = p.b2[1];
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
+    for (int j = 0; j < H; ++j) {
         float acc = p.b1[j];
         acc = __fmaf_rn(p.w1[j][0], z.x, acc);
         acc = __fmaf_rn(p.w1[j][1], z.xd, acc);

@@ -43,7 +43,7 @@ struct RolloutParams {
     float *trajectory;
     uint32_t max_steps;              // episode step limit, 0 = none
     const uint32_t *action_bits_in;  // [T][words] supplied actions or nullptr
-    float w[114];
+    float w[450];  // largest policy: MLP with 64 hidden units, 7*64 + 2 floats
 };
 
 struct LaunchTuning {

@@ -17,7 +17,8 @@
 
 namespace cp {
 
-// POLICY: 0 hashed random action, 1 linear, 2 MLP, 3 action bits supplied by the caller.
+// POLICY: 0 hashed random action, 1 linear, 2 MLP with 16 hidden units, 3 action bits supplied by
+// the caller, 4 / 5 MLP with 32 / 64 hidden units.
 template <int POLICY>
 __device__ __forceinline__ uint32_t policy_signbit(const RolloutParams &p, const Keys &ka, uint32_t t,
                                                    const State &z) {
@@ -25,8 +26,12 @@ __device__ __forceinline__ uint32_t policy_signbit(const RolloutParams &p, const
         return action_signbit(ka, t);
     } else if (POLICY == 1) {
         return linear_action(*reinterpret_cast<const LinearW *>(p.w), z);
+    } else if (POLICY == 2) {
+        return mlp_action<16>(*reinterpret_cast<const MlpWT<16> *>(p.w), z);
+    } else if (POLICY == 4) {
+        return mlp_action<32>(*reinterpret_cast<const MlpWT<32> *>(p.w), z);
     } else {
-        return mlp_action(*reinterpret_cast<const MlpW *>(p.w), z);
+        return mlp_action<64>(*reinterpret_cast<const MlpWT<64> *>(p.w), z);
     }
 }
 
@@ -238,7 +243,9 @@ cudaError_t launch_rollout(RolloutParams &p, int policy, bool streams, cudaStrea
         case 0: return launch_mode<0>(p, mode, ept, s);
         case 1: return launch_mode<1>(p, mode, ept, s);
         case 2: return launch_mode<2>(p, mode, ept, s);
-        default: return launch_mode<3>(p, mode, ept, s);
+        case 3: return launch_mode<3>(p, mode, ept, s);
+        case 4: return launch_mode<4>(p, mode, ept, s);
+        default: return launch_mode<5>(p, mode, ept, s);
     }
 }
 

@@ -207,3 +207,20 @@ def test_general_call_argument_checks(cp):
     with pytest.raises(cp.CartpoleError):
         cp.cp_rollout_ex(n_envs=n, T=(1 << 30), seed=0, t0=5, totals=torch.zeros(2, dtype=torch.int64, device="cuda"))
     assert cp.cp_launch_count() == before
+
+
+@pytest.mark.parametrize("kind", [inputs.POLICY_MLP32, inputs.POLICY_MLP64])
+def test_wider_mlp_policies_against_oracle(cp, oracle, kind):
+    n, T, seed = 20000, 150, 1
+    w = inputs.policy_weights(kind, 3)  # a draw for which both networks use both actions
+    out = outputs(n, T)
+    cp.cp_rollout(n, T, seed, cp.policy(kind, w), **out)
+    r = fetch(out)
+    o = oracle.rollout(n, T, seed, kind, w, action_bits=True, done_bits=True, min_gap=True, nthreads=8)
+    H.assert_returns_match(r["ep_return_sum"], r["ep_count"], o["ep_return_sum"], o["ep_count"],
+                           o["min_gap"] < 1e-5)
+    ga, oa = H.unpack_bits(r["action_bits"], n), H.unpack_bits(o["action_bits"], n)
+    gd, od = H.unpack_bits(r["done_bits"], n), H.unpack_bits(o["done_bits"], n)
+    agree = (ga == oa).all(axis=0) & (gd == od).all(axis=0)
+    assert agree.mean() >= 0.99
+    assert 0.02 < ga.mean() < 0.98  # the policy really decides: both actions occur
