@@ -23,10 +23,18 @@ N_WEIGHTS = {POLICY_RANDOM: 0, POLICY_LINEAR: 10, POLICY_MLP: 114, POLICY_MLP32:
 
 def build(force: bool = False) -> str:
     """Compile the oracle with strict float32 semantics (no contraction, no fast-math)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    import hashlib
+    with open(_SRC, "rb") as f:
+        want = hashlib.sha256(f.read()).hexdigest()
+    stamp = _LIB + ".stamp"
+    have = open(stamp).read().strip() if os.path.exists(stamp) else ""
+    if force or not os.path.exists(_LIB) or have != want:  # content hash, not file times
         cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared",
-               "-o", _LIB, _SRC, "-lm", "-lpthread"]
+               "-o", _LIB + ".tmp", _SRC, "-lm", "-lpthread"]
         subprocess.run(cmd, check=True)
+        os.replace(_LIB + ".tmp", _LIB)
+        with open(stamp, "w") as f:
+            f.write(want + "\n")
     return _LIB
 
 

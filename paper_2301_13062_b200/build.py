@@ -3,16 +3,24 @@
 Run as ``python -m paper_2301_13062_b200.build``. nvcc cross-compiles without a GPU.
 No fast-math; separate multiply/add are never contracted (``--fmad=false`` on top
 of the explicit round-to-nearest intrinsics in the kernels).
+
+The library is rebuilt when the hash of the sources and flags differs from the one
+recorded beside it at the last build (file times are not used: a copy of the tree keeps
+a valid library valid).
 """
 from __future__ import annotations
 
+import hashlib
 import os
 import subprocess
 import sys
+import tempfile
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcartpole.so")
+STAMP = os.path.join(HERE, "libcartpole.so.stamp")
 SOURCES = ["capi.cu", "step_kernel.cu", "ladder_kernels.cu", "rollout_kernel.cu", "ladder_noalloc.cu"]
 HEADERS = ["cartpole_device.cuh", "cartpole_internal.h", os.path.join("..", "..", "include", "cartpole.h")]
 
@@ -23,55 +31,53 @@ NVCC_FLAGS = [
 
 
 def _nvcc() -> str:
-    for cand in (os.environ.get("NVCC"), "/usr/local/cuda/bin/nvcc", "nvcc"):
-        if cand and (os.path.isabs(cand) and os.path.exists(cand) or not os.path.isabs(cand)):
+    for cand in (os.environ.get("NVCC"), "/usr/local/cuda/bin/nvcc"):
+        if cand and os.path.exists(cand):
             return cand
     return "nvcc"
 
 
-def _stale(target: str, deps: list[str]) -> bool:
-    if not os.path.exists(target):
-        return True
-    t = os.path.getmtime(target)
-    return any(os.path.getmtime(d) > t for d in deps)
+def source_hash(extra: list[str] | None = None) -> str:
+    h = hashlib.sha256()
+    for name in SOURCES + HEADERS:
+        with open(os.path.normpath(os.path.join(CSRC, name)), "rb") as f:
+            h.update(name.encode() + b"\0" + f.read() + b"\0")
+    h.update(" ".join(NVCC_FLAGS + (extra or [])).encode())
+    return h.hexdigest()
 
 
-def build(force: bool = False, verbose: bool = False, extra: list[str] | None = None, out: str | None = None) -> str:
-    """Compile and link. `extra` adds nvcc flags (e.g. -DCP_ROLLOUT_MIN_CTAS=5) and `out` names
-    another output file; both are for tuning experiments and force a full rebuild."""
-    if extra or out:
-        return _build_variant(extra or [], out or LIB, verbose)
-    hdrs = [os.path.normpath(os.path.join(CSRC, h)) for h in HEADERS] + [os.path.abspath(__file__)]
-    objs = []
-    for src in SOURCES:
-        s = os.path.join(CSRC, src)
-        o = os.path.join(CSRC, src.replace(".cu", ".o"))
-        if force or _stale(o, [s] + hdrs):
-            cmd = [_nvcc(), *NVCC_FLAGS, "-c", s, "-o", o]
-            if verbose:
-                cmd.insert(1, "-Xptxas=-v")
-                print(" ".join(cmd), flush=True)
-            subprocess.run(cmd, check=True)
-        objs.append(o)
-    if force or _stale(LIB, objs):
-        cmd = [_nvcc(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB, *objs]
-        subprocess.run(cmd, check=True)
-    return LIB
-
-
-def _build_variant(extra: list[str], out: str, verbose: bool) -> str:
-    import tempfile
+def _compile_and_link(out: str, extra: list[str], verbose: bool) -> None:
     with tempfile.TemporaryDirectory() as tmp:
-        objs = []
-        for src in SOURCES:
+        def compile_one(src: str) -> str:
             o = os.path.join(tmp, src.replace(".cu", ".o"))
             cmd = [_nvcc(), *NVCC_FLAGS, *extra, "-c", os.path.join(CSRC, src), "-o", o]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
+                print(" ".join(cmd), flush=True)
             subprocess.run(cmd, check=True)
-            objs.append(o)
-        subprocess.run([_nvcc(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", out, *objs], check=True)
-    return out
+            return o
+
+        with ThreadPoolExecutor(max_workers=len(SOURCES)) as pool:
+            objs = list(pool.map(compile_one, SOURCES))
+        tmp_out = out + ".tmp"
+        subprocess.run([_nvcc(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp_out, *objs],
+                       check=True)
+        os.replace(tmp_out, out)
+
+
+def build(force: bool = False, verbose: bool = False, extra: list[str] | None = None, out: str | None = None) -> str:
+    """Compile and link if needed. `extra` adds nvcc flags (e.g. -DCP_ROLLOUT_MIN_CTAS=5) and `out`
+    names another output file; both are for tuning experiments and always rebuild."""
+    if extra or out:
+        _compile_and_link(out or LIB, extra or [], verbose)
+        return out or LIB
+    want = source_hash()
+    have = open(STAMP).read().strip() if os.path.exists(STAMP) else ""
+    if force or not os.path.exists(LIB) or have != want:
+        _compile_and_link(LIB, [], verbose)
+        with open(STAMP, "w") as f:
+            f.write(want + "\n")
+    return LIB
 
 
 if __name__ == "__main__":

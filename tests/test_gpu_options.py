@@ -18,7 +18,8 @@ torch = pytest.importorskip("torch")
 def cp():
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
-    from paper_2301_13062_b200 import binding
+    from paper_2301_13062_b200 import binding, build
+    build.build()  # no-op when the in-tree library matches the sources
     binding.lib()
     torch.cuda.set_device(0)
     return binding

@@ -16,7 +16,8 @@ torch = pytest.importorskip("torch")
 def cp():
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
-    from paper_2301_13062_b200 import binding
+    from paper_2301_13062_b200 import binding, build
+    build.build()  # no-op when the in-tree library matches the sources
     binding.lib()  # raises if the library is missing: there is no fallback
     torch.cuda.set_device(0)
     return binding
