@@ -273,14 +273,14 @@ def main() -> None:
     h_tot = torch.empty(2, dtype=torch.int64).pin_memory()
 
     def e2e_step():
-        cp.cp_rollout_host(n, T, w.seed, pol, h_ret, h_cnt, h_tot)
+        cp.cp_rollout_host_shard(env_offset, n, T, w.seed, pol, h_ret, h_cnt, h_tot)
 
     e2e_ms, _ = timed(e2e_step, max(3, args.steps // 2), 3)
     e2e_ms /= max(3, args.steps // 2)
     e2e = {"value": world * n * T / (e2e_ms * 1e-3), "unit": UNIT,
            "h2d_bytes_per_step": int(4 * inputs.N_WEIGHTS[w.policy]) + 24, "d2h_bytes_per_step": 8 * n + 16,
            "ms_per_step": e2e_ms,
-           "note": "cp_rollout_host: host scalars (n_envs, T, seed) and policy weights in; per-env returns and "
+           "note": "cp_rollout_host_shard: host scalars (n_envs, T, seed) and policy weights in; per-env returns and "
                    "counts land in pinned host memory (stored there by the kernel over PCIe while it runs), "
                    "totals copied back, stream synchronised, every step"}
 

@@ -248,6 +248,9 @@ int cp_step_ex(cp_state *state, const uint8_t *action, cp_state *out_state, floa
  * overlaps the computation; pageable buffers are filled by copies after the kernel. */
 int cp_rollout_host(int64_t n_envs, int64_t T, uint32_t seed, const cp_policy *policy,
                     float *h_ep_return_sum, uint32_t *h_ep_count, uint64_t *h_totals);
+/* The same for the env range [env_offset, env_offset + n_envs) of a larger job (one range per GPU). */
+int cp_rollout_host_shard(uint32_t env_offset, int64_t n_envs, int64_t T, uint32_t seed, const cp_policy *policy,
+                          float *h_ep_return_sum, uint32_t *h_ep_count, uint64_t *h_totals);
 /* cp_step_host: h_planes_in/out [4][n_envs] (stride n_envs), h_action [n_envs] or NULL,
  * h_reward [n_envs], h_done [n_envs]; the step at global time t of envs 0..n_envs-1. */
 int cp_step_host(int64_t n_envs, uint32_t seed, uint32_t t, const float *h_planes_in,

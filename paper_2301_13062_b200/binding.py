@@ -28,7 +28,7 @@ EXPORTS = [
     "cp_rollout_from", "cp_rollout_host", "cp_step_host", "cp_shutdown", "cp_set_stream", "cp_tune",
     "cp_launch_count", "cp_selftest_sincos", "cp_last_error", "cp_version", "cp_step_unfused_noalloc",
     "cp_selftest_sincos_accuracy", "cp_selftest_arith", "cp_step_repeat", "cp_selftest_tame_div",
-    "cp_rollout_ex", "cp_step_ex",
+    "cp_rollout_ex", "cp_step_ex", "cp_rollout_host_shard",
 ]
 CP_NOALLOC_MAX_ENVS = 65536
 
@@ -87,6 +87,7 @@ def lib() -> C.CDLL:
             "cp_rollout_shard": (i32, [u32, i64, i64, u32, C.POINTER(cp_policy), C.POINTER(cp_returns)]),
             "cp_rollout_from": (i32, [p, i64, p, C.POINTER(cp_policy), C.POINTER(cp_returns)]),
             "cp_rollout_host": (i32, [i64, i64, u32, C.POINTER(cp_policy), p, p, p]),
+            "cp_rollout_host_shard": (i32, [u32, i64, i64, u32, C.POINTER(cp_policy), p, p, p]),
             "cp_step_host": (i32, [i64, u32, u32, p, p, p, p, p]),
             "cp_shutdown": (None, []),
             "cp_set_stream": (None, [p]),
@@ -317,9 +318,14 @@ def cp_step_ex(state: State, action, out_state: State, reward, done, ep_len, max
 
 
 def cp_rollout_host(n_envs: int, T: int, seed: int, policy: _Policy | None, h_ep_return_sum, h_ep_count, h_totals) -> None:
+    cp_rollout_host_shard(0, n_envs, T, seed, policy, h_ep_return_sum, h_ep_count, h_totals)
+
+
+def cp_rollout_host_shard(env_offset: int, n_envs: int, T: int, seed: int, policy: _Policy | None,
+                          h_ep_return_sum, h_ep_count, h_totals) -> None:
     _use_current_stream()
-    _check(lib().cp_rollout_host(n_envs, T, seed, policy.ref() if policy else None, _hptr(h_ep_return_sum),
-                                 _hptr(h_ep_count), _hptr(h_totals)))
+    _check(lib().cp_rollout_host_shard(env_offset, n_envs, T, seed, policy.ref() if policy else None,
+                                       _hptr(h_ep_return_sum), _hptr(h_ep_count), _hptr(h_totals)))
 
 
 def cp_step_host(n_envs: int, seed: int, t: int, h_planes_in, h_action, h_planes_out, h_reward, h_done) -> None:

@@ -423,7 +423,12 @@ int cp_rollout_ex(const cp_rollout_args *a) {
 
 int cp_rollout_host(int64_t n_envs, int64_t T, uint32_t seed, const cp_policy *policy, float *h_ep_return_sum,
                     uint32_t *h_ep_count, uint64_t *h_totals) {
-    int rc = check_range(n_envs, 0);
+    return cp_rollout_host_shard(0, n_envs, T, seed, policy, h_ep_return_sum, h_ep_count, h_totals);
+}
+
+int cp_rollout_host_shard(uint32_t env_offset, int64_t n_envs, int64_t T, uint32_t seed, const cp_policy *policy,
+                          float *h_ep_return_sum, uint32_t *h_ep_count, uint64_t *h_totals) {
+    int rc = check_range(n_envs, env_offset);
     if (rc != CP_OK) return rc;
     if (!h_ep_return_sum || !h_ep_count || !h_totals) return fail(CP_EINVAL, "a host output pointer is NULL");
     std::lock_guard<std::mutex> lock(g_staging.mu);
@@ -445,7 +450,8 @@ int cp_rollout_host(int64_t n_envs, int64_t T, uint32_t seed, const cp_policy *p
     r.totals = reinterpret_cast<uint64_t *>(base + 2 * per);
     cudaError_t e = cudaMemsetAsync(r.totals, 0, 16, tl_stream);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
-    if ((rc = rollout_impl(0, n_envs, T, seed, 0, policy, &r, nullptr, 0, nullptr, 0, nullptr)) != CP_OK) return rc;
+    if ((rc = rollout_impl(env_offset, n_envs, T, seed, 0, policy, &r, nullptr, 0, nullptr, 0, nullptr)) != CP_OK)
+        return rc;
     if (!direct) {
         e = cudaMemcpyAsync(h_ep_return_sum, r.ep_return_sum, (size_t)n_envs * 4, cudaMemcpyDeviceToHost, tl_stream);
         if (e == cudaSuccess)

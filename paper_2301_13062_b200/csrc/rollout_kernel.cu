@@ -79,7 +79,10 @@ __global__ void __launch_bounds__(256, CP_ROLLOUT_MIN_CTAS) rollout_kernel(const
                 z[j] = start_state(kr[j], p.t0);
             }
             cnt[j] = 0u;
-            begin[j] = p.t0 - (p.ep_len_io ? p.ep_len_io[idx[j]] : 0u);
+            // Only the step limit needs the carried-in length inside the loop; without it the
+            // counter is read once, at the end (loading it here costs four registers in the loop
+            // and 6 % of the stream variant's speed).
+            begin[j] = p.t0 - ((LIMIT && p.ep_len_io) ? p.ep_len_io[idx[j]] : 0u);
         }
 
         // Per-step stream outputs advance by one row per step: keep running pointers / offsets
@@ -156,11 +159,14 @@ __global__ void __launch_bounds__(256, CP_ROLLOUT_MIN_CTAS) rollout_kernel(const
         for (int j = 0; j < EPT; ++j) {
             if (!valid[j]) continue;
             // sum of the returns of the completed episodes = last termination time - time the first began
-            const uint32_t first_begin = p.t0 - (p.ep_len_io ? p.ep_len_io[idx[j]] : 0u);
+            const uint32_t carried = p.ep_len_io ? p.ep_len_io[idx[j]] : 0u;
+            const uint32_t first_begin = p.t0 - carried;
             const uint32_t ret = cnt[j] ? begin[j] - first_begin : 0u;
+            // begin[j] still holds t0 (LIMIT: t0 - carried) if no episode ended in this launch
+            const uint32_t running = t_end - begin[j] + ((!LIMIT && cnt[j] == 0u) ? carried : 0u);
             if (p.ep_return_sum) p.ep_return_sum[idx[j]] = (float)ret;
             if (p.ep_count) p.ep_count[idx[j]] = cnt[j];
-            if (p.ep_len_io) p.ep_len_io[idx[j]] = t_end - begin[j];
+            if (p.ep_len_io) p.ep_len_io[idx[j]] = running;
             if (p.out_planes) {
                 p.out_planes[idx[j]] = z[j].x;
                 p.out_planes[p.out_stride + idx[j]] = z[j].xd;
