@@ -376,6 +376,29 @@ def measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args) -> dict:
     del a, b, sa, sb, reward, done, ws
     torch.cuda.empty_cache()
 
+    # size sweep of the fused step, 2^16 .. 2^26 envs: launch-bound -> L2-resident -> HBM-bound
+    sweep = []
+    for lg in range(16, 27, 2):
+        n = 1 << lg
+        a, b, sa, sb, reward, done = step_setup(n)
+        cp.cp_rollout_from(sa, 40)
+        flip = {"f": False}
+
+        def one():
+            if flip["f"]:
+                cp.cp_step(sb, None, sa, reward, done)
+            else:
+                cp.cp_step(sa, None, sb, reward, done)
+            flip["f"] = not flip["f"]
+
+        ms, _ = timed(one, 10, 4)
+        ms /= 10
+        sweep.append({"n_envs": n, "us_per_launch": 1e3 * ms, "gbs": n * STEP_BYTES / (ms * 1e-3) / 1e9,
+                      "frac_of_hbm": n * STEP_BYTES / (ms * 1e-3) / hbm})
+        del a, b, sa, sb, reward, done
+        torch.cuda.empty_cache()
+    out["fused_step_sweep"] = sweep
+
     # config 2: 65,536 envs, per-step launches (launch-bound), 1,000 steps per timed iteration
     w2 = inputs.WORKLOADS["c2"]
     n = w2.n_envs

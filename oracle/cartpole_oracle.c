@@ -239,6 +239,7 @@ void co_mlp_logits(const float *w, const float z[4], float logits[2])
  * W1[H][4], b1[H], W2[2][H], b2[2] (7H + 2 floats), same chain order. */
 #define CO_POLICY_MLP32 4
 #define CO_POLICY_MLP64 5
+#define CO_POLICY_LINEAR_PER_ENV 6 /* one linear policy per environment (rollouts only) */
 void co_mlp_logits_wide(const float *w, int H, const float z[4], float logits[2])
 {
     const float *w1 = w;
@@ -363,6 +364,13 @@ static void co_rollout_range(co_rollout_job *J)
             if (J->action_bits_in) {
                 a = (int)((J->action_bits_in[k * words + i / 32] >> (i % 32)) & 1u);
                 gap = INFINITY;
+            } else if (J->kind == CO_POLICY_LINEAR_PER_ENV) {
+                /* every environment has its own linear policy: parameter q of env i at w[q*n + i]
+                 * (q = 0..7 the 2x4 matrix row-major, 8..9 the biases) */
+                float wi[10];
+                for (int q = 0; q < 10; ++q)
+                    wi[q] = J->w[q * n + i];
+                a = co_policy_action(CO_POLICY_LINEAR, wi, ka0, ka1, t, z, &gap);
             } else {
                 a = co_policy_action(J->kind, J->w, ka0, ka1, t, z, &gap);
             }

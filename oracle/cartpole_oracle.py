@@ -18,6 +18,7 @@ _SRC = os.path.join(_HERE, "cartpole_oracle.c")
 _LIB = os.path.join(_HERE, "libcartpole_oracle.so")
 
 POLICY_RANDOM, POLICY_LINEAR, POLICY_MLP, POLICY_MLP32, POLICY_MLP64 = 0, 1, 2, 4, 5
+POLICY_LINEAR_PER_ENV = 6
 N_WEIGHTS = {POLICY_RANDOM: 0, POLICY_LINEAR: 10, POLICY_MLP: 114, POLICY_MLP32: 226, POLICY_MLP64: 450}
 
 
@@ -215,7 +216,8 @@ def rollout(n: int, T: int, seed: int, policy_kind: int = POLICY_RANDOM, weights
     w = None
     if policy_kind != POLICY_RANDOM:
         w = np.ascontiguousarray(weights, np.float32).ravel()
-        assert w.size == N_WEIGHTS[policy_kind]
+        # kind 6: one linear policy per environment, weights [10, n] (parameter-major)
+        assert w.size == (10 * n if policy_kind == POLICY_LINEAR_PER_ENV else N_WEIGHTS[policy_kind])
     words = (n + 31) // 32
     res = {
         "ep_return_sum": np.empty(n, np.float32) if per_env else None,

@@ -21,6 +21,7 @@ POLICY_RANDOM, POLICY_LINEAR, POLICY_MLP, POLICY_MLP32, POLICY_MLP64 = 0, 1, 2, 
 N_WEIGHTS = {POLICY_RANDOM: 0, POLICY_LINEAR: 10, POLICY_MLP: 114, POLICY_MLP32: 226, POLICY_MLP64: 450}
 MLP_HIDDEN = 16
 HIDDEN_OF = {POLICY_MLP: 16, POLICY_MLP32: 32, POLICY_MLP64: 64}
+POLICY_LINEAR_PER_ENV = 6  # a different linear policy for every environment (population search)
 
 
 @dataclass(frozen=True)
@@ -65,6 +66,12 @@ def policy_weights(kind: int, seed: int) -> np.ndarray:
         l2 = (1.0 / np.sqrt(h)) * rng.standard_normal(2 * h + 2)
         return np.concatenate([l1, l2]).astype(np.float32)
     raise ValueError(f"unknown policy kind {kind}")
+
+
+def per_env_linear_weights(n: int, seed: int) -> np.ndarray:
+    """float32 [10, n]: one linear policy per environment, parameter-major (row q holds parameter
+    q of every env: rows 0-7 the 2x4 matrix row-major, rows 8-9 the biases), all N(0, std=0.5)."""
+    return (0.5 * np.random.default_rng(seed).standard_normal((10, n))).astype(np.float32)
 
 
 def random_states(n: int, seed: int, spread: str = "live") -> np.ndarray:

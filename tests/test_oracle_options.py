@@ -194,3 +194,31 @@ def test_wide_mlp_routine_reduces_to_the_16_unit_network(oracle):
         a = oracle.mlp_logits(w, zs[:, i])
         b = oracle.mlp_logits_wide(w, 16, zs[:, i])
         assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
+
+
+def test_per_env_linear_policies(oracle):
+    n, T, seed = 70, 40, 2
+    kind = inputs.POLICY_LINEAR_PER_ENV
+    wp = inputs.per_env_linear_weights(n, 5)
+    assert wp.shape == (10, n)
+    r = oracle.rollout(n, T, seed, kind, wp, trajectory=True, action_bits=True, done_bits=True, nthreads=3)
+    # brute force: every env is a one-env rollout of the shared linear policy with its own column
+    for i in range(0, n, 3):
+        one = oracle.rollout(1, T, seed, inputs.POLICY_LINEAR, wp[:, i], env_offset=i, trajectory=True)
+        assert np.array_equal(one["trajectory"][:, :, 0], r["trajectory"][:, :, i])
+        assert one["ep_return_sum"][0] == r["ep_return_sum"][i] and one["ep_count"][0] == r["ep_count"][i]
+    # the action at every step is the argmax of that env's own logits on the pre-step state
+    z = oracle.initial_state(n, seed)
+    for t in range(T):
+        ab = unpack_bits(r["action_bits"][t], n)
+        for i in range(n):
+            lg = oracle.linear_logits(wp[:, i], z[:, i])
+            assert ab[i] == int(lg[1] > lg[0])
+        z = r["trajectory"][t]
+    # identical columns reduce to the shared policy
+    w = inputs.policy_weights(inputs.POLICY_LINEAR, 1)
+    same = oracle.rollout(n, T, seed, kind, np.repeat(w[:, None], n, axis=1))
+    shared = oracle.rollout(n, T, seed, inputs.POLICY_LINEAR, w)
+    assert np.array_equal(same["ep_return_sum"], shared["ep_return_sum"])
+    # policies differ between envs: so do the outcomes
+    assert len(set(r["ep_return_sum"].tolist())) > 5
