@@ -457,7 +457,16 @@ def measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args) -> dict:
         ms, _ = timed(fn, 10, 3)
         ms /= 10
         out[key] = {"n_envs": n, "T": T, "ms_per_launch": ms, "env_steps_per_sec": n * T / (ms * 1e-3)}
-    del outs, act
+    # a population of linear policies, one per environment (weights read once into registers)
+    pop = cp.policy(cp.CP_POLICY_LINEAR_PER_ENV, torch.from_numpy(inputs.per_env_linear_weights(n, 11)).cuda())
+
+    def pop_fn():
+        cp.cp_rollout(n, T, w3.seed, pop, **outs)
+    ms, _ = timed(pop_fn, 10, 3)
+    ms /= 10
+    out["c3_rollout_per_env_linear"] = {"n_envs": n, "T": T, "ms_per_launch": ms,
+                                        "env_steps_per_sec": n * T / (ms * 1e-3)}
+    del outs, act, pop
     torch.cuda.empty_cache()
 
     # wider in-kernel policies on config 5's shape (16,777,216 envs x 200 steps)

@@ -84,6 +84,11 @@ extern "C" {
 #define CP_MLP_HIDDEN 16
 #define CP_POLICY_MLP32 4  /* the same network with 32 hidden units (226 floats) */
 #define CP_POLICY_MLP64 5  /* ... with 64 hidden units (450 floats); kind 3 is not a policy */
+#define CP_POLICY_LINEAR_PER_ENV 6 /* a different linear policy for every environment (population
+                                      search): `weights` is then a DEVICE pointer to [10][n_envs]
+                                      floats, parameter q of env i at weights[q * n_envs + i], rows
+                                      0-7 the 2x4 matrix row-major, rows 8-9 the biases; loaded into
+                                      registers once per launch */
 #define CP_MAX_T (1LL << 30)
 
 /* Opaque HOST handle of a batch: n_envs, plane_stride, seed, global step t,
@@ -100,7 +105,7 @@ typedef struct cp_state cp_state;
  * pushes left. */
 typedef struct cp_policy {
     int32_t kind;
-    const float *weights; /* HOST; NULL for CP_POLICY_RANDOM */
+    const float *weights; /* HOST (DEVICE for CP_POLICY_LINEAR_PER_ENV); NULL for CP_POLICY_RANDOM */
 } cp_policy;
 
 /* Outputs of a rollout; every pointer is DEVICE memory of the caller and may be

@@ -18,6 +18,7 @@ LIB_PATH = os.environ.get("CARTPOLE_LIB") or os.path.join(_HERE, "libcartpole.so
 
 CP_OK, CP_EINVAL, CP_ECUDA, CP_ENOMEM = 0, -1, -2, -3
 CP_POLICY_RANDOM, CP_POLICY_LINEAR, CP_POLICY_MLP, CP_POLICY_MLP32, CP_POLICY_MLP64 = 0, 1, 2, 4, 5
+CP_POLICY_LINEAR_PER_ENV = 6
 N_WEIGHTS = {CP_POLICY_RANDOM: 0, CP_POLICY_LINEAR: 10, CP_POLICY_MLP: 114, CP_POLICY_MLP32: 226,
              CP_POLICY_MLP64: 450}
 
@@ -148,7 +149,13 @@ class _Policy:
         self.kind = int(kind)
         self.weights = None
         self.struct = cp_policy(self.kind, None)
-        if self.kind != CP_POLICY_RANDOM:
+        if self.kind == CP_POLICY_LINEAR_PER_ENV:
+            # one linear policy per environment: a CUDA float32 tensor [10, n_envs], used in place
+            if not (weights.is_cuda and weights.is_contiguous() and weights.dim() == 2 and weights.shape[0] == 10):
+                raise ValueError("per-environment weights must be a contiguous CUDA tensor of shape [10, n_envs]")
+            self.weights = weights
+            self.struct.weights = weights.data_ptr()
+        elif self.kind != CP_POLICY_RANDOM:
             self.weights = np.ascontiguousarray(weights, np.float32).ravel()
             if self.weights.size != N_WEIGHTS.get(self.kind, -1):
                 raise ValueError(f"policy kind {kind} needs {N_WEIGHTS.get(self.kind)} weights, got {self.weights.size}")

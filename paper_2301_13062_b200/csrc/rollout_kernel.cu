@@ -18,7 +18,8 @@
 namespace cp {
 
 // POLICY: 0 hashed random action, 1 linear, 2 MLP with 16 hidden units, 3 action bits supplied by
-// the caller, 4 / 5 MLP with 32 / 64 hidden units.
+// the caller, 4 / 5 MLP with 32 / 64 hidden units, 6 one linear policy per environment (its ten
+// parameters are loaded into registers before the time loop; handled in the kernel body).
 template <int POLICY>
 __device__ __forceinline__ uint32_t policy_signbit(const RolloutParams &p, const Keys &ka, uint32_t t,
                                                    const State &z) {
@@ -54,6 +55,7 @@ __global__ void __launch_bounds__(256, CP_ROLLOUT_MIN_CTAS) rollout_kernel(const
         const int64_t base = task * (32 * EPT);
         State z[EPT];
         Keys ka[EPT], kr[EPT];
+        LinearW own[POLICY == 6 ? EPT : 1];  // per-environment policies live in registers
         // Episode bookkeeping: every step earns reward 1, so the returns of the episodes completed
         // in this launch add up to (time of the last termination) - (time the first of them began),
         // and only the count and the start time of the running episode need to live in the loop.
@@ -77,6 +79,13 @@ __global__ void __launch_bounds__(256, CP_ROLLOUT_MIN_CTAS) rollout_kernel(const
                 z[j].thd = p.init_planes[3 * p.init_stride + idx[j]];
             } else {
                 z[j] = start_state(kr[j], p.t0);
+            }
+            if (POLICY == 6) {  // parameter q of env i at env_weights[q*n + i]: coalesced per plane
+                LinearW &o = own[POLICY == 6 ? j : 0];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) o.w[q / 4][q % 4] = p.env_weights[(int64_t)q * p.n + idx[j]];
+                o.b[0] = p.env_weights[8 * p.n + idx[j]];
+                o.b[1] = p.env_weights[9 * p.n + idx[j]];
             }
             cnt[j] = 0u;
             // Only the step limit needs the carried-in length inside the loop; without it the
@@ -113,6 +122,8 @@ __global__ void __launch_bounds__(256, CP_ROLLOUT_MIN_CTAS) rollout_kernel(const
                 if (POLICY == 3) {
                     sb = (__ldg(act_ptr[j]) << (31u - lane)) & 0x80000000u;  // one word per warp, broadcast
                     act_ptr[j] += words;
+                } else if (POLICY == 6) {
+                    sb = linear_action(own[POLICY == 6 ? j : 0], z[j]);
                 } else {
                     sb = policy_signbit<POLICY>(p, ka[j], t, z[j]);
                 }
@@ -251,7 +262,8 @@ cudaError_t launch_rollout(RolloutParams &p, int policy, bool streams, cudaStrea
         case 2: return launch_mode<2>(p, mode, ept, s);
         case 3: return launch_mode<3>(p, mode, ept, s);
         case 4: return launch_mode<4>(p, mode, ept, s);
-        default: return launch_mode<5>(p, mode, ept, s);
+        case 5: return launch_mode<5>(p, mode, ept, s);
+        default: return launch_mode<6>(p, mode, ept, s);
     }
 }
 

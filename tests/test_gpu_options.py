@@ -225,3 +225,36 @@ def test_wider_mlp_policies_against_oracle(cp, oracle, kind):
     agree = (ga == oa).all(axis=0) & (gd == od).all(axis=0)
     assert agree.mean() >= 0.99
     assert 0.02 < ga.mean() < 0.98  # the policy really decides: both actions occur
+
+
+def test_per_env_linear_policies_against_oracle(cp, oracle):
+    n, T, seed, off = 30001, 200, 4, 96
+    wp = inputs.per_env_linear_weights(n, 11)
+    d_w = torch.from_numpy(wp).cuda()
+    res = []
+    for ept in (1, 2):
+        cp.cp_tune("rollout_ept", ept)
+        try:
+            out = outputs(n, T)
+            cp.cp_rollout_shard(off, n, T, seed, cp.policy(cp.CP_POLICY_LINEAR_PER_ENV, d_w), **out)
+            res.append(fetch(out))
+        finally:
+            cp.cp_tune("rollout_ept", 0)
+    for k in res[0]:
+        assert np.array_equal(res[0][k], res[1][k]), k
+    r = res[0]
+    o = oracle.rollout(n, T, seed, inputs.POLICY_LINEAR_PER_ENV, wp, env_offset=off, done_bits=True,
+                       action_bits=True, min_gap=True, nthreads=8)
+    H.assert_returns_match(r["ep_return_sum"], r["ep_count"], o["ep_return_sum"], o["ep_count"], o["min_gap"] < 1e-5)
+    agree = (H.unpack_bits(r["action_bits"], n) == H.unpack_bits(o["action_bits"], n)).all(axis=0)
+    assert agree.mean() >= 0.995
+    # identical columns reproduce the shared linear policy bit for bit
+    w = inputs.policy_weights(1, 1)
+    a, b = outputs(n, T), outputs(n, T)
+    cp.cp_rollout(n, T, seed, cp.policy(1, w), **a)
+    cp.cp_rollout(n, T, seed, cp.policy(cp.CP_POLICY_LINEAR_PER_ENV, torch.from_numpy(np.repeat(w[:, None], n, axis=1)).cuda()), **b)
+    ra, rb = fetch(a), fetch(b)
+    for k in ra:
+        assert np.array_equal(ra[k], rb[k]), k
+    # fitness differs across the population
+    assert r["ep_return_sum"].std() > 1 and len(set(r["ep_count"].tolist())) > 5
