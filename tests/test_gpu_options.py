@@ -186,6 +186,29 @@ def test_supplied_action_stream(cp, oracle):
         assert np.array_equal(ra[k], rb[k]), k
 
 
+def test_long_horizons_and_late_global_times(cp, oracle):
+    """Few environments for very many steps, and a rollout that ends at the largest global time the
+    hash counters allow (t0 + T = 2^30): the 32-bit time arithmetic agrees with the oracle's."""
+    n, T = 64, 200_000
+    out = outputs(n, T, streams=False)
+    cp.cp_rollout(n, T, 7, None, **out)
+    r = fetch(out)
+    o = oracle.rollout(n, T, 7, final_state=True, nthreads=4)
+    assert (r["ep_return_sum"] == o["ep_return_sum"]).mean() >= 0.95  # 64 envs x 200,000 steps: a flip or two
+    assert abs(float(r["ep_return_sum"].sum()) - float(o["ep_return_sum"].sum())) <= 200
+    assert r["ep_return_sum"].max() <= T and r["ep_return_sum"].min() > T - 500
+    n, T = 3000, 500
+    t0 = (1 << 30) - T
+    out = outputs(n, T)
+    cp.cp_rollout_ex(n_envs=n, T=T, seed=9, t0=t0, max_episode_steps=40, **out)
+    r = fetch(out)
+    o = oracle.rollout(n, T, 9, t0=t0, max_episode_steps=40, done_bits=True, action_bits=True)
+    H.assert_returns_match(r["ep_return_sum"], r["ep_count"], o["ep_return_sum"], o["ep_count"])
+    assert np.array_equal(H.unpack_bits(r["action_bits"], n), H.unpack_bits(o["action_bits"], n))
+    with pytest.raises(cp.CartpoleError):
+        cp.cp_rollout_ex(n_envs=n, T=T + 1, seed=9, t0=t0, **outputs(n, T + 1, streams=False))
+
+
 def test_general_call_argument_checks(cp):
     L = cp.lib()
     r = cp.cp_returns()
