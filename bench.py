@@ -450,8 +450,15 @@ def measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args) -> dict:
             "totals": torch.zeros(2, dtype=torch.int64, device="cuda")}
     act = torch.empty(T, (n + 31) // 32, dtype=torch.int32, device="cuda")
     cp.cp_rollout(n, T, w3.seed, None, action_bits=act, **outs)
+    # ... and the contracted arithmetic (fused multiply-adds, folded constants): within the
+    # tolerances, but not the bits of the per-op ladder, so never the headline
+    mlp_pol = cp.policy(inputs.POLICY_MLP, inputs.policy_weights(inputs.POLICY_MLP, inputs.WORKLOADS["c5"].policy_seed))
     for key, kwargs in (("c3_rollout_step_limit_500", {"max_episode_steps": 500}),
-                        ("c3_rollout_supplied_actions", {"action_bits_in": act})):
+                        ("c3_rollout_supplied_actions", {"action_bits_in": act}),
+                        ("c3_rollout_contracted_arithmetic", {"arithmetic": cp.CP_ARITH_CONTRACTED}),
+                        ("c3_rollout_mlp", {"policy": mlp_pol}),
+                        ("c3_rollout_mlp_contracted_arithmetic",
+                         {"policy": mlp_pol, "arithmetic": cp.CP_ARITH_CONTRACTED})):
         def fn():
             cp.cp_rollout_ex(n_envs=n, T=T, seed=w3.seed, **kwargs, **outs)
         ms, _ = timed(fn, 10, 3)

@@ -216,13 +216,29 @@ int cp_rollout_from(cp_state *state, int64_t T, uint32_t *ep_len, const cp_polic
  *     length added to ep_return_sum, counted in ep_count — and the environment restarts;
  *   - actions given as data instead of drawn by a policy (the paper's baseline, Sec. V-A, feeds
  *     precomputed random values): action_bits_in DEVICE [T][ceil(n_envs/32)], bit (i%32) of word
- *     (i/32) of row k = action of env i at the k-th step of this call; overrides `policy`.
+ *     (i/32) of row k = action of env i at the k-th step of this call; overrides `policy`;
+ *   - a choice of arithmetic. CP_ARITH_EXACT (0, what every other entry point uses): each operation
+ *     of the step rounded once, in the order of the per-op ladder, so that ladder, fused step and
+ *     rollout give the same bits. CP_ARITH_CONTRACTED: the step as a contracting compiler would
+ *     emit it for a fused kernel (Sec. V-B, V-G: generated fused code carries no such promise) —
+ *     fused multiply-adds, divisions by the total mass folded into constants, theta_acc by
+ *     reciprocal; 25 instead of 43 floating-point operations per step. One step from the same
+ *     state differs by at most 2e-6 relative (on the scale of value and update) and a done flag
+ *     only where x' or theta' lies within 1e-5 of its threshold. Start states, actions of the
+ *     hashed policy and the bookkeeping are the same bits in both. Free-running returns stay
+ *     identical on more than 99.9 % of environments when the actions do not depend on the state
+ *     (hashed or supplied actions: every restart re-synchronises the two arithmetics); under a
+ *     state-feedback policy the per-step differences are amplified through the action choice and
+ *     only the statistics (mean return, episode count) agree — use CP_ARITH_EXACT where
+ *     reproducibility against the per-op order matters.
  * struct_size must be sizeof(cp_rollout_args) (guards against a caller built for another layout).
  * state == NULL: start states of global time t0, env range [env_offset, env_offset + n_envs);
  * state != NULL: that batch is advanced in place from its own time (n_envs, seed, env_offset, t0 of
  * the struct are ignored, returns->final_state too) and state->t grows by T.
  * ep_len: DEVICE [n_envs] steps already taken in each running episode, read and rewritten, or NULL
  * (all episodes start at this call; nothing written). t0 + T <= CP_MAX_T. */
+#define CP_ARITH_EXACT 0u
+#define CP_ARITH_CONTRACTED 1u
 typedef struct cp_rollout_args {
     uint32_t struct_size;
     uint32_t env_offset;
@@ -233,6 +249,7 @@ typedef struct cp_rollout_args {
     cp_state *state;               /* or NULL */
     uint32_t *ep_len;              /* DEVICE or NULL */
     uint32_t max_episode_steps;    /* 0 = no limit */
+    uint32_t arithmetic;           /* CP_ARITH_EXACT or CP_ARITH_CONTRACTED */
     const uint32_t *action_bits_in; /* DEVICE or NULL */
 } cp_rollout_args;
 int cp_rollout_ex(const cp_rollout_args *args);

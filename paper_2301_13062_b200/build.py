@@ -21,8 +21,9 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcartpole.so")
 STAMP = os.path.join(HERE, "libcartpole.so.stamp")
-SOURCES = ["capi.cu", "step_kernel.cu", "ladder_kernels.cu", "rollout_kernel.cu", "ladder_noalloc.cu"]
-HEADERS = ["cartpole_device.cuh", "cartpole_internal.h", os.path.join("..", "..", "include", "cartpole.h")]
+SOURCES = ["capi.cu", "step_kernel.cu", "ladder_kernels.cu", "rollout_kernel.cu", "rollout_contracted.cu",
+           "ladder_noalloc.cu"]
+HEADERS = ["cartpole_device.cuh", "cartpole_internal.h", "rollout_kernel.cuh", os.path.join("..", "..", "include", "cartpole.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "--fmad=false",

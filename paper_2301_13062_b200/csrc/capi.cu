@@ -124,8 +124,10 @@ void advance(cp_state *state, cp_state *out_state, uint32_t steps) {
 int rollout_impl(uint32_t env_offset, int64_t n_envs, int64_t T, uint32_t seed, uint32_t t0, const cp_policy *policy,
                  const cp_returns *ret, const float *init_planes, int64_t init_stride, float *out_planes,
                  int64_t out_stride, uint32_t *ep_len, uint32_t max_steps = 0,
-                 const uint32_t *action_bits_in = nullptr) {
+                 const uint32_t *action_bits_in = nullptr, uint32_t arithmetic = CP_ARITH_EXACT) {
     int kind, rc;
+    if (arithmetic != CP_ARITH_EXACT && arithmetic != CP_ARITH_CONTRACTED)
+        return fail(CP_EINVAL, "arithmetic must be CP_ARITH_EXACT or CP_ARITH_CONTRACTED (got %u)", arithmetic);
     if ((rc = check_range(n_envs, env_offset)) != CP_OK) return rc;
     if (T <= 0 || T > CP_MAX_T || (int64_t)t0 + T > CP_MAX_T)
         return fail(CP_EINVAL, "T must be in [1, 2^30] and t0 + T <= 2^30 (got T=%lld, t0=%u)", (long long)T, t0);
@@ -160,7 +162,7 @@ int rollout_impl(uint32_t env_offset, int64_t n_envs, int64_t T, uint32_t seed, 
     if (kind == CP_POLICY_MLP64) memcpy(p.w, policy->weights, 450 * sizeof(float));
     if (kind == CP_POLICY_LINEAR_PER_ENV) p.env_weights = policy->weights;  // DEVICE [10][n_envs]
     const bool streams = p.reward_stream || p.done_bits || p.action_bits || p.trajectory;
-    cudaError_t e = cp::launch_rollout(p, kind, streams, tl_stream);
+    cudaError_t e = cp::launch_rollout(p, kind, streams, arithmetic == CP_ARITH_CONTRACTED, tl_stream);
     if (e != cudaSuccess) return cuda_fail(e, "rollout launch");
     return CP_OK;
 }
@@ -415,13 +417,14 @@ int cp_rollout_ex(const cp_rollout_args *a) {
         if (rc != CP_OK) return rc;
         cp_state *st = a->state;
         rc = rollout_impl(st->env_offset, st->n, a->T, st->seed, st->t, a->policy, a->returns, st->planes, st->stride,
-                          st->planes, st->stride, a->ep_len, a->max_episode_steps, a->action_bits_in);
+                          st->planes, st->stride, a->ep_len, a->max_episode_steps, a->action_bits_in, a->arithmetic);
         if (rc != CP_OK) return rc;
         st->t += (uint32_t)a->T;
         return CP_OK;
     }
     return rollout_impl(a->env_offset, a->n_envs, a->T, a->seed, a->t0, a->policy, a->returns, nullptr, 0,
-                        a->returns->final_state, a->n_envs, a->ep_len, a->max_episode_steps, a->action_bits_in);
+                        a->returns->final_state, a->n_envs, a->ep_len, a->max_episode_steps, a->action_bits_in,
+                        a->arithmetic);
 }
 
 int cp_rollout_host(int64_t n_envs, int64_t T, uint32_t seed, const cp_policy *policy, float *h_ep_return_sum,

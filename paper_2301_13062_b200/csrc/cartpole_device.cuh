@@ -251,6 +251,39 @@ __device__ __forceinline__ bool euler_step(State &z, float force) {
     return (fabsf(nx) > kXT) | (fabsf(nth) > kTT);
 }
 
+// ---- contracted arithmetic (an optional, separately reported rollout variant) ----
+// The same step with the roundings a compiler allowed to contract would drop (the paper's
+// fused kernels are generated without a one-rounding-per-op promise, Sec. V-B/V-G): fused
+// multiply-adds in temp, num, den, xacc and the four Euler updates, the divisions by the
+// total mass folded into constants, theta_acc = num * rcp(den) with the hardware reciprocal
+// (den lies in [0.62, 0.67] for every real c). 25 floating-point operations instead of 43.
+// Results differ from the canonical order by a few 1e-7 relative per step; they are NOT the
+// bits of the per-op ladder. sin / cos are the same routines as in the exact path.
+constexpr float kDenK = (float)(-(0.5 * 0.1) / (double)1.1f);    // -l * m_p / M
+constexpr float kDenC = (float)(0.5 * (4.0 / 3.0));              // l * 4/3
+constexpr float kXaccK = (float)(-(0.1 * 0.5) / (double)1.1f);   // -m_p * l / M
+__device__ __forceinline__ bool euler_step_contracted(State &z, float force) {
+    float s, c;
+    sin_cos(z.th, s, c);
+    const float t1 = __fmul_rn(__fmul_rn(z.thd, z.thd), kPML);
+    const float temp = __fmul_rn(__fmaf_rn(t1, s, force), kRcpMTot);
+    const float num = __fmaf_rn(-c, temp, __fmul_rn(kG, s));
+    const float den = __fmaf_rn(__fmul_rn(c, c), kDenK, kDenC);
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(den));
+    const float thacc = __fmul_rn(num, r);
+    const float xacc = __fmaf_rn(__fmul_rn(thacc, c), kXaccK, temp);
+    const float nx = __fmaf_rn(kTau, z.xd, z.x);
+    const float nxd = __fmaf_rn(kTau, xacc, z.xd);
+    const float nth = __fmaf_rn(kTau, z.thd, z.th);
+    const float nthd = __fmaf_rn(kTau, thacc, z.thd);
+    z.x = nx;
+    z.xd = nxd;
+    z.th = nth;
+    z.thd = nthd;
+    return (fabsf(nx) > kXT) | (fabsf(nth) > kTT);
+}
+
 // ---- policies (observation = state before the step) ----
 struct LinearW {
     float w[2][4];

@@ -71,7 +71,8 @@ cudaError_t launch_fill_start(float *planes, int64_t stride, int64_t n, uint32_t
                               uint32_t t, cudaStream_t s);
 cudaError_t launch_actions(uint8_t *out, int64_t n, uint32_t env_offset, uint32_t salt_a, uint32_t t,
                            cudaStream_t s);
-cudaError_t launch_rollout(RolloutParams &p, int policy, bool streams, cudaStream_t s);
+cudaError_t launch_rollout(RolloutParams &p, int policy, bool streams, bool contracted, cudaStream_t s);
+cudaError_t launch_rollout_contracted(RolloutParams &p, int policy, bool streams, cudaStream_t s);
 cudaError_t launch_sincos_selftest(uint32_t lo_bits, uint32_t hi_bits, unsigned long long *mismatches,
                                    cudaStream_t s);
 

@@ -20,6 +20,7 @@ def main() -> None:
     ap.add_argument("--T", type=int, default=100)
     ap.add_argument("--policy", default="random", choices=["random", "linear", "mlp"])
     ap.add_argument("--streams", action="store_true", help="rollout: also write the reward plane and done bitmask")
+    ap.add_argument("--contracted", action="store_true", help="rollout: contracted arithmetic (CP_ARITH_CONTRACTED)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=1)
@@ -48,7 +49,10 @@ def main() -> None:
             outs["done_bits"] = torch.empty(T, (n + 31) // 32, dtype=torch.int32, device="cuda")
 
         def fn():
-            cp.cp_rollout(n, T, args.seed, pol, **outs)
+            if args.contracted:
+                cp.cp_rollout_ex(n_envs=n, T=T, seed=args.seed, policy=pol, arithmetic=cp.CP_ARITH_CONTRACTED, **outs)
+            else:
+                cp.cp_rollout(n, T, args.seed, pol, **outs)
         units = n * T
     else:
         stride = (n + 3) // 4 * 4

@@ -1,0 +1,163 @@
+"""GPU tests of the contracted-arithmetic rollout (CP_ARITH_CONTRACTED): the same step with fused
+multiply-adds and folded constants. It is not bit-identical to the canonical order, so it is held
+to the tolerances themselves against the (unchanged, canonical) CPU oracle: one step from the same
+state within 2e-6 relative, done flags equal outside the 1e-5 threshold band, start states and
+hashed actions bit-exact, free-running returns identical on >= 99.9 % of environments."""
+import numpy as np
+import pytest
+
+from paper_2301_13062_b200 import inputs
+from tests import gpu_helpers as H
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def cp():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2301_13062_b200 import binding, build
+    build.build()
+    binding.lib()
+    torch.cuda.set_device(0)
+    return binding
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def host(t):
+    return t.cpu().numpy()
+
+
+def contracted_step(cp, z, seed, t, env_offset, general_streams, ept):
+    """One step of the contracted rollout kernel from the given states."""
+    n = z.shape[1]
+    planes = torch.zeros(4, (n + 3) // 4 * 4, dtype=torch.float32, device="cuda")
+    planes[:, :n] = dev(z)
+    st = cp.cp_wrap(planes, n, seed, t, env_offset)
+    words = (n + 31) // 32
+    out = {"reward_stream": torch.zeros(1, n, device="cuda"),
+           "done_bits": torch.zeros(1, words, dtype=torch.int32, device="cuda")}
+    if general_streams:
+        out["action_bits"] = torch.zeros(1, words, dtype=torch.int32, device="cuda")
+    cp.cp_tune("rollout_ept", ept)
+    try:
+        cp.cp_rollout_ex(state=st, T=1, arithmetic=cp.CP_ARITH_CONTRACTED, **out)
+    finally:
+        cp.cp_tune("rollout_ept", 0)
+    torch.cuda.synchronize()
+    assert st.info()["t"] == t + 1
+    act = H.unpack_bits(host(out["action_bits"]), n)[0] if general_streams else None
+    return host(planes[:, :n]), host(out["reward_stream"])[0], H.unpack_bits(host(out["done_bits"]), n)[0], act
+
+
+@pytest.mark.parametrize("spread", ["start", "live", "edge", "wide"])
+@pytest.mark.parametrize("n", [1, 33, 1025, 65537])
+def test_one_contracted_step_within_tolerance_of_the_oracle(cp, oracle, spread, n):
+    z = inputs.random_states(n, seed=3 * n + len(spread), spread=spread)
+    worst = 0.0
+    for (off, t, general, ept) in ((0, 0, False, 2), (4321, 17, True, 1)):
+        want = oracle.step(z, seed=1, t=t, env_offset=off, want_pre_reset=True)
+        state, reward, done, act = contracted_step(cp, z, 1, t, off, general, ept)
+        stats = H.assert_step_matches(want, z, state, reward, done, act)
+        worst = max(worst, 1.0 - stats["bit_exact_fraction"])
+    if spread == "live" and n >= 1025:
+        # a sanity check that the variant really ran: its roundings differ from the canonical order
+        assert worst > 0.01
+
+
+def rollout(cp, n, T, seed, kind=0, weights=None, arithmetic=1, **extra):
+    out = {"ep_return_sum": torch.full((n,), -1.0, device="cuda"),
+           "ep_count": torch.full((n,), -1, dtype=torch.int32, device="cuda"),
+           "totals": torch.zeros(2, dtype=torch.int64, device="cuda")}
+    out.update(extra)
+    pol = cp.policy(kind, weights) if kind else None
+    cp.cp_rollout_ex(n_envs=n, T=T, seed=seed, policy=pol, arithmetic=arithmetic, **out)
+    torch.cuda.synchronize()
+    res = {k: host(v) for k, v in out.items()}
+    res["ep_count"] = res["ep_count"].view(np.uint32)
+    return res
+
+
+def test_contracted_random_rollout_returns_match_the_oracle(cp, oracle):
+    w = inputs.WORKLOADS["c1"]
+    n, T, words = 50001, 400, (50001 + 31) // 32
+    r = rollout(cp, n, T, w.seed, action_bits=torch.zeros(T, words, dtype=torch.int32, device="cuda"),
+                done_bits=torch.zeros(T, words, dtype=torch.int32, device="cuda"))
+    o = oracle.rollout(n, T, w.seed, action_bits=True, done_bits=True, nthreads=4)
+    # hashed actions do not depend on the arithmetic: bit-exact
+    assert np.array_equal(r["action_bits"].view(np.uint32), o["action_bits"].view(np.uint32))
+    s = H.assert_returns_match(r["ep_return_sum"], r["ep_count"], o["ep_return_sum"], o["ep_count"])
+    gd, od = H.unpack_bits(r["done_bits"], n), H.unpack_bits(o["done_bits"], n)
+    assert (gd == od).all(axis=0).mean() >= 0.999
+    assert int(r["totals"][0]) == int(r["ep_return_sum"].astype(np.int64).sum())
+    assert 21.5 < s["mean_gpu"] < 22.5
+
+
+@pytest.mark.parametrize("kind,pseed,T", [(1, 1, 300), (2, 2, 200)])
+def test_contracted_policy_rollouts_stay_statistically_equal(cp, oracle, kind, pseed, T):
+    """With a state-feedback policy the 1e-7 per-step differences feed back through the action
+    choice (an unstable pendulum amplifies them until some logit pair falls on the other side of
+    a tie), so per-env return identity is NOT held to 99.9 % here — which is why this arithmetic
+    is an option and not the parity path. What must hold: most envs identical, mean return and
+    episode count within 0.1 % / 0.2 %."""
+    n = 40000
+    wts = inputs.policy_weights(kind, pseed)
+    r = rollout(cp, n, T, 0, kind, wts)
+    o = oracle.rollout(n, T, 0, kind, wts, min_gap=True, nthreads=4)
+    s = H.assert_returns_match(r["ep_return_sum"], r["ep_count"], o["ep_return_sum"], o["ep_count"],
+                               excuse=o["min_gap"] < 1e-5, min_identical=0.9)
+    print(f"contracted, policy kind {kind}: identical returns on {s['identical']:.4f} of envs, "
+          f"mean {s['mean_gpu']:.4f} vs {s['mean_oracle']:.4f}")
+    episodes_gpu, episodes_oracle = int(r["ep_count"].sum()), int(o["ep_count"].sum())
+    assert abs(episodes_gpu - episodes_oracle) <= 2e-3 * episodes_oracle
+
+
+def test_full_size_contracted_rollout_against_the_oracle(cp, oracle):
+    """1,048,576 envs x 500 steps in the benchmark's launch configuration."""
+    import os
+    w = inputs.WORKLOADS["c3"]
+    r = rollout(cp, w.n_envs, w.T, w.seed)
+    o = oracle.rollout(w.n_envs, w.T, w.seed, nthreads=os.cpu_count() or 1)
+    H.assert_returns_match(r["ep_return_sum"], r["ep_count"], o["ep_return_sum"], o["ep_count"])
+
+
+def test_contracted_chunks_and_step_limit_compose(cp):
+    """GPU-internal: chunked contracted rollouts with carried episode lengths and a step limit give
+    the bits of one long contracted rollout, and differ from nothing but arithmetic."""
+    n, T, seed, limit = 3001, 240, 4, 60
+    wts = inputs.policy_weights(1, 11)  # linear policy: some episodes reach the limit
+    pol = cp.policy(1, wts)
+
+    def run(chunks):
+        planes = torch.zeros(4, (n + 3) // 4 * 4, device="cuda")
+        st = cp.cp_wrap(planes, n, seed)
+        cp.cp_fill_start(st)
+        ep_len = torch.zeros(n, dtype=torch.int32, device="cuda")
+        ret_total = np.zeros(n, np.float64)
+        cnt_total = np.zeros(n, np.int64)
+        for Tc in chunks:
+            ret = torch.empty(n, device="cuda")
+            cnt = torch.empty(n, dtype=torch.int32, device="cuda")
+            cp.cp_rollout_ex(state=st, T=Tc, policy=pol, ep_len=ep_len, max_episode_steps=limit,
+                             arithmetic=cp.CP_ARITH_CONTRACTED, ep_return_sum=ret, ep_count=cnt)
+            torch.cuda.synchronize()
+            ret_total += host(ret)
+            cnt_total += host(cnt)
+        return host(planes[:, :n]), ret_total, cnt_total, host(ep_len)
+
+    whole = run([T])
+    parts = run([100, 1, 77, 62])
+    for a, b in zip(whole, parts):
+        assert np.array_equal(a, b)
+    assert whole[2].sum() > 0 and (whole[1] / np.maximum(whole[2], 1)).max() <= limit
+
+
+def test_unknown_arithmetic_is_rejected(cp):
+    ret = torch.empty(8, device="cuda")
+    with pytest.raises(cp.CartpoleError):
+        cp.cp_rollout_ex(n_envs=8, T=1, arithmetic=2, ep_return_sum=ret)

@@ -70,6 +70,55 @@ def test_host_side_argument_errors(cp):
     assert L.cp_unfused_workspace_bytes(1024) >= 1024 * (33 * 4 + 7)
 
 
+def test_binding_structs_have_the_layout_the_header_declares(cp, tmp_path):
+    """Compile the header with the host C compiler, print sizeof/offsetof of every struct member,
+    and compare with the ctypes mirror in the binding."""
+    import subprocess
+    structs = {"cp_policy": cp.cp_policy, "cp_returns": cp.cp_returns, "cp_rollout_args": cp.cp_rollout_args}
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "cartpole.h"', 'int main(void) {']
+    for name, cls in structs.items():
+        lines.append(f'printf("{name} %zu\\n", sizeof({name}));')
+        for field, _ in cls._fields_:
+            lines.append(f'printf("{name}.{field} %zu\\n", offsetof({name}, {field}));')
+    lines += ['return 0; }']
+    src = tmp_path / "layout.c"
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-std=c99", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    got = dict(l.split() for l in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.splitlines())
+    for name, cls in structs.items():
+        assert int(got[name]) == C.sizeof(cls), name
+        for field, _ in cls._fields_:
+            assert int(got[f"{name}.{field}"]) == getattr(cls, field).offset, f"{name}.{field}"
+    # and every member the header declares is mirrored (count the members of each struct body)
+    text = re.sub(r"/\*.*?\*/", "", open(HEADER).read(), flags=re.S)
+    for name, cls in structs.items():
+        body = re.search(r"typedef struct %s \{(.*?)\} %s;" % (name, name), text, flags=re.S).group(1)
+        members = [m for decl in body.split(";") for m in decl.split(",") if m.strip()]
+        assert len(members) == len(cls._fields_), (name, members)
+
+
+def test_general_rollout_rejects_bad_arguments_on_the_host(cp):
+    L = cp.lib()
+    r = cp.cp_returns()
+    a = cp.cp_rollout_args()
+    a.n_envs, a.T, a.returns = 16, 10, C.pointer(r)
+    a.struct_size = C.sizeof(cp.cp_rollout_args) - 8
+    assert L.cp_rollout_ex(C.byref(a)) == cp.CP_EINVAL
+    assert b"struct_size" in L.cp_last_error()
+    a.struct_size = C.sizeof(cp.cp_rollout_args)
+    a.arithmetic = 2
+    assert L.cp_rollout_ex(C.byref(a)) == cp.CP_EINVAL
+    assert b"arithmetic" in L.cp_last_error()
+    a.arithmetic = cp.CP_ARITH_CONTRACTED
+    a.T = 0
+    assert L.cp_rollout_ex(C.byref(a)) == cp.CP_EINVAL
+    a.T = 10
+    a.returns = None
+    assert L.cp_rollout_ex(C.byref(a)) == cp.CP_EINVAL
+    assert L.cp_rollout_ex(None) == cp.CP_EINVAL
+
+
 def test_wrap_bookkeeping_needs_no_gpu(cp):
     L = cp.lib()
     fake = C.c_void_p(0x7000_0000_0100)  # never dereferenced on the host
