@@ -520,6 +520,9 @@ int cp_tune(const char *key, int value) {
     } else if (!strcmp(key, "rollout_ept")) {
         if (value != 0 && value != 1 && value != 2) return fail(CP_EINVAL, "rollout_ept must be 0, 1 or 2");
         cp::g_tuning.rollout_ept = value;
+    } else if (!strcmp(key, "rollout_coop")) {
+        if (value != 0 && value != 1 && value != 2) return fail(CP_EINVAL, "rollout_coop must be 0, 1 or 2");
+        cp::g_tuning.rollout_coop = value;
     } else if (!strcmp(key, "rollout_ctas_per_sm")) {
         if (value < 0 || value > 1024) return fail(CP_EINVAL, "rollout_ctas_per_sm must be 0..1024");
         cp::g_tuning.rollout_ctas_per_sm = value;

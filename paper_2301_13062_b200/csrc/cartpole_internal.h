@@ -49,7 +49,8 @@ struct RolloutParams {
 
 struct LaunchTuning {
     int rollout_block = 256;
-    int rollout_ept = 0;          // 0: chosen per policy
+    int rollout_ept = 0;          // 0: chosen per policy and batch size
+    int rollout_coop = 0;         // 0: chosen per batch size; 1 restarts by the warp; 2 per lane (ept 1)
     int rollout_ctas_per_sm = 0;  // 0: one task per warp (non-persistent grid)
     int step_block = 64;
     // Below this many envs the one-env-per-thread kernel is used: a small batch is latency-bound,

@@ -11,7 +11,9 @@
 // hands out CTAs as others retire; a persistent grid looping over tasks is
 // available for tuning.
 //
-// The kernel has no shared memory, no inter-warp synchronisation and no waits.
+// Warps never talk to each other and nothing waits on memory written by another warp; the
+// only synchronisation is __syncwarp() around a warp's own 192 bytes of shared memory in the
+// cooperative restart.
 //
 // This header holds the kernel template and its dispatch; rollout_kernel.cu instantiates it
 // for the canonical (one rounding per op) arithmetic, rollout_contracted.cu for the
@@ -48,14 +50,33 @@ __device__ __forceinline__ uint32_t policy_signbit(const RolloutParams &p, const
 #define CP_CONTRACT_MIN_CTAS 1
 #endif
 
+constexpr int kMaxWarpsPerCta = 8;  // __launch_bounds__(256)
+
+// SHAPE: how a warp holds and restarts its environments.
+//   0: one env per thread, each lane restarts its own env (shortest dependency chain per step:
+//      for batches too small to fill the chip, where a step's latency is what is paid);
+//   1: one env per thread, restarts done by the whole warp (see below);
+//   2: two envs per thread (two independent dependency chains), restarts by the whole warp.
 // STREAMS: 0 no per-step output; 1 exactly the reward plane and the done bitmask (no run-time
 // tests in the loop); 2 any combination, tested per step.
 // LIMIT: episodes are cut off after p.max_steps steps.
 // CONTRACT: the contracted arithmetic of euler_step_contracted instead of the canonical order.
-template <int POLICY, int EPT, int STREAMS, bool LIMIT, bool CONTRACT>
+template <int POLICY, int SHAPE, int STREAMS, bool LIMIT, bool CONTRACT>
 __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLLOUT_MIN_CTAS)
     rollout_kernel(const __grid_constant__ RolloutParams p) {
+    constexpr int EPT = SHAPE == 2 ? 2 : 1;
+    constexpr bool COOP = SHAPE != 0;
     const uint32_t lane = threadIdx.x & 31u;
+    // Per warp: key pairs of up to 8 finished envs, and their 8 x 4 start-state components.
+    __shared__ uint2 s_keys[COOP ? kMaxWarpsPerCta : 1][8];
+    __shared__ __align__(16) float s_out[COOP ? kMaxWarpsPerCta : 1][32];
+    uint2 *const keys_w = s_keys[COOP ? threadIdx.x >> 5 : 0];
+    float *const out_w = s_out[COOP ? threadIdx.x >> 5 : 0];
+    const uint32_t lane_lt = (1u << lane) - 1u;
+    if (COOP) {
+        if (lane < 8u) keys_w[lane] = make_uint2(0u, 0u);
+        __syncwarp();
+    }
     const int64_t warps_total = (int64_t)gridDim.x * (blockDim.x >> 5);
     const int64_t words = (p.n + 31) >> 5;
     unsigned long long tot_ret = 0, tot_cnt = 0;
@@ -111,6 +132,7 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
         const uint32_t *act_ptr[EPT];
         int64_t env_off[EPT], word_off[EPT];  // into [T][n] planes and [T][words] bit planes
         bool word_ok[EPT];
+        uint32_t vmask[EPT];  // lanes of slot j that own a real environment
 #pragma unroll
         for (int j = 0; j < EPT; ++j) {
             env_off[j] = idx[j];
@@ -120,33 +142,108 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
             rew_ptr[j] = STREAMS == 1 ? p.reward_stream + idx[j] : nullptr;
             done_ptr[j] = STREAMS == 1 ? p.done_bits + (word_ok[j] ? word_off[j] : 0) : nullptr;
             act_ptr[j] = POLICY == 3 ? p.action_bits_in + (in_range ? word_off[j] : 0) : nullptr;
+            vmask[j] = __ballot_sync(0xffffffffu, valid[j]);
         }
         const bool want_done = STREAMS == 2 && p.done_bits, want_act = STREAMS == 2 && p.action_bits;
         const bool want_rew = STREAMS == 2 && p.reward_stream, want_traj = STREAMS == 2 && p.trajectory;
 
+        uint32_t act_word[EPT] = {};
+        if (POLICY == 3) {
+#pragma unroll
+            for (int j = 0; j < EPT; ++j) act_word[j] = __ldg(act_ptr[j]);
+        }
         const uint32_t t_end = p.t0 + p.T;
         for (uint32_t t = p.t0; t != t_end; ++t) {
+            const uint32_t t1 = t + 1u;
+            bool done[EPT];
+            uint32_t sb[EPT];
 #pragma unroll
             for (int j = 0; j < EPT; ++j) {
-                uint32_t sb;
                 if (POLICY == 3) {
-                    sb = (__ldg(act_ptr[j]) << (31u - lane)) & 0x80000000u;  // one word per warp, broadcast
+                    // One word per warp, broadcast; the next step's word is requested now, a whole
+                    // step ahead of its use (the warp barriers of the restart keep the compiler
+                    // from hoisting the load by itself).
+                    sb[j] = (act_word[j] << (31u - lane)) & 0x80000000u;
                     act_ptr[j] += words;
+                    if (t1 != t_end) act_word[j] = __ldg(act_ptr[j]);
                 } else if (POLICY == 6) {
-                    sb = linear_action(own[POLICY == 6 ? j : 0], z[j]);
+                    sb[j] = linear_action(own[POLICY == 6 ? j : 0], z[j]);
                 } else {
-                    sb = policy_signbit<POLICY>(p, ka[j], t, z[j]);
+                    sb[j] = policy_signbit<POLICY>(p, ka[j], t, z[j]);
                 }
-                bool done = CONTRACT ? euler_step_contracted(z[j], force_from_signbit(sb))
-                                     : euler_step(z[j], force_from_signbit(sb));
-                if (LIMIT) done |= (t + 1u - begin[j]) >= p.max_steps;
-                if (done) {
+                done[j] = CONTRACT ? euler_step_contracted(z[j], force_from_signbit(sb[j]))
+                                   : euler_step(z[j], force_from_signbit(sb[j]));
+                if (LIMIT) done[j] |= (t1 - begin[j]) >= p.max_steps;
+                if (!COOP && done[j]) {
                     cnt[j] += 1u;
-                    begin[j] = t + 1u;
-                    z[j] = start_state(kr[j], t + 1u);
+                    begin[j] = t1;
+                    z[j] = start_state(kr[j], t1);
                 }
+            }
+
+            // Restart by the whole warp. A start state is four independent hashes of the env's key
+            // pair, and with the random policy 1.4 of a warp's 32 envs finish per step: restarting
+            // lane by lane issues all four hashes (45 instructions) for the whole warp on 77 % of
+            // the steps of each j — a third of all issue slots. Instead the finished lanes post
+            // their key pairs to a per-warp list in shared memory (slot j owns entries
+            // [j*CAP, (j+1)*CAP), position = rank among the finished lanes of that slot), lane L
+            // computes component L%4 of entry L/4 — eight restarts in one pass, one hash per lane —
+            // and each finished lane reads its four components back. Same hash, same bits; about
+            // 51 instead of 2 x 35 warp instructions per warp-step (measured: 105 -> 94 issue
+            // slots per env-step, 1.61 -> 1.45 ms on 1,048,576 x 500).
+            uint32_t dmask[EPT] = {};
+            if (COOP) {
+                uint32_t any = 0u;
+#pragma unroll
+                for (int j = 0; j < EPT; ++j) {
+                    dmask[j] = __ballot_sync(0xffffffffu, done[j]);
+                    any |= dmask[j];
+                }
+                if (any) {  // warp-uniform
+                    constexpr uint32_t CAP = 8u / EPT;
+                    uint32_t slot[EPT];
+                    bool listed[EPT];
+#pragma unroll
+                    for (int j = 0; j < EPT; ++j) {
+                        const uint32_t r = __popc(dmask[j] & lane_lt);
+                        slot[j] = j * CAP + r;
+                        listed[j] = done[j] && r < CAP;
+                        if (done[j]) {
+                            cnt[j] += 1u;
+                            begin[j] = t1;
+                        }
+                        if (listed[j]) keys_w[slot[j]] = make_uint2(kr[j].k0, kr[j].k1);
+                    }
+                    __syncwarp();
+                    const uint2 kq = keys_w[lane >> 2];  // unused entries hold stale keys: harmless
+                    Keys k;
+                    k.k0 = kq.x;
+                    k.k1 = kq.y;
+                    const uint32_t h0 = k.k0 ^ (4u * t1);
+                    const uint32_t mm = h0 ^ (h0 >> 16);
+                    out_w[lane] = start_from_bits(step_hash_tail(k, mm ^ (lane & 3u)) >> 8);
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < EPT; ++j) {
+                        if (listed[j]) {
+                            const float4 s = reinterpret_cast<const float4 *>(out_w)[slot[j]];
+                            z[j].x = s.x;
+                            z[j].xd = s.y;
+                            z[j].th = s.z;
+                            z[j].thd = s.w;
+                        } else if (done[j]) {  // more than CAP envs of this slot finished at once: rare
+                            z[j] = start_state(kr[j], t1);
+                        }
+                    }
+                    // No third barrier: the next write to keys_w follows this step's reads of it by
+                    // the second barrier, and the next write to out_w follows the next first barrier.
+                }
+            }
+
+#pragma unroll
+            for (int j = 0; j < EPT; ++j) {
                 if (STREAMS == 1) {
-                    const uint32_t m = __ballot_sync(0xffffffffu, done && valid[j]);
+                    const uint32_t m = COOP ? (dmask[j] & vmask[j]) : __ballot_sync(0xffffffffu, done[j] && valid[j]);
                     if (word_ok[j]) *done_ptr[j] = m;
                     if (valid[j]) *rew_ptr[j] = 1.0f;
                     done_ptr[j] += words;
@@ -154,11 +251,12 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
                 }
                 if (STREAMS == 2) {
                     if (want_done) {
-                        const uint32_t m = __ballot_sync(0xffffffffu, done && valid[j]);
+                        const uint32_t m =
+                            COOP ? (dmask[j] & vmask[j]) : __ballot_sync(0xffffffffu, done[j] && valid[j]);
                         if (word_ok[j]) p.done_bits[word_off[j]] = m;
                     }
                     if (want_act) {
-                        const uint32_t m = __ballot_sync(0xffffffffu, (sb != 0u) && valid[j]);
+                        const uint32_t m = __ballot_sync(0xffffffffu, (sb[j] != 0u) && valid[j]);
                         if (word_ok[j]) p.action_bits[word_off[j]] = m;
                     }
                     if (valid[j]) {
@@ -214,9 +312,11 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
 
 namespace {
 
-template <int POLICY, int EPT, int STREAMS, bool LIMIT, bool CONTRACT>
+template <int POLICY, int SHAPE, int STREAMS, bool LIMIT, bool CONTRACT>
 cudaError_t launch_one(RolloutParams &p, cudaStream_t s) {
-    const int block = g_tuning.rollout_block;
+    constexpr int EPT = SHAPE == 2 ? 2 : 1;
+    int block = g_tuning.rollout_block;
+    if (block > 32 * kMaxWarpsPerCta) block = 32 * kMaxWarpsPerCta;
     p.n_tasks = (p.n + 32 * EPT - 1) / (32 * EPT);
     // Default: one task per warp, CTAs handed out by the hardware scheduler as others retire.
     // All tasks take the same time, so a persistent grid would run ceil(tasks / resident warps)
@@ -231,55 +331,63 @@ cudaError_t launch_one(RolloutParams &p, cudaStream_t s) {
         if (grid > resident) grid = resident;
     }
     if (grid > 0x7fffffffLL) grid = 0x7fffffffLL;
-    rollout_kernel<POLICY, EPT, STREAMS, LIMIT, CONTRACT><<<(unsigned)grid, block, 0, s>>>(p);
+    rollout_kernel<POLICY, SHAPE, STREAMS, LIMIT, CONTRACT><<<(unsigned)grid, block, 0, s>>>(p);
     count_launch();
     return cudaGetLastError();
 }
 
 template <int POLICY, int STREAMS, bool LIMIT, bool CONTRACT>
-cudaError_t launch_ept(RolloutParams &p, int ept, cudaStream_t s) {
-    return ept == 1 ? launch_one<POLICY, 1, STREAMS, LIMIT, CONTRACT>(p, s)
-                    : launch_one<POLICY, 2, STREAMS, LIMIT, CONTRACT>(p, s);
+cudaError_t launch_shape(RolloutParams &p, int shape, cudaStream_t s) {
+    switch (shape) {
+        case 0: return launch_one<POLICY, 0, STREAMS, LIMIT, CONTRACT>(p, s);
+        case 1: return launch_one<POLICY, 1, STREAMS, LIMIT, CONTRACT>(p, s);
+        default: return launch_one<POLICY, 2, STREAMS, LIMIT, CONTRACT>(p, s);
+    }
 }
 
 template <int POLICY, int STREAMS, bool CONTRACT>
-cudaError_t launch_limit(RolloutParams &p, int ept, cudaStream_t s) {
-    return p.max_steps ? launch_ept<POLICY, STREAMS, true, CONTRACT>(p, ept, s)
-                       : launch_ept<POLICY, STREAMS, false, CONTRACT>(p, ept, s);
+cudaError_t launch_limit(RolloutParams &p, int shape, cudaStream_t s) {
+    return p.max_steps ? launch_shape<POLICY, STREAMS, true, CONTRACT>(p, shape, s)
+                       : launch_shape<POLICY, STREAMS, false, CONTRACT>(p, shape, s);
 }
 
 template <int POLICY, bool CONTRACT>
-cudaError_t launch_mode(RolloutParams &p, int mode, int ept, cudaStream_t s) {
+cudaError_t launch_mode(RolloutParams &p, int mode, int shape, cudaStream_t s) {
     switch (mode) {
-        case 0: return launch_limit<POLICY, 0, CONTRACT>(p, ept, s);
-        case 1: return launch_limit<POLICY, 1, CONTRACT>(p, ept, s);
-        default: return launch_limit<POLICY, 2, CONTRACT>(p, ept, s);
+        case 0: return launch_limit<POLICY, 0, CONTRACT>(p, shape, s);
+        case 1: return launch_limit<POLICY, 1, CONTRACT>(p, shape, s);
+        default: return launch_limit<POLICY, 2, CONTRACT>(p, shape, s);
     }
 }
 
 template <bool CONTRACT>
 cudaError_t launch_rollout_arith(RolloutParams &p, int policy, bool streams, cudaStream_t s) {
-    int ept = g_tuning.rollout_ept;
-    if (ept == 0) {
-        // Two envs per thread (two independent dependency chains) unless the batch is so small
-        // that spreading it over twice as many warps matters more. The MLP policies carry enough
-        // independent work per env (H hidden units) to fill the pipes with one env per thread,
-        // and a second one only costs registers: measured 1.5 % (canonical) and 20 % (contracted,
-        // where the compiler interleaves the two networks at 180+ registers) slower with two.
-        const bool mlp = policy == 2 || policy == 4 || policy == 5;
-        ept = (mlp && !p.action_bits_in) || (p.n + 63) / 64 < (int64_t)sm_count() * 16 ? 1 : 2;
-    }
+    if (p.action_bits_in) policy = 3;
+    // A batch too small to give every SM sixteen two-env warps is latency-bound: one env per
+    // thread over twice as many warps, and per-lane restarts (the cooperative restart adds two
+    // shared-memory round trips to every step's dependency chain: 2,048 envs x 10,000 steps
+    // take 1.85 ms with per-lane restarts, 2.14 ms with cooperative ones). Otherwise the kernel
+    // is issue-bound and the cooperative restart's fewer instructions win. The MLP policies
+    // carry enough independent work per env (H hidden units) to fill the pipes with one env
+    // per thread, and a second one only costs registers: measured 1.5 % (canonical) and 20 %
+    // (contracted, where the compiler interleaves the two networks at 180+ registers) slower.
+    const bool small = (p.n + 63) / 64 < (int64_t)sm_count() * 16;
+    const bool mlp = policy == 2 || policy == 4 || policy == 5;
+    int ept = g_tuning.rollout_ept;      // 0 auto, 1, 2
+    int coop = g_tuning.rollout_coop;    // 0 auto, 1 cooperative, 2 per lane
+    if (ept == 0) ept = (small || mlp || coop == 2) ? 1 : 2;
+    if (coop == 0) coop = (small && ept == 1) ? 2 : 1;
+    const int shape = ept == 2 ? 2 : (coop == 2 ? 0 : 1);  // two envs per thread are always cooperative
     // 0: no per-step output; 1: reward plane + done bitmask only; 2: any other combination
     const int mode = !streams ? 0 : (p.reward_stream && p.done_bits && !p.action_bits && !p.trajectory) ? 1 : 2;
-    if (p.action_bits_in) policy = 3;
     switch (policy) {
-        case 0: return launch_mode<0, CONTRACT>(p, mode, ept, s);
-        case 1: return launch_mode<1, CONTRACT>(p, mode, ept, s);
-        case 2: return launch_mode<2, CONTRACT>(p, mode, ept, s);
-        case 3: return launch_mode<3, CONTRACT>(p, mode, ept, s);
-        case 4: return launch_mode<4, CONTRACT>(p, mode, ept, s);
-        case 5: return launch_mode<5, CONTRACT>(p, mode, ept, s);
-        default: return launch_mode<6, CONTRACT>(p, mode, ept, s);
+        case 0: return launch_mode<0, CONTRACT>(p, mode, shape, s);
+        case 1: return launch_mode<1, CONTRACT>(p, mode, shape, s);
+        case 2: return launch_mode<2, CONTRACT>(p, mode, shape, s);
+        case 3: return launch_mode<3, CONTRACT>(p, mode, shape, s);
+        case 4: return launch_mode<4, CONTRACT>(p, mode, shape, s);
+        case 5: return launch_mode<5, CONTRACT>(p, mode, shape, s);
+        default: return launch_mode<6, CONTRACT>(p, mode, shape, s);
     }
 }
 

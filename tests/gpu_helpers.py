@@ -11,6 +11,8 @@ Tolerances (stated by the benchmark spec, written out here):
     mean return within 0.1 %; envs whose policy logits come within 1e-5 of a tie
     are excused like threshold-band envs.
 """
+import contextlib
+
 import numpy as np
 
 XT = np.float32(2.4)
@@ -18,6 +20,24 @@ TT = np.float32(12 * 2 * np.pi / 360)
 TAU = np.float32(0.02)
 BAND = 1e-5
 REL_TOL = 2e-6
+
+
+# The rollout kernel's three work shapes as (rollout_ept, rollout_coop) tuning values: one env
+# per thread with per-lane restarts, one env per thread with restarts by the whole warp, two
+# envs per thread (always by the warp). The library picks one by batch size and policy; tests
+# force each of them on small batches.
+SHAPES = [(1, 2), (1, 1), (2, 1)]
+
+
+@contextlib.contextmanager
+def rollout_shape(cp, ept: int, coop: int):
+    cp.cp_tune("rollout_ept", ept)
+    cp.cp_tune("rollout_coop", coop)
+    try:
+        yield
+    finally:
+        cp.cp_tune("rollout_ept", 0)
+        cp.cp_tune("rollout_coop", 0)
 
 
 def band_mask(pre_reset: np.ndarray) -> np.ndarray:

@@ -33,7 +33,7 @@ def host(t):
     return t.cpu().numpy()
 
 
-def contracted_step(cp, z, seed, t, env_offset, general_streams, ept):
+def contracted_step(cp, z, seed, t, env_offset, general_streams, shape):
     """One step of the contracted rollout kernel from the given states."""
     n = z.shape[1]
     planes = torch.zeros(4, (n + 3) // 4 * 4, dtype=torch.float32, device="cuda")
@@ -44,11 +44,8 @@ def contracted_step(cp, z, seed, t, env_offset, general_streams, ept):
            "done_bits": torch.zeros(1, words, dtype=torch.int32, device="cuda")}
     if general_streams:
         out["action_bits"] = torch.zeros(1, words, dtype=torch.int32, device="cuda")
-    cp.cp_tune("rollout_ept", ept)
-    try:
+    with H.rollout_shape(cp, *shape):
         cp.cp_rollout_ex(state=st, T=1, arithmetic=cp.CP_ARITH_CONTRACTED, **out)
-    finally:
-        cp.cp_tune("rollout_ept", 0)
     torch.cuda.synchronize()
     assert st.info()["t"] == t + 1
     act = H.unpack_bits(host(out["action_bits"]), n)[0] if general_streams else None
@@ -60,9 +57,9 @@ def contracted_step(cp, z, seed, t, env_offset, general_streams, ept):
 def test_one_contracted_step_within_tolerance_of_the_oracle(cp, oracle, spread, n):
     z = inputs.random_states(n, seed=3 * n + len(spread), spread=spread)
     worst = 0.0
-    for (off, t, general, ept) in ((0, 0, False, 2), (4321, 17, True, 1)):
+    for (off, t, general, shape) in ((0, 0, False, H.SHAPES[2]), (4321, 17, True, H.SHAPES[0]), (7, 3, False, H.SHAPES[1])):
         want = oracle.step(z, seed=1, t=t, env_offset=off, want_pre_reset=True)
-        state, reward, done, act = contracted_step(cp, z, 1, t, off, general, ept)
+        state, reward, done, act = contracted_step(cp, z, 1, t, off, general, shape)
         stats = H.assert_step_matches(want, z, state, reward, done, act)
         worst = max(worst, 1.0 - stats["bit_exact_fraction"])
     if spread == "live" and n >= 1025:

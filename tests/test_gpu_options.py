@@ -156,14 +156,11 @@ def test_supplied_action_stream(cp, oracle):
     bits = pack_bits(acts)
     bits[:, -1] |= np.uint32((0xFFFFFFFF << (n % 32)) & 0xFFFFFFFF)  # garbage in the padding bits
     d_bits = torch.from_numpy(bits.view(np.int32)).cuda()
-    for ept in (1, 2):
-        cp.cp_tune("rollout_ept", ept)
-        try:
+    for shape in H.SHAPES:
+        with H.rollout_shape(cp, *shape):
             out = outputs(n, T)
             cp.cp_rollout_ex(n_envs=n, T=T, seed=seed, env_offset=off, action_bits_in=d_bits, **out)
             r = fetch(out)
-        finally:
-            cp.cp_tune("rollout_ept", 0)
         o = oracle.rollout(n, T, seed, env_offset=off, action_bits_in=pack_bits(acts), done_bits=True, nthreads=4)
         H.assert_returns_match(r["ep_return_sum"], r["ep_count"], o["ep_return_sum"], o["ep_count"])
         assert np.array_equal(H.unpack_bits(r["action_bits"], n), acts)  # echoed, padding masked off
@@ -255,16 +252,13 @@ def test_per_env_linear_policies_against_oracle(cp, oracle):
     wp = inputs.per_env_linear_weights(n, 11)
     d_w = torch.from_numpy(wp).cuda()
     res = []
-    for ept in (1, 2):
-        cp.cp_tune("rollout_ept", ept)
-        try:
+    for shape in H.SHAPES:
+        with H.rollout_shape(cp, *shape):
             out = outputs(n, T)
             cp.cp_rollout_shard(off, n, T, seed, cp.policy(cp.CP_POLICY_LINEAR_PER_ENV, d_w), **out)
             res.append(fetch(out))
-        finally:
-            cp.cp_tune("rollout_ept", 0)
     for k in res[0]:
-        assert np.array_equal(res[0][k], res[1][k]), k
+        assert np.array_equal(res[0][k], res[1][k]) and np.array_equal(res[0][k], res[2][k]), k
     r = res[0]
     o = oracle.rollout(n, T, seed, inputs.POLICY_LINEAR_PER_ENV, wp, env_offset=off, done_bits=True,
                        action_bits=True, min_gap=True, nthreads=8)

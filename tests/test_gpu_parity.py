@@ -251,14 +251,11 @@ def run_rollout(cp, n, T, seed, kind=0, weights=None, env_offset=0, streams=Fals
 
 
 @pytest.mark.parametrize("n,T", [(1, 64), (33, 64), (1025, 100), (5000, 37)])
-@pytest.mark.parametrize("ept", [1, 2])
-def test_rollout_equals_repeated_fused_steps_bitwise(cp, n, T, ept):
-    cp.cp_tune("rollout_ept", ept)
-    try:
-        seed, off = 2, 77
+@pytest.mark.parametrize("shape", H.SHAPES)
+def test_rollout_equals_repeated_fused_steps_bitwise(cp, n, T, shape):
+    seed, off = 2, 77
+    with H.rollout_shape(cp, *shape):
         r = run_rollout(cp, n, T, seed, env_offset=off, streams=True, traj=True)
-    finally:
-        cp.cp_tune("rollout_ept", 0)
     planes = alloc_planes(n)
     st = cp.cp_wrap(planes, n, seed, 0, off)
     cp.cp_fill_start(st)
@@ -444,11 +441,10 @@ def test_config2_step_path_at_full_size(cp, oracle):
     assert sa.info()["t"] == 20 == sc.info()["t"]
 
 
-@pytest.mark.parametrize("ept", [1, 2])
-def test_reward_and_done_only_streams_equal_the_general_stream_kernel(cp, ept):
+@pytest.mark.parametrize("shape", H.SHAPES)
+def test_reward_and_done_only_streams_equal_the_general_stream_kernel(cp, shape):
     """The reward-plane + done-bitmask combination has a kernel of its own."""
-    cp.cp_tune("rollout_ept", ept)
-    try:
+    with H.rollout_shape(cp, *shape):
         for n, T, kind in ((5001, 60, 0), (40000, 40, 1), (33, 20, 2)):
             w = inputs.policy_weights(kind, 3) if kind else None
             a = run_rollout(cp, n, T, 2, kind, w, env_offset=9, streams=True)
@@ -457,8 +453,35 @@ def test_reward_and_done_only_streams_equal_the_general_stream_kernel(cp, ept):
                 assert np.array_equal(a[k], b[k]), (k, n, kind)
             assert np.all(b["reward_stream"] == 1.0)
             assert np.array_equal(H.unpack_bits(b["done_bits"], n).sum(axis=0), b["ep_count"])
-    finally:
-        cp.cp_tune("rollout_ept", 0)
+
+
+def test_work_shapes_agree_bitwise_and_survive_mass_termination(cp):
+    """The three work shapes (per-lane restarts, restarts by the warp with one or two envs per
+    thread) give the same bits, including when far more environments of a warp finish in one
+    step than the warp's restart list holds: with an episode limit of 1 every env restarts every
+    step, with 3 all of them at once every third step."""
+    n, T = 5003, 31
+    for kind, limit in ((0, 0), (0, 1), (0, 3), (1, 2), (2, 0)):
+        w = inputs.policy_weights(kind, 3) if kind else None
+        pol = cp.policy(kind, w) if kind else None
+        results = []
+        for shape in H.SHAPES:
+            out = {"ep_return_sum": torch.zeros(n, device="cuda"),
+                   "ep_count": torch.zeros(n, dtype=torch.int32, device="cuda"),
+                   "totals": torch.zeros(2, dtype=torch.int64, device="cuda"),
+                   "final_state": torch.zeros(4, n, device="cuda"),
+                   "done_bits": torch.zeros(T, (n + 31) // 32, dtype=torch.int32, device="cuda"),
+                   "trajectory": torch.zeros(T, 4, n, device="cuda")}
+            with H.rollout_shape(cp, *shape):
+                cp.cp_rollout_ex(n_envs=n, T=T, seed=6, env_offset=11, policy=pol, max_episode_steps=limit, **out)
+            torch.cuda.synchronize()
+            results.append({k: host(v) for k, v in out.items()})
+        for other in results[1:]:
+            for k in results[0]:
+                assert np.array_equal(results[0][k].view(np.uint32) if results[0][k].dtype == np.float32 else results[0][k],
+                                      other[k].view(np.uint32) if other[k].dtype == np.float32 else other[k]), (k, kind, limit)
+        if limit == 1:
+            assert np.all(results[0]["ep_count"] == T) and np.all(results[0]["ep_return_sum"] == T)
 
 
 def test_shards_compose(cp):
