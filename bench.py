@@ -31,15 +31,18 @@ METRIC = "env_steps_per_sec"
 UNIT = "env-steps/s"
 SMS = 148
 # Work per env-step of each rollout variant, counted by ncu on 1,048,576 envs x 100 steps
-# (summaries under profiles/): "thread" = smsp__thread_inst_executed.sum / (N*T), the
-# instructions environments actually execute (the algorithmic figure: an env that does not
-# terminate executes no restart code); "slot" = 32 * smsp__inst_executed.sum / (N*T), the issue
-# slots the warps occupy, which also counts lanes idling while a neighbour restarts.
+# (summaries under profiles/). "thread" = smsp__thread_inst_executed.sum / (N*T) of the
+# per-lane formulation (one env per thread, each lane restarts its own env; tuning
+# rollout_ept=1 rollout_coop=2): the instructions an environment needs, none counted for
+# lanes that idle or help a neighbour — the algorithmic figure. "slot" = 32 *
+# smsp__inst_executed.sum / (N*T) of the kernel the library launches by default at this size
+# (restarts by the whole warp): the issue slots it really occupies.
 ROLLOUT_OPS = {
-    "random": {"thread": 71.5, "slot": 104.9},
-    "linear": {"thread": 75.5, "slot": 85.0},
-    "linear+streams": {"thread": 90.2, "slot": 99.8},
-    "mlp": {"thread": 442.2, "slot": 473.7},
+    "random": {"thread": 72.6, "slot": 92.8},
+    "linear": {"thread": 76.8, "slot": 83.5},
+    "linear+streams": {"thread": 94.9, "slot": 98.6},
+    "mlp": {"thread": 441.3, "slot": 470.2},
+    "random+contracted": {"thread": 55.6, "slot": 74.4},
 }
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch in the same captures.
 ROLLOUT_DRAM_BYTES = {"random": 20.7e3, "linear": 20.5e3, "linear+streams": 381.2e6, "mlp": 32.5e3}

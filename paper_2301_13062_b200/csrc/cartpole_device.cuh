@@ -71,6 +71,27 @@ __device__ __forceinline__ uint32_t action_signbit(Keys k, uint32_t t) {
     return h & 0x80000000u;
 }
 
+// Keys for loops over time. A right shift distributes over xor, so the first xorshift of
+// step_hash splits into a part that depends only on the key and one that depends only on the
+// counter:  (k0 ^ c) ^ ((k0 ^ c) >> 16) == fold16(k0) ^ fold16(c).  A kernel that hashes many
+// counters with one key keeps fold16(k0), and computes fold16(c) once per step for all its envs.
+__device__ __forceinline__ uint32_t fold16(uint32_t v) { return v ^ (v >> 16); }
+struct FoldedKeys {
+    uint32_t f0, k1;  // fold16(k0), k1
+};
+__device__ __forceinline__ FoldedKeys fold_keys(Keys k) {
+    FoldedKeys f;
+    f.f0 = fold16(k.k0);
+    f.k1 = k.k1;
+    return f;
+}
+// action_signbit(k, t) with folded_t = fold16(t)
+__device__ __forceinline__ uint32_t action_signbit_folded(FoldedKeys k, uint32_t folded_t) {
+    uint32_t h = (k.f0 ^ folded_t) * kMA + k.k1;
+    h = (h ^ (h >> 15)) * kMB;
+    return h & 0x80000000u;
+}
+
 // force = a ? +F : -F, from the action's sign-bit form (0x80000000 = push right).
 __device__ __forceinline__ float force_from_signbit(uint32_t sb) {
     return __uint_as_float(sb ^ 0xC1200000u);  // -10.0f with the sign flipped when a = 1
@@ -117,6 +138,23 @@ __device__ __forceinline__ State start_state(Keys kr, uint32_t t) {
     z.xd = start_from_bits(step_hash_tail(kr, m ^ 1u) >> 8);
     z.th = start_from_bits(step_hash_tail(kr, m ^ 2u) >> 8);
     z.thd = start_from_bits(step_hash_tail(kr, m ^ 3u) >> 8);
+    return z;
+}
+
+// The same from folded keys; folded_4t = fold16(4 * t). The counters 4t + j (j < 4) fold to
+// fold16(4t) ^ j because 4t has its two low bits clear and j >> 16 == 0.
+__device__ __forceinline__ float start_component_folded(FoldedKeys kr, uint32_t folded_4t, uint32_t j) {
+    Keys k;
+    k.k0 = 0u;  // not used by the tail
+    k.k1 = kr.k1;
+    return start_from_bits(step_hash_tail(k, kr.f0 ^ folded_4t ^ j) >> 8);
+}
+__device__ __forceinline__ State start_state_folded(FoldedKeys kr, uint32_t folded_4t) {
+    State z;
+    z.x = start_component_folded(kr, folded_4t, 0u);
+    z.xd = start_component_folded(kr, folded_4t, 1u);
+    z.th = start_component_folded(kr, folded_4t, 2u);
+    z.thd = start_component_folded(kr, folded_4t, 3u);
     return z;
 }
 

@@ -28,10 +28,10 @@ namespace cp {
 // the caller, 4 / 5 MLP with 32 / 64 hidden units, 6 one linear policy per environment (its ten
 // parameters are loaded into registers before the time loop; handled in the kernel body).
 template <int POLICY>
-__device__ __forceinline__ uint32_t policy_signbit(const RolloutParams &p, const Keys &ka, uint32_t t,
-                                                   const State &z) {
+__device__ __forceinline__ uint32_t policy_signbit(const RolloutParams &p, const FoldedKeys &ka,
+                                                   uint32_t folded_t, const State &z) {
     if (POLICY == 0) {
-        return action_signbit(ka, t);
+        return action_signbit_folded(ka, folded_t);
     } else if (POLICY == 1) {
         return linear_action(*reinterpret_cast<const LinearW *>(p.w), z);
     } else if (POLICY == 2) {
@@ -85,7 +85,7 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
          task += warps_total) {
         const int64_t base = task * (32 * EPT);
         State z[EPT];
-        Keys ka[EPT], kr[EPT];
+        FoldedKeys ka[EPT], kr[EPT];  // action and restart streams (see fold16)
         LinearW own[POLICY == 6 ? EPT : 1];  // per-environment policies live in registers
         // Episode bookkeeping: every step earns reward 1, so the returns of the episodes completed
         // in this launch add up to (time of the last termination) - (time the first of them began),
@@ -101,15 +101,15 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
             valid[j] = idx[j] < p.n;
             if (!valid[j]) idx[j] = p.n - 1;  // idle lanes shadow the last environment and store nothing
             const uint32_t env = p.env_offset + (uint32_t)idx[j];
-            if (POLICY == 0) ka[j] = make_keys(p.salt_a, env);
-            kr[j] = make_keys(p.salt_r, env);
+            if (POLICY == 0) ka[j] = fold_keys(make_keys(p.salt_a, env));
+            kr[j] = fold_keys(make_keys(p.salt_r, env));
             if (p.init_planes) {
                 z[j].x = p.init_planes[idx[j]];
                 z[j].xd = p.init_planes[p.init_stride + idx[j]];
                 z[j].th = p.init_planes[2 * p.init_stride + idx[j]];
                 z[j].thd = p.init_planes[3 * p.init_stride + idx[j]];
             } else {
-                z[j] = start_state(kr[j], p.t0);
+                z[j] = start_state_folded(kr[j], fold16(4u * p.t0));
             }
             if (POLICY == 6) {  // parameter q of env i at env_weights[q*n + i]: coalesced per plane
                 LinearW &o = own[POLICY == 6 ? j : 0];
@@ -155,6 +155,7 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
         const uint32_t t_end = p.t0 + p.T;
         for (uint32_t t = p.t0; t != t_end; ++t) {
             const uint32_t t1 = t + 1u;
+            const uint32_t folded_t = fold16(t), folded_4t1 = fold16(4u * t1);  // warp-uniform
             bool done[EPT];
             uint32_t sb[EPT];
 #pragma unroll
@@ -169,7 +170,7 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
                 } else if (POLICY == 6) {
                     sb[j] = linear_action(own[POLICY == 6 ? j : 0], z[j]);
                 } else {
-                    sb[j] = policy_signbit<POLICY>(p, ka[j], t, z[j]);
+                    sb[j] = policy_signbit<POLICY>(p, ka[j], folded_t, z[j]);
                 }
                 done[j] = CONTRACT ? euler_step_contracted(z[j], force_from_signbit(sb[j]))
                                    : euler_step(z[j], force_from_signbit(sb[j]));
@@ -177,7 +178,7 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
                 if (!COOP && done[j]) {
                     cnt[j] += 1u;
                     begin[j] = t1;
-                    z[j] = start_state(kr[j], t1);
+                    z[j] = start_state_folded(kr[j], folded_4t1);
                 }
             }
 
@@ -212,16 +213,14 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
                             cnt[j] += 1u;
                             begin[j] = t1;
                         }
-                        if (listed[j]) keys_w[slot[j]] = make_uint2(kr[j].k0, kr[j].k1);
+                        if (listed[j]) keys_w[slot[j]] = make_uint2(kr[j].f0, kr[j].k1);
                     }
                     __syncwarp();
                     const uint2 kq = keys_w[lane >> 2];  // unused entries hold stale keys: harmless
-                    Keys k;
-                    k.k0 = kq.x;
+                    FoldedKeys k;
+                    k.f0 = kq.x;
                     k.k1 = kq.y;
-                    const uint32_t h0 = k.k0 ^ (4u * t1);
-                    const uint32_t mm = h0 ^ (h0 >> 16);
-                    out_w[lane] = start_from_bits(step_hash_tail(k, mm ^ (lane & 3u)) >> 8);
+                    out_w[lane] = start_component_folded(k, folded_4t1, lane & 3u);
                     __syncwarp();
 #pragma unroll
                     for (int j = 0; j < EPT; ++j) {
@@ -232,7 +231,7 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
                             z[j].th = s.z;
                             z[j].thd = s.w;
                         } else if (done[j]) {  // more than CAP envs of this slot finished at once: rare
-                            z[j] = start_state(kr[j], t1);
+                            z[j] = start_state_folded(kr[j], folded_4t1);
                         }
                     }
                     // No third barrier: the next write to keys_w follows this step's reads of it by
@@ -371,11 +370,13 @@ cudaError_t launch_rollout_arith(RolloutParams &p, int policy, bool streams, cud
     // carry enough independent work per env (H hidden units) to fill the pipes with one env
     // per thread, and a second one only costs registers: measured 1.5 % (canonical) and 20 %
     // (contracted, where the compiler interleaves the two networks at 180+ registers) slower.
+    // Per-environment linear policies keep ten weights per env in registers: 89 registers with
+    // two envs per thread, 63 with one, which is 8 % faster.
     const bool small = (p.n + 63) / 64 < (int64_t)sm_count() * 16;
-    const bool mlp = policy == 2 || policy == 4 || policy == 5;
+    const bool heavy = policy == 2 || policy == 4 || policy == 5 || policy == 6;
     int ept = g_tuning.rollout_ept;      // 0 auto, 1, 2
     int coop = g_tuning.rollout_coop;    // 0 auto, 1 cooperative, 2 per lane
-    if (ept == 0) ept = (small || mlp || coop == 2) ? 1 : 2;
+    if (ept == 0) ept = (small || heavy || coop == 2) ? 1 : 2;
     if (coop == 0) coop = (small && ept == 1) ? 2 : 1;
     const int shape = ept == 2 ? 2 : (coop == 2 ? 0 : 1);  // two envs per thread are always cooperative
     // 0: no per-step output; 1: reward plane + done bitmask only; 2: any other combination
