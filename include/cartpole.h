@@ -43,7 +43,7 @@
  *   xacc  = temp - ((pml*thacc)*c)/m_total
  *   x' = x + tau*xd; xd' = xd + tau*xacc; th' = th + tau*thd; thd' = thd + tau*thacc
  *   every operation rounded once to float32 (no fused multiply-add, IEEE division; no
- *   fast-math). sinf/cosf: for |theta| <= 0.25 (every angle an episode can hold; the
+ *   fast-math). sinf/cosf: for |theta| <= 0.22 (every angle an episode can hold; the
  *   termination threshold is 0.2095) a polynomial with measured error <= 0.53 ulp, for any
  *   other argument the CUDA library's accurate sinf/cosf;
  *   done = x'<-x_max | x'>x_max | th'<-theta_max | th'>theta_max  (strict, on the
@@ -317,7 +317,7 @@ int cp_selftest_sincos_accuracy(uint32_t lo_bits, uint32_t hi_bits, uint64_t *ou
  * they are used. out DEVICE [4] uint64, caller zeroes; every count must come back 0. */
 int cp_selftest_arith(uint64_t *out);
 
-/* Diagnostics: for states inside the range episodes visit (|theta| <= 0.25, |theta_dot| <= 20) the
+/* Diagnostics: for states inside the range episodes visit (|theta| <= 0.22, |theta_dot| <= 20) the
  * kernels compute the angular acceleration's quotient with the hardware reciprocal plus one exact
  * correction instead of the general division. This compares the two over the whole operand domain
  * of such states: every den_step-th float32 denominator in [0.6210, 0.6242] (53,688 values at
