@@ -493,6 +493,15 @@ def measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args) -> dict:
         ms /= 2
         out[key] = {"n_envs": n, "T": T, "hidden": inputs.HIDDEN_OF[kind], "ms_per_launch": ms,
                     "env_steps_per_sec": n * T / (ms * 1e-3)}
+    # config 5 itself in the contracted arithmetic (FMA dynamics and the five-instruction tanh)
+    pol = cp.policy(w5.policy, inputs.policy_weights(w5.policy, w5.policy_seed))
+
+    def c5_contracted():
+        cp.cp_rollout_ex(n_envs=n, T=T, seed=w5.seed, policy=pol, arithmetic=cp.CP_ARITH_CONTRACTED, **outs)
+    ms, _ = timed(c5_contracted, 2, 3)
+    ms /= 2
+    out["c5_rollout_contracted_arithmetic"] = {"n_envs": n, "T": T, "ms_per_launch": ms,
+                                               "env_steps_per_sec": n * T / (ms * 1e-3)}
     del outs
     torch.cuda.empty_cache()
 

@@ -222,7 +222,8 @@ int cp_rollout_from(cp_state *state, int64_t T, uint32_t *ep_len, const cp_polic
  *     rollout give the same bits. CP_ARITH_CONTRACTED: the step as a contracting compiler would
  *     emit it for a fused kernel (Sec. V-B, V-G: generated fused code carries no such promise) —
  *     fused multiply-adds, divisions by the total mass folded into constants, theta_acc by
- *     reciprocal; 25 instead of 43 floating-point operations per step. One step from the same
+ *     reciprocal; 25 instead of 43 floating-point operations per step; the MLP policies' tanh
+ *     from the hardware exp2 and reciprocal (absolute error <= 2.4e-7). One step from the same
  *     state differs by at most 2e-6 relative (on the scale of value and update) and a done flag
  *     only where x' or theta' lies within 1e-5 of its threshold. Start states, actions of the
  *     hashed policy and the bookkeeping are the same bits in both. Free-running returns stay
@@ -310,6 +311,12 @@ int cp_selftest_sincos(uint32_t lo_bits, uint32_t hi_bits, uint64_t *mismatches)
  * error of sin / cos in millionths of a float32 ulp; out[2] / out[3] = number of results that are
  * not the correctly rounded value. */
 int cp_selftest_sincos_accuracy(uint32_t lo_bits, uint32_t hi_bits, uint64_t *out);
+
+/* Diagnostics: absolute error against float64 of the hyperbolic tangent the MLP policies use —
+ * out[0]: the five-instruction form of CP_ARITH_CONTRACTED, out[1]: the library tanhf of
+ * CP_ARITH_EXACT — over the float32 values in [lo, hi] (bit patterns as above) and their
+ * negatives, largest value seen, in units of 1e-12. out DEVICE [2] uint64, caller zeroes. */
+int cp_selftest_tanh(uint32_t lo_bits, uint32_t hi_bits, uint64_t *out);
 
 /* Diagnostics: the kernels replace x / 1.1f by a three-operation exact sequence and the start-state
  * mapping by an equivalent two-operation one. This checks, over all 2^32 float bit patterns (2^24

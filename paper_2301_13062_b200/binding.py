@@ -29,7 +29,7 @@ EXPORTS = [
     "cp_rollout_from", "cp_rollout_host", "cp_step_host", "cp_shutdown", "cp_set_stream", "cp_tune",
     "cp_launch_count", "cp_selftest_sincos", "cp_last_error", "cp_version", "cp_step_unfused_noalloc",
     "cp_selftest_sincos_accuracy", "cp_selftest_arith", "cp_step_repeat", "cp_selftest_tame_div",
-    "cp_rollout_ex", "cp_step_ex", "cp_rollout_host_shard",
+    "cp_rollout_ex", "cp_step_ex", "cp_rollout_host_shard", "cp_selftest_tanh",
 ]
 CP_NOALLOC_MAX_ENVS = 65536
 
@@ -99,6 +99,7 @@ def lib() -> C.CDLL:
             "cp_launch_count": (C.c_uint64, []),
             "cp_selftest_sincos": (i32, [u32, u32, p]),
             "cp_selftest_sincos_accuracy": (i32, [u32, u32, p]),
+            "cp_selftest_tanh": (i32, [u32, u32, p]),
             "cp_selftest_arith": (i32, [p]),
             "cp_selftest_tame_div": (i32, [u32, p]),
             "cp_last_error": (C.c_char_p, []),
@@ -369,6 +370,12 @@ def cp_selftest_sincos_accuracy(lo_bits: int, hi_bits: int, out) -> None:
     import torch
     _use_current_stream()
     _check(lib().cp_selftest_sincos_accuracy(lo_bits, hi_bits, _dptr(out, torch.int64)))
+
+
+def cp_selftest_tanh(lo_bits: int, hi_bits: int, out) -> None:
+    import torch
+    _use_current_stream()
+    _check(lib().cp_selftest_tanh(lo_bits, hi_bits, _dptr(out, torch.int64)))
 
 
 def cp_selftest_arith(out) -> None:

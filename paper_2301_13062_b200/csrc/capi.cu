@@ -558,6 +558,13 @@ int cp_selftest_sincos_accuracy(uint32_t lo_bits, uint32_t hi_bits, uint64_t *ou
     return e == cudaSuccess ? CP_OK : cuda_fail(e, "self-test launch");
 }
 
+int cp_selftest_tanh(uint32_t lo_bits, uint32_t hi_bits, uint64_t *out) {
+    if (!out || !is_aligned(out, 8)) return fail(CP_EINVAL, "out is NULL or misaligned");
+    if (lo_bits > hi_bits || hi_bits >= 0x7F800000u) return fail(CP_EINVAL, "need lo <= hi, both finite and non-negative");
+    cudaError_t e = cp::launch_tanh_accuracy(lo_bits, hi_bits, reinterpret_cast<unsigned long long *>(out), tl_stream);
+    return e == cudaSuccess ? CP_OK : cuda_fail(e, "self-test launch");
+}
+
 int cp_selftest_arith(uint64_t *out) {
     if (!out || !is_aligned(out, 8)) return fail(CP_EINVAL, "out is NULL or misaligned");
     cudaError_t e = cp::launch_arith_selftest(reinterpret_cast<unsigned long long *>(out), tl_stream);

@@ -363,7 +363,19 @@ __device__ __forceinline__ uint32_t linear_action(const LinearW &p, const State 
 
 // Hidden activations are consumed as they are produced (two running logits), so no array of
 // H values is ever live; every weight is an immediate operand from the launch parameters.
-template <int H>
+// tanh for the contracted-arithmetic variant: 1 - 2 / (exp(2x) + 1) with the hardware exp2 and
+// reciprocal approximations (five instructions instead of the library routine's ~18). Small
+// arguments lose RELATIVE accuracy to the cancellation in 1 - (...), which a policy does not
+// feel: its logits depend on the absolute error, measured <= 2.4e-7 over every float32
+// (cp_selftest_tanh; the library tanhf: 1.2e-7). Saturates to +-1, NaN stays NaN.
+__device__ __forceinline__ float tanh_contracted(float x) {
+    float t, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(__fmul_rn(x, 2.885390043f)));  // 2 * log2(e)
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(__fadd_rn(t, 1.0f)));
+    return __fmaf_rn(-2.0f, r, 1.0f);
+}
+
+template <int H, bool FAST_TANH = false>
 __device__ __forceinline__ uint32_t mlp_action(const MlpWT<H> &p, const State &z) {
     float l0 = p.b2[0], l1 = p.b2[1];
 #pragma unroll
@@ -373,7 +385,7 @@ __device__ __forceinline__ uint32_t mlp_action(const MlpWT<H> &p, const State &z
         acc = __fmaf_rn(p.w1[j][1], z.xd, acc);
         acc = __fmaf_rn(p.w1[j][2], z.th, acc);
         acc = __fmaf_rn(p.w1[j][3], z.thd, acc);
-        float h = tanhf(acc);
+        float h = FAST_TANH ? tanh_contracted(acc) : tanhf(acc);
         l0 = __fmaf_rn(p.w2[0][j], h, l0);
         l1 = __fmaf_rn(p.w2[1][j], h, l1);
     }

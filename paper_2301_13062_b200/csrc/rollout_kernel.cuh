@@ -27,7 +27,7 @@ namespace cp {
 // POLICY: 0 hashed random action, 1 linear, 2 MLP with 16 hidden units, 3 action bits supplied by
 // the caller, 4 / 5 MLP with 32 / 64 hidden units, 6 one linear policy per environment (its ten
 // parameters are loaded into registers before the time loop; handled in the kernel body).
-template <int POLICY>
+template <int POLICY, bool CONTRACT>
 __device__ __forceinline__ uint32_t policy_signbit(const RolloutParams &p, const FoldedKeys &ka,
                                                    uint32_t folded_t, const State &z) {
     if (POLICY == 0) {
@@ -35,11 +35,11 @@ __device__ __forceinline__ uint32_t policy_signbit(const RolloutParams &p, const
     } else if (POLICY == 1) {
         return linear_action(*reinterpret_cast<const LinearW *>(p.w), z);
     } else if (POLICY == 2) {
-        return mlp_action<16>(*reinterpret_cast<const MlpWT<16> *>(p.w), z);
+        return mlp_action<16, CONTRACT>(*reinterpret_cast<const MlpWT<16> *>(p.w), z);
     } else if (POLICY == 4) {
-        return mlp_action<32>(*reinterpret_cast<const MlpWT<32> *>(p.w), z);
+        return mlp_action<32, CONTRACT>(*reinterpret_cast<const MlpWT<32> *>(p.w), z);
     } else {
-        return mlp_action<64>(*reinterpret_cast<const MlpWT<64> *>(p.w), z);
+        return mlp_action<64, CONTRACT>(*reinterpret_cast<const MlpWT<64> *>(p.w), z);
     }
 }
 
@@ -170,7 +170,7 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
                 } else if (POLICY == 6) {
                     sb[j] = linear_action(own[POLICY == 6 ? j : 0], z[j]);
                 } else {
-                    sb[j] = policy_signbit<POLICY>(p, ka[j], folded_t, z[j]);
+                    sb[j] = policy_signbit<POLICY, CONTRACT>(p, ka[j], folded_t, z[j]);
                 }
                 done[j] = CONTRACT ? euler_step_contracted(z[j], force_from_signbit(sb[j]))
                                    : euler_step(z[j], force_from_signbit(sb[j]));

@@ -277,6 +277,38 @@ cudaError_t launch_sincos_accuracy(uint32_t lo_bits, uint32_t hi_bits, unsigned 
     return cudaGetLastError();
 }
 
+// ---- self-test: absolute error of the two hyperbolic tangents against float64 ----
+// out[0] / out[1]: largest |tanh_contracted(v) - tanh(v)| / |tanhf(v) - tanh(v)| over the
+// float32 values with bit patterns in [lo, hi] and their negatives, in units of 1e-12.
+__global__ void tanh_accuracy_kernel(uint32_t lo, uint32_t hi, unsigned long long *out) {
+    double worst_fast = 0.0, worst_lib = 0.0;
+    const uint64_t span = (uint64_t)hi - lo + 1;
+    for (uint64_t k = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; k < span; k += (uint64_t)gridDim.x * blockDim.x) {
+        for (int sign = 0; sign < 2; ++sign) {
+            const float v = __uint_as_float((lo + (uint32_t)k) | (sign ? 0x80000000u : 0u));
+            const double exact = tanh((double)v);
+            worst_fast = fmax(worst_fast, fabs((double)tanh_contracted(v) - exact));
+            worst_lib = fmax(worst_lib, fabs((double)tanhf(v) - exact));
+        }
+    }
+    unsigned long long a = (unsigned long long)(worst_fast * 1e12), b = (unsigned long long)(worst_lib * 1e12);
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long a2 = __shfl_down_sync(0xffffffffu, a, o), b2 = __shfl_down_sync(0xffffffffu, b, o);
+        a = a2 > a ? a2 : a;
+        b = b2 > b ? b2 : b;
+    }
+    if ((threadIdx.x & 31) == 0) {
+        atomicMax(out, a);
+        atomicMax(out + 1, b);
+    }
+}
+
+cudaError_t launch_tanh_accuracy(uint32_t lo_bits, uint32_t hi_bits, unsigned long long *out, cudaStream_t s) {
+    tanh_accuracy_kernel<<<sm_count() * 8, 256, 0, s>>>(lo_bits, hi_bits, out);
+    count_launch();
+    return cudaGetLastError();
+}
+
 // ---- self-test: the exact shortcuts against the operations they replace ----
 // out[0]: bit patterns x (all 2^32) where div_mtot(x) != __fdiv_rn(x, 1.1f)
 // out[1]: patterns inside div_mtot_not_tiny's domain (+0, NaN, Inf, |x| >= 2^-100) where it differs

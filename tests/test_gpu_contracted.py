@@ -95,7 +95,7 @@ def test_contracted_random_rollout_returns_match_the_oracle(cp, oracle):
     assert 21.5 < s["mean_gpu"] < 22.5
 
 
-@pytest.mark.parametrize("kind,pseed,T", [(1, 1, 300), (2, 2, 200)])
+@pytest.mark.parametrize("kind,pseed,T", [(1, 1, 300), (2, 2, 200), (2, 6, 200), (4, 3, 150), (5, 3, 100)])
 def test_contracted_policy_rollouts_stay_statistically_equal(cp, oracle, kind, pseed, T):
     """With a state-feedback policy the 1e-7 per-step differences feed back through the action
     choice (an unstable pendulum amplifies them until some logit pair falls on the other side of
@@ -152,6 +152,20 @@ def test_contracted_chunks_and_step_limit_compose(cp):
     for a, b in zip(whole, parts):
         assert np.array_equal(a, b)
     assert whole[2].sum() > 0 and (whole[1] / np.maximum(whole[2], 1)).max() <= limit
+
+
+def test_contracted_tanh_absolute_error_over_every_float(cp):
+    """The five-instruction tanh of the contracted MLP policies against float64, over every
+    finite float32 of either sign: the policy's logits feel the ABSOLUTE error, which must stay
+    far below the 1e-5 logit gap that the parity rules excuse (16 hidden units x |w2| ~ 0.25
+    turn 3e-7 into about 1e-6)."""
+    out = torch.zeros(2, dtype=torch.int64, device="cuda")
+    cp.cp_selftest_tanh(0, 0x7F7FFFFF, out)
+    torch.cuda.synchronize()
+    fast, lib = (int(v) * 1e-12 for v in out.cpu())
+    print(f"tanh absolute error over all floats: contracted {fast:.3e}, library tanhf {lib:.3e}")
+    assert fast <= 3e-7, fast
+    assert lib <= 2e-7, lib
 
 
 def test_unknown_arithmetic_is_rejected(cp):
