@@ -285,11 +285,13 @@ void cp_shutdown(void);
 void cp_set_stream(void *cuda_stream);
 
 /* Launch tuning, process-wide. key: "rollout_block" (threads per CTA, 32..256, multiple of 32;
- * default 256), "rollout_ept" (environments per thread: 1 or 2; 0 = default, 2 for large
+ * 0 = default: 128 for very small batches, else 256), "rollout_ept" (environments per thread: 1 or 2; 0 = default, 2 for large
  * batches except with the MLP policies), "rollout_coop" (how finished environments get their
- * start state: 1 = by the whole warp through shared memory, 2 = each lane its own, only with one
- * environment per thread; 0 = default: per lane for batches too small to fill the GPU, by the
- * warp otherwise; every choice gives the same bits), "rollout_ctas_per_sm" (0 = default: one 32*ept-environment task per warp and as many
+ * start state: 1 = by the whole warp through shared memory, 2 = each lane its own when its env
+ * finishes, 3 = each lane computes it every step ahead of the dynamics (hashed or supplied
+ * actions only, otherwise as 2), 2 and 3 only with one environment per thread; 0 = default: per
+ * lane for batches too small to fill the GPU (ahead for the very small), by the warp otherwise;
+ * every choice gives the same bits), "rollout_ctas_per_sm" (0 = default: one 32*ept-environment task per warp and as many
  * CTAs as that takes; k > 0 = persistent grid of k CTAs per SM looping over tasks), "step_block"
  * (32..256, default 64), "step_vec_min_envs" (batches smaller than this use the one-env-per-thread
  * step kernel even when the four-envs-per-thread vector form is possible; default 262144),

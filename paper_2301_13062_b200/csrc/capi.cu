@@ -515,13 +515,14 @@ void cp_set_stream(void *cuda_stream) { tl_stream = static_cast<cudaStream_t>(cu
 int cp_tune(const char *key, int value) {
     if (!key) return fail(CP_EINVAL, "key is NULL");
     if (!strcmp(key, "rollout_block")) {
-        if (value < 32 || value > 256 || value % 32) return fail(CP_EINVAL, "rollout_block must be 32..256, multiple of 32");
+        if (value != 0 && (value < 32 || value > 256 || value % 32))
+            return fail(CP_EINVAL, "rollout_block must be 0 or 32..256, multiple of 32");
         cp::g_tuning.rollout_block = value;
     } else if (!strcmp(key, "rollout_ept")) {
         if (value != 0 && value != 1 && value != 2) return fail(CP_EINVAL, "rollout_ept must be 0, 1 or 2");
         cp::g_tuning.rollout_ept = value;
     } else if (!strcmp(key, "rollout_coop")) {
-        if (value != 0 && value != 1 && value != 2) return fail(CP_EINVAL, "rollout_coop must be 0, 1 or 2");
+        if (value < 0 || value > 3) return fail(CP_EINVAL, "rollout_coop must be 0, 1, 2 or 3");
         cp::g_tuning.rollout_coop = value;
     } else if (!strcmp(key, "rollout_ctas_per_sm")) {
         if (value < 0 || value > 1024) return fail(CP_EINVAL, "rollout_ctas_per_sm must be 0..1024");

@@ -48,7 +48,7 @@ struct RolloutParams {
 };
 
 struct LaunchTuning {
-    int rollout_block = 256;
+    int rollout_block = 0;        // 0: 128 for very small batches, 256 otherwise
     int rollout_ept = 0;          // 0: chosen per policy and batch size
     int rollout_coop = 0;         // 0: chosen per batch size; 1 restarts by the warp; 2 per lane (ept 1)
     int rollout_ctas_per_sm = 0;  // 0: one task per warp (non-persistent grid)

@@ -22,11 +22,11 @@ BAND = 1e-5
 REL_TOL = 2e-6
 
 
-# The rollout kernel's three work shapes as (rollout_ept, rollout_coop) tuning values: one env
-# per thread with per-lane restarts, one env per thread with restarts by the whole warp, two
-# envs per thread (always by the warp). The library picks one by batch size and policy; tests
-# force each of them on small batches.
-SHAPES = [(1, 2), (1, 1), (2, 1)]
+# The rollout kernel's work shapes as (rollout_ept, rollout_coop) tuning values: one env per
+# thread with per-lane restarts, the same with start states computed ahead every step, one env
+# per thread with restarts by the whole warp, two envs per thread (always by the warp). The
+# library picks one by batch size and policy; tests force each of them on small batches.
+SHAPES = [(1, 2), (1, 3), (1, 1), (2, 1)]
 
 
 @contextlib.contextmanager

@@ -258,7 +258,7 @@ def test_per_env_linear_policies_against_oracle(cp, oracle):
             cp.cp_rollout_shard(off, n, T, seed, cp.policy(cp.CP_POLICY_LINEAR_PER_ENV, d_w), **out)
             res.append(fetch(out))
     for k in res[0]:
-        assert np.array_equal(res[0][k], res[1][k]) and np.array_equal(res[0][k], res[2][k]), k
+        assert all(np.array_equal(res[0][k], other[k]) for other in res[1:]), k
     r = res[0]
     o = oracle.rollout(n, T, seed, inputs.POLICY_LINEAR_PER_ENV, wp, env_offset=off, done_bits=True,
                        action_bits=True, min_gap=True, nthreads=8)
