@@ -38,11 +38,11 @@ SMS = 148
 # smsp__inst_executed.sum / (N*T) of the kernel the library launches by default at this size
 # (restarts by the whole warp): the issue slots it really occupies.
 ROLLOUT_OPS = {
-    "random": {"thread": 72.6, "slot": 92.8},
-    "linear": {"thread": 76.8, "slot": 83.5},
-    "linear+streams": {"thread": 94.9, "slot": 98.6},
-    "mlp": {"thread": 441.3, "slot": 470.2},
-    "random+contracted": {"thread": 55.6, "slot": 74.4},
+    "random": {"thread": 69.6, "slot": 89.8},
+    "linear": {"thread": 73.8, "slot": 80.5},
+    "linear+streams": {"thread": 91.9, "slot": 95.6},
+    "mlp": {"thread": 438.3, "slot": 467.2},
+    "random+contracted": {"thread": 53.6, "slot": 72.4},
 }
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch in the same captures.
 ROLLOUT_DRAM_BYTES = {"random": 20.7e3, "linear": 20.5e3, "linear+streams": 381.2e6, "mlp": 32.5e3}
