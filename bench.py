@@ -45,8 +45,8 @@ ROLLOUT_OPS = {
     "random+contracted": {"thread": 53.6, "slot": 72.4},
 }
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch in the same captures.
-ROLLOUT_DRAM_BYTES = {"random": 20.7e3, "linear": 20.5e3, "linear+streams": 381.2e6, "mlp": 32.5e3}
-STEP_DRAM_BYTES_16M = 567.8e6  # step_kernel at 16,777,216 envs, same kind of capture
+ROLLOUT_DRAM_BYTES = {"random": 24.3e3, "linear": 24.6e3, "linear+streams": 382.3e6, "mlp": 22.5e3}
+STEP_DRAM_BYTES_16M = 566.9e6  # step_kernel at 16,777,216 envs, same kind of capture
 # Algorithmic HBM bytes per env-step of the step paths.
 STEP_BYTES = 37.0      # 16 in + 16 out + 4 reward + 1 done, hashed action
 LADDER_BYTES = 375.0   # sum over the 46 one-op kernels of their input and output planes
