@@ -284,6 +284,15 @@ void cp_shutdown(void);
 /* Stream used by this thread's later calls (a cudaStream_t; NULL = legacy default stream). */
 void cp_set_stream(void *cuda_stream);
 
+/* Device allocator used by cp_reset for the batches it owns, process-wide: alloc(bytes) returns a
+ * DEVICE pointer aligned to at least 16 bytes or NULL, release(ptr) takes it back (a handle keeps
+ * the release function it was created under, so the allocator may change while handles live).
+ * Both NULL (the default) = cudaMalloc / cudaFree. A host program that runs its own caching
+ * allocator (torch's, for instance) passes that, so that cp_reset neither synchronises the device
+ * nor takes memory the host program cannot see. Everything else the library touches is
+ * caller-provided, except the staging buffer of the HOST-buffer calls (always cudaMalloc). */
+int cp_set_allocator(void *(*alloc)(size_t), void (*release)(void *));
+
 /* Launch tuning, process-wide. key: "rollout_block" (threads per CTA, 32..256, multiple of 32;
  * 0 = default: 128 for very small batches, else 256), "rollout_ept" (environments per thread: 1 or 2; 0 = default, 2 for large
  * batches except with the MLP policies), "rollout_coop" (how finished environments get their

@@ -29,7 +29,7 @@ EXPORTS = [
     "cp_rollout_from", "cp_rollout_host", "cp_step_host", "cp_shutdown", "cp_set_stream", "cp_tune",
     "cp_launch_count", "cp_selftest_sincos", "cp_last_error", "cp_version", "cp_step_unfused_noalloc",
     "cp_selftest_sincos_accuracy", "cp_selftest_arith", "cp_step_repeat", "cp_selftest_tame_div",
-    "cp_rollout_ex", "cp_step_ex", "cp_rollout_host_shard", "cp_selftest_tanh",
+    "cp_rollout_ex", "cp_step_ex", "cp_rollout_host_shard", "cp_selftest_tanh", "cp_set_allocator",
 ]
 CP_NOALLOC_MAX_ENVS = 65536
 
@@ -60,6 +60,9 @@ class CartpoleError(RuntimeError):
 
 
 _lib = None
+ALLOC_FN = C.CFUNCTYPE(C.c_void_p, C.c_size_t)
+RELEASE_FN = C.CFUNCTYPE(None, C.c_void_p)
+_allocator_callbacks = None  # keeps the ctypes thunks alive while the library may call them
 
 
 def lib() -> C.CDLL:
@@ -95,6 +98,7 @@ def lib() -> C.CDLL:
             "cp_step_host": (i32, [i64, u32, u32, p, p, p, p, p]),
             "cp_shutdown": (None, []),
             "cp_set_stream": (None, [p]),
+            "cp_set_allocator": (i32, [ALLOC_FN, RELEASE_FN]),
             "cp_tune": (i32, [C.c_char_p, i32]),
             "cp_launch_count": (C.c_uint64, []),
             "cp_selftest_sincos": (i32, [u32, u32, p]),
@@ -144,6 +148,31 @@ def _hptr(a):
 def _use_current_stream() -> None:
     import torch
     lib().cp_set_stream(C.c_void_p(torch.cuda.current_stream().cuda_stream))
+
+
+def cp_set_allocator(alloc=None, release=None) -> None:
+    """Device allocator of cp_reset: two callables (bytes -> device address or 0, address -> None),
+    or nothing for cudaMalloc / cudaFree. `use_torch_allocator()` passes torch's caching allocator."""
+    global _allocator_callbacks
+    if (alloc is None) != (release is None):
+        raise ValueError("alloc and release go together")
+    if alloc is None:
+        _check(lib().cp_set_allocator(ALLOC_FN(0), RELEASE_FN(0)))
+        return
+    thunks = (ALLOC_FN(lambda n: alloc(n) or 0), RELEASE_FN(lambda ptr: release(ptr)))
+    _check(lib().cp_set_allocator(*thunks))
+    # never dropped: a live handle keeps the release function it was created under
+    _allocator_callbacks = (_allocator_callbacks or []) + [thunks]
+
+
+def use_torch_allocator(enable: bool = True) -> None:
+    """Let cp_reset take its batches from torch's CUDA caching allocator (no cudaMalloc, hence no
+    device-wide synchronisation, and the memory shows up in torch's own accounting)."""
+    import torch
+    if enable:
+        cp_set_allocator(torch.cuda.caching_allocator_alloc, torch.cuda.caching_allocator_delete)
+    else:
+        cp_set_allocator(None, None)
 
 
 class _Policy:

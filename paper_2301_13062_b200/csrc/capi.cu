@@ -18,6 +18,7 @@ struct cp_state {
     uint32_t seed, t, env_offset;
     float *planes;
     bool owns;
+    void (*release)(void *);  // how owned planes go back: the allocator's release, or NULL = cudaFree
 };
 
 namespace cp {
@@ -45,6 +46,11 @@ namespace {
 
 thread_local cudaStream_t tl_stream = nullptr;
 thread_local char tl_error[512] = "";
+
+// Device allocator of cp_reset (cp_set_allocator); both NULL = cudaMalloc / cudaFree.
+std::mutex g_alloc_mu;
+void *(*g_alloc)(size_t) = nullptr;
+void (*g_release)(void *) = nullptr;
 
 int fail(int code, const char *fmt, ...) {
     va_list ap;
@@ -238,22 +244,51 @@ cp_state *cp_reset(int64_t n_envs, uint32_t seed) {
     s->env_offset = 0;
     s->owns = true;
     s->planes = nullptr;
-    cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&s->planes), (size_t)s->stride * 4 * sizeof(float));
-    if (e != cudaSuccess) {
-        (void)cudaGetLastError();
-        fail(CP_ENOMEM, "cudaMalloc of %lld envs failed: %s", (long long)n_envs, cudaGetErrorString(e));
-        delete s;
-        return nullptr;
+    s->release = nullptr;
+    const size_t bytes = (size_t)s->stride * 4 * sizeof(float);
+    void *(*alloc)(size_t);
+    {
+        std::lock_guard<std::mutex> lock(g_alloc_mu);
+        alloc = g_alloc;
+        s->release = g_release;
+    }
+    cudaError_t e;
+    if (alloc) {
+        s->planes = static_cast<float *>(alloc(bytes));
+        if (!s->planes || !is_aligned(s->planes, 16)) {
+            fail(CP_ENOMEM, "the allocator returned %s for %zu bytes", s->planes ? "a pointer not 16-byte aligned" : "NULL",
+                 bytes);
+            if (s->planes && s->release) s->release(s->planes);
+            delete s;
+            return nullptr;
+        }
+    } else {
+        e = cudaMalloc(reinterpret_cast<void **>(&s->planes), bytes);
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();
+            fail(CP_ENOMEM, "cudaMalloc of %lld envs failed: %s", (long long)n_envs, cudaGetErrorString(e));
+            delete s;
+            return nullptr;
+        }
     }
     // pad lanes hold start states too, so vector loads never see uninitialised memory
     e = cp::launch_fill_start(s->planes, s->stride, s->stride, 0, cp::salt(seed, 1u), 0, tl_stream);
     if (e != cudaSuccess) {
         cuda_fail(e, "start-state launch");
-        cudaFree(s->planes);
+        if (s->release) s->release(s->planes); else cudaFree(s->planes);
         delete s;
         return nullptr;
     }
     return s;
+}
+
+int cp_set_allocator(void *(*alloc)(size_t), void (*release)(void *)) {
+    if ((alloc == nullptr) != (release == nullptr))
+        return fail(CP_EINVAL, "alloc and release must be given together (or both NULL for cudaMalloc / cudaFree)");
+    std::lock_guard<std::mutex> lock(g_alloc_mu);
+    g_alloc = alloc;
+    g_release = release;
+    return CP_OK;
 }
 
 cp_state *cp_wrap(float *planes, int64_t n_envs, int64_t plane_stride, uint32_t seed, uint32_t t,
@@ -276,7 +311,7 @@ cp_state *cp_wrap(float *planes, int64_t n_envs, int64_t plane_stride, uint32_t 
         fail(CP_ENOMEM, "out of host memory");
         return nullptr;
     }
-    *s = cp_state{n_envs, plane_stride, seed, t, env_offset, planes, false};
+    *s = cp_state{n_envs, plane_stride, seed, t, env_offset, planes, false, nullptr};
     return s;
 }
 
@@ -297,7 +332,9 @@ int cp_set_time(cp_state *state, uint32_t t) {
 
 void cp_free(cp_state *state) {
     if (!state) return;
-    if (state->owns && state->planes) cudaFree(state->planes);
+    if (state->owns && state->planes) {
+        if (state->release) state->release(state->planes); else cudaFree(state->planes);
+    }
     delete state;
 }
 

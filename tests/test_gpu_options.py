@@ -275,3 +275,43 @@ def test_per_env_linear_policies_against_oracle(cp, oracle):
         assert np.array_equal(ra[k], rb[k]), k
     # fitness differs across the population
     assert r["ep_return_sum"].std() > 1 and len(set(r["ep_count"].tolist())) > 5
+
+
+def test_reset_through_the_host_program_allocator(cp, oracle):
+    """cp_set_allocator: cp_reset takes its batch from torch's caching allocator (visible in torch's
+    accounting, returned on cp_free) and the batch behaves like any other."""
+    n = 200_003
+    torch.cuda.synchronize()
+    before = torch.cuda.memory_allocated()
+    cp.use_torch_allocator(True)
+    try:
+        st = cp.cp_reset(n, 9)
+        held = torch.cuda.memory_allocated() - before
+        assert held >= 16 * n, held
+        cp.use_torch_allocator(False)          # the handle keeps the release function it was made with
+        # one step out of the library-owned batch into torch memory: the start states were filled
+        reward = torch.empty(n, device="cuda")
+        done = torch.empty(n, dtype=torch.uint8, device="cuda")
+        planes = torch.zeros(4, (n + 3) // 4 * 4, device="cuda")
+        out = cp.cp_wrap(planes, n, 9)
+        cp.cp_step(st, None, out, reward, done)
+        torch.cuda.synchronize()
+        z0 = oracle.initial_state(n, 9)
+        H.assert_step_matches(oracle.step(z0, seed=9, t=0, want_pre_reset=True), z0, host(planes[:, :n]),
+                              host(reward), host(done))
+        # and a rollout in place on it
+        ret = torch.empty(n, device="cuda")
+        cnt = torch.empty(n, dtype=torch.int32, device="cuda")
+        cp.cp_rollout_from(st, 50, None, None, ep_return_sum=ret, ep_count=cnt)
+        torch.cuda.synchronize()
+        o = oracle.rollout(n, 50, 9, nthreads=4)
+        H.assert_returns_match(host(ret), host(cnt).view(np.uint32), o["ep_return_sum"], o["ep_count"])
+        assert st.info()["t"] == 50
+        with_batch = torch.cuda.memory_allocated()
+        cp.cp_free(st)
+        assert torch.cuda.memory_allocated() == with_batch - held   # went back through torch
+        st2 = cp.cp_reset(1000, 1)             # default allocator again: invisible to torch
+        assert torch.cuda.memory_allocated() == with_batch - held
+        cp.cp_free(st2)
+    finally:
+        cp.use_torch_allocator(False)

@@ -122,6 +122,38 @@ def test_general_rollout_rejects_bad_arguments_on_the_host(cp):
     assert L.cp_rollout_ex(None) == cp.CP_EINVAL
 
 
+def test_allocator_hooks_are_called_and_paired(cp):
+    """cp_reset takes its batch from the installed allocator and gives it back through the paired
+    release function: checked with a fake allocator (on a machine without a GPU the start-state
+    launch fails, and the batch must come back through release before cp_reset returns NULL)."""
+    import torch
+    L = cp.lib()
+    assert L.cp_set_allocator(cp.ALLOC_FN(lambda n: 0), cp.RELEASE_FN(0)) == cp.CP_EINVAL
+    if torch.cuda.is_available():
+        pytest.skip("the fake device pointer must never reach a real launch")
+    calls = []
+
+    def alloc(nbytes):
+        calls.append(("alloc", nbytes))
+        return 0x7000_0000_0000 if nbytes < (1 << 30) else 0
+
+    def release(ptr):
+        calls.append(("release", ptr))
+
+    cp.cp_set_allocator(alloc, release)
+    try:
+        assert not L.cp_reset(1001, 3)                     # no device: launch error
+        assert calls == [("alloc", 1004 * 16), ("release", 0x7000_0000_0000)]
+        calls.clear()
+        assert not L.cp_reset(1 << 27, 3)                  # allocator says no
+        assert calls == [("alloc", (1 << 27) * 16)] and b"allocator returned NULL" in L.cp_last_error()
+    finally:
+        cp.cp_set_allocator(None, None)
+    calls.clear()
+    assert not L.cp_reset(8, 0)                            # default allocator again: hooks untouched
+    assert calls == []
+
+
 def test_wrap_bookkeeping_needs_no_gpu(cp):
     L = cp.lib()
     fake = C.c_void_p(0x7000_0000_0100)  # never dereferenced on the host
