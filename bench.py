@@ -444,6 +444,43 @@ def measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args) -> dict:
                      "fused_step_over_ladder_hbm": out["fused_step_hbm"]["env_steps_per_sec"] / out["ladder_hbm"]["env_steps_per_sec"]}
     del a, b, sa, sb, reward, done, ws
 
+    # the paper's own batch shape (2,048 envs; Sec. V) on the per-step paths, for its ratios:
+    # ladder -> fused step -> (paper_rollout below), all launch-bound at this size
+    wp = inputs.WORKLOADS["paper"]
+    n = wp.n_envs
+    a, b, sa, sb, reward, done = step_setup(n)
+    ws = torch.empty(cp.cp_unfused_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+
+    def paper_fused():
+        cp.cp_set_time(sa, 0)
+        cp.cp_step_repeat(sa, 1000, reward, done)
+
+    def paper_ladder():
+        cp.cp_set_time(sa, 0)
+        for _ in range(50):
+            cp.cp_step_unfused(sa, None, sb, reward, done, ws)
+            cp.cp_step_unfused(sb, None, sa, reward, done, ws)
+
+    ms, _ = timed(paper_fused, 3, 3, flush=False)
+    ms /= 3
+    out["paper_fused_step"] = {"n_envs": n, "T": 1000, "us_per_launch": 1e3 * ms / 1000, "env_steps_per_sec": n * 1000 / (ms * 1e-3)}
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        paper_fused()
+        side.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            paper_fused()
+    torch.cuda.synchronize()
+    ms, _ = timed(graph.replay, 3, 3, flush=False)
+    ms /= 3
+    out["paper_fused_step_graph"] = {"n_envs": n, "T": 1000, "us_per_launch": 1e3 * ms / 1000,
+                                     "env_steps_per_sec": n * 1000 / (ms * 1e-3)}
+    ms, _ = timed(paper_ladder, 3, 3, flush=False)
+    ms /= 3
+    out["paper_ladder"] = {"n_envs": n, "T": 100, "us_per_step": 1e3 * ms / 100,
+                           "env_steps_per_sec": n * 100 / (ms * 1e-3), "launches_per_step": 46}
+    del a, b, sa, sb, reward, done, ws, graph
+
     # options of the general rollout call on the headline shape: CartPole-v1's 500-step episode
     # limit, and actions supplied as a packed bit stream (here: the hashed ones, written by a
     # first rollout) instead of drawn in the kernel

@@ -259,6 +259,41 @@ void co_mlp_logits_wide(const float *w, int H, const float z[4], float logits[2]
     logits[1] = acc1;
 }
 
+/* A deeper network (kind 7): 4 -> 16 (tanh) -> 16 (tanh) -> 2, the paper's
+ * future work "fusing simulation with neural network inference" (Sec. VI)
+ * one layer further. W1[16][4], b1[16], W2[16][16], b2[16], W3[2][16],
+ * b3[2] (386 floats); every unit is the left-to-right fmaf chain that
+ * starts from its bias. */
+#define CO_POLICY_MLP_DEEP 7
+void co_mlp_deep_logits(const float *w, const float z[4], float logits[2])
+{
+    const float *w1 = w;
+    const float *b1 = w + 64;
+    const float *w2 = w + 80;
+    const float *b2 = w + 336;
+    const float *w3 = w + 352;
+    const float *b3 = w + 384;
+    float h1[16], h2[16];
+    for (int j = 0; j < 16; ++j) {
+        float acc = b1[j];
+        for (int i = 0; i < 4; ++i)
+            acc = fmaf(w1[4 * j + i], z[i], acc);
+        h1[j] = tanhf(acc);
+    }
+    for (int k = 0; k < 16; ++k) {
+        float acc = b2[k];
+        for (int j = 0; j < 16; ++j)
+            acc = fmaf(w2[16 * k + j], h1[j], acc);
+        h2[k] = tanhf(acc);
+    }
+    for (int m = 0; m < 2; ++m) {
+        float acc = b3[m];
+        for (int k = 0; k < 16; ++k)
+            acc = fmaf(w3[16 * m + k], h2[k], acc);
+        logits[m] = acc;
+    }
+}
+
 /* Action for one environment; *gap (optional) receives |logit1 - logit0|
  * (infinity for the random policy) so tests can excuse argmax near-ties. */
 static int co_policy_action(int kind, const float *w, uint32_t ka0, uint32_t ka1, uint32_t t,
@@ -273,6 +308,8 @@ static int co_policy_action(int kind, const float *w, uint32_t ka0, uint32_t ka1
         co_linear_logits(w, z, logits);
     else if (kind == CO_POLICY_MLP)
         co_mlp_logits(w, z, logits);
+    else if (kind == CO_POLICY_MLP_DEEP)
+        co_mlp_deep_logits(w, z, logits);
     else
         co_mlp_logits_wide(w, kind == CO_POLICY_MLP32 ? 32 : 64, z, logits);
     if (gap) *gap = fabsf(logits[1] - logits[0]);

@@ -19,7 +19,9 @@ _LIB = os.path.join(_HERE, "libcartpole_oracle.so")
 
 POLICY_RANDOM, POLICY_LINEAR, POLICY_MLP, POLICY_MLP32, POLICY_MLP64 = 0, 1, 2, 4, 5
 POLICY_LINEAR_PER_ENV = 6
-N_WEIGHTS = {POLICY_RANDOM: 0, POLICY_LINEAR: 10, POLICY_MLP: 114, POLICY_MLP32: 226, POLICY_MLP64: 450}
+POLICY_MLP_DEEP = 7
+N_WEIGHTS = {POLICY_RANDOM: 0, POLICY_LINEAR: 10, POLICY_MLP: 114, POLICY_MLP32: 226, POLICY_MLP64: 450,
+             POLICY_MLP_DEEP: 386}
 
 
 def build(force: bool = False) -> str:
@@ -74,6 +76,8 @@ def lib() -> C.CDLL:
         L.co_mlp_logits.argtypes = [p, p, p]
         L.co_mlp_logits_wide.restype = None
         L.co_mlp_logits_wide.argtypes = [p, i32, p, p]
+        L.co_mlp_deep_logits.restype = None
+        L.co_mlp_deep_logits.argtypes = [p, p, p]
         L.co_step.restype = None
         L.co_step.argtypes = [u32, i64, i64, i64, u32, u32, p, p, p, p, p, p, p]
         L.co_rollout.restype = None
@@ -172,6 +176,15 @@ def mlp_logits_wide(w, hidden: int, z) -> np.ndarray:
     assert w.size == 7 * hidden + 2
     out = np.empty(2, np.float32)
     lib().co_mlp_logits_wide(_ptr(w), int(hidden), _ptr(z), _ptr(out))
+    return out
+
+
+def mlp_deep_logits(w, z) -> np.ndarray:
+    w = np.ascontiguousarray(w, np.float32)
+    z = np.ascontiguousarray(z, np.float32)
+    assert w.size == 386
+    out = np.empty(2, np.float32)
+    lib().co_mlp_deep_logits(_ptr(w), _ptr(z), _ptr(out))
     return out
 
 

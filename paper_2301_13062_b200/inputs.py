@@ -18,7 +18,9 @@ from dataclasses import dataclass
 import numpy as np
 
 POLICY_RANDOM, POLICY_LINEAR, POLICY_MLP, POLICY_MLP32, POLICY_MLP64 = 0, 1, 2, 4, 5
-N_WEIGHTS = {POLICY_RANDOM: 0, POLICY_LINEAR: 10, POLICY_MLP: 114, POLICY_MLP32: 226, POLICY_MLP64: 450}
+POLICY_MLP_DEEP = 7  # 4 -> 16 (tanh) -> 16 (tanh) -> 2
+N_WEIGHTS = {POLICY_RANDOM: 0, POLICY_LINEAR: 10, POLICY_MLP: 114, POLICY_MLP32: 226, POLICY_MLP64: 450,
+             POLICY_MLP_DEEP: 386}
 MLP_HIDDEN = 16
 HIDDEN_OF = {POLICY_MLP: 16, POLICY_MLP32: 32, POLICY_MLP64: 64}
 POLICY_LINEAR_PER_ENV = 6  # a different linear policy for every environment (population search)
@@ -65,6 +67,11 @@ def policy_weights(kind: int, seed: int) -> np.ndarray:
         l1 = 0.5 * rng.standard_normal(4 * h + h)
         l2 = (1.0 / np.sqrt(h)) * rng.standard_normal(2 * h + 2)
         return np.concatenate([l1, l2]).astype(np.float32)
+    if kind == POLICY_MLP_DEEP:  # W1[16][4], b1[16]; W2[16][16], b2[16]; W3[2][16], b3[2]; std 1/sqrt(fan_in)
+        l1 = 0.5 * rng.standard_normal(64 + 16)
+        l2 = 0.25 * rng.standard_normal(256 + 16)
+        l3 = 0.25 * rng.standard_normal(32 + 2)
+        return np.concatenate([l1, l2, l3]).astype(np.float32)
     raise ValueError(f"unknown policy kind {kind}")
 
 

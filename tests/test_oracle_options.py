@@ -196,6 +196,61 @@ def test_wide_mlp_routine_reduces_to_the_16_unit_network(oracle):
         assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
 
 
+def test_deep_mlp_policy(oracle):
+    """4 -> 16 (tanh) -> 16 (tanh) -> 2: against a float64 matrix evaluation, a probe that isolates
+    one path through both hidden layers (catches a transposed or shifted weight block), the
+    reduction to the one-hidden-layer network when the second layer is a scaled identity in the
+    linear range of tanh, and the use of the pre-step observation in rollouts."""
+    kind = inputs.POLICY_MLP_DEEP
+    w = inputs.policy_weights(kind, 4)
+    assert w.size == 386 == inputs.N_WEIGHTS[kind]
+    w1, b1 = w[:64].reshape(16, 4).astype(np.float64), w[64:80].astype(np.float64)
+    w2, b2 = w[80:336].reshape(16, 16).astype(np.float64), w[336:352].astype(np.float64)
+    w3, b3 = w[352:384].reshape(2, 16).astype(np.float64), w[384:].astype(np.float64)
+    zs = inputs.random_states(100, seed=8, spread="live")
+    for i in range(zs.shape[1]):
+        z = zs[:, i].astype(np.float64)
+        want = w3 @ np.tanh(w2 @ np.tanh(w1 @ z + b1) + b2) + b3
+        got = oracle.mlp_deep_logits(w, zs[:, i])
+        assert np.all(np.abs(got - want) < 6e-6)
+    # one path: input 2 -> first-layer unit j -> second-layer unit k -> both outputs
+    for j, k in ((0, 15), (7, 3), (15, 0)):
+        probe = np.zeros(386, np.float32)
+        probe[4 * j + 2] = 1.5                 # W1[j][2]
+        probe[64 + j] = 0.25                   # b1[j]
+        probe[80 + 16 * k + j] = 2.0           # W2[k][j]
+        probe[336 + k] = -0.125                # b2[k]
+        probe[352 + k] = 1.0                   # W3[0][k]
+        probe[352 + 16 + k] = -2.0             # W3[1][k]
+        probe[384:] = (0.5, 0.75)
+        got = oracle.mlp_deep_logits(probe, [9, 9, 0.2, 9])
+        h2 = np.tanh(2.0 * np.tanh(1.5 * 0.2 + 0.25) - 0.125)
+        assert abs(got[0] - (0.5 + h2)) < 1e-6 and abs(got[1] - (0.75 - 2 * h2)) < 1e-6
+    # second layer = eps * identity: tanh(eps*h) ~ eps*h, so logits ~ b3 + eps * W3 h1, i.e. the
+    # one-hidden-layer network with its output weights scaled by eps
+    shallow = inputs.policy_weights(inputs.POLICY_MLP, 2)
+    eps = 1e-3
+    deep = np.zeros(386, np.float32)
+    deep[:80] = shallow[:80]
+    deep[80:336] = (eps * np.eye(16)).astype(np.float32).ravel()
+    deep[352:384] = shallow[80:112]
+    for i in range(20):
+        a = oracle.mlp_logits(shallow, zs[:, i]) - shallow[112:]
+        b = oracle.mlp_deep_logits(deep, zs[:, i])
+        assert np.all(np.abs(b - eps * a) < 1e-8)
+    # rollouts: the action is the argmax of the logits on the state BEFORE the step
+    n, T = 32, 25
+    r = oracle.rollout(n, T, 0, kind, w, trajectory=True, action_bits=True, min_gap=True)
+    z = oracle.initial_state(n, 0)
+    for t in range(T):
+        ab = unpack_bits(r["action_bits"][t], n)
+        for i in range(n):
+            lg = oracle.mlp_deep_logits(w, z[:, i])
+            assert ab[i] == int(lg[1] > lg[0])
+        z = r["trajectory"][t]
+    assert np.all(np.isfinite(r["min_gap"])) and 0 < unpack_bits(r["action_bits"], n).mean() < 1
+
+
 def test_per_env_linear_policies(oracle):
     n, T, seed = 70, 40, 2
     kind = inputs.POLICY_LINEAR_PER_ENV
