@@ -521,14 +521,16 @@ def measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args) -> dict:
     n, T = w5.n_envs, w5.T
     outs = {"ep_return_sum": torch.empty(n, device="cuda"), "ep_count": torch.empty(n, dtype=torch.int32, device="cuda"),
             "totals": torch.zeros(2, dtype=torch.int64, device="cuda")}
-    for key, kind in (("c5_rollout_mlp32", inputs.POLICY_MLP32), ("c5_rollout_mlp64", inputs.POLICY_MLP64)):
-        pol = cp.policy(kind, inputs.policy_weights(kind, 3))
+    for key, kind in (("c5_rollout_mlp32", inputs.POLICY_MLP32), ("c5_rollout_mlp64", inputs.POLICY_MLP64),
+                      ("c5_rollout_mlp_deep_16_16", inputs.POLICY_MLP_DEEP)):
+        # weight draws for which the network uses both actions (3; 7 for the deep one)
+        pol = cp.policy(kind, inputs.policy_weights(kind, 7 if kind == inputs.POLICY_MLP_DEEP else 3))
 
         def fn():
             cp.cp_rollout(n, T, w5.seed, pol, **outs)
         ms, _ = timed(fn, 2, 3)
         ms /= 2
-        out[key] = {"n_envs": n, "T": T, "hidden": inputs.HIDDEN_OF[kind], "ms_per_launch": ms,
+        out[key] = {"n_envs": n, "T": T, "hidden": inputs.HIDDEN_OF.get(kind, "16+16"), "ms_per_launch": ms,
                     "env_steps_per_sec": n * T / (ms * 1e-3)}
     # config 5 itself in the contracted arithmetic (FMA dynamics and the five-instruction tanh)
     pol = cp.policy(w5.policy, inputs.policy_weights(w5.policy, w5.policy_seed))

@@ -89,6 +89,7 @@ extern "C" {
                                       floats, parameter q of env i at weights[q * n_envs + i], rows
                                       0-7 the 2x4 matrix row-major, rows 8-9 the biases; loaded into
                                       registers once per launch */
+#define CP_POLICY_MLP_DEEP 7 /* two hidden layers, 4 -> 16 (tanh) -> 16 (tanh) -> 2 (386 floats) */
 #define CP_MAX_T (1LL << 30)
 
 /* Opaque HOST handle of a batch: n_envs, plane_stride, seed, global step t,
@@ -100,6 +101,7 @@ typedef struct cp_state cp_state;
  * weights is a HOST pointer, copied into the launch parameters by the call:
  *   linear: W[2][4] row-major, b[2]                         (10 floats)
  *   MLP:    W1[H][4], b1[H], W2[2][H], b2[2], H = 16 / 32 / 64   (7H + 2 = 114 / 226 / 450 floats)
+ *   deep:   W1[16][4], b1[16], W2[16][16], b2[16], W3[2][16], b3[2]   (386 floats)
  * Each logit is a left-to-right chain acc = fmaf(w_i, v_i, acc) starting from the
  * bias; hidden units use accurate tanhf; action = (logit[1] > logit[0]), so a tie
  * pushes left. */

@@ -19,8 +19,9 @@ LIB_PATH = os.environ.get("CARTPOLE_LIB") or os.path.join(_HERE, "libcartpole.so
 CP_OK, CP_EINVAL, CP_ECUDA, CP_ENOMEM = 0, -1, -2, -3
 CP_POLICY_RANDOM, CP_POLICY_LINEAR, CP_POLICY_MLP, CP_POLICY_MLP32, CP_POLICY_MLP64 = 0, 1, 2, 4, 5
 CP_POLICY_LINEAR_PER_ENV = 6
+CP_POLICY_MLP_DEEP = 7
 N_WEIGHTS = {CP_POLICY_RANDOM: 0, CP_POLICY_LINEAR: 10, CP_POLICY_MLP: 114, CP_POLICY_MLP32: 226,
-             CP_POLICY_MLP64: 450}
+             CP_POLICY_MLP64: 450, CP_POLICY_MLP_DEEP: 386}
 
 # every symbol include/cartpole.h declares
 EXPORTS = [

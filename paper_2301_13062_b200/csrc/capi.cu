@@ -77,7 +77,8 @@ int check_state(const cp_state *s, const char *name) {
 int check_policy(const cp_policy *policy, int *kind) {
     *kind = policy ? policy->kind : CP_POLICY_RANDOM;
     if (*kind != CP_POLICY_RANDOM && *kind != CP_POLICY_LINEAR && *kind != CP_POLICY_MLP &&
-        *kind != CP_POLICY_MLP32 && *kind != CP_POLICY_MLP64 && *kind != CP_POLICY_LINEAR_PER_ENV)
+        *kind != CP_POLICY_MLP32 && *kind != CP_POLICY_MLP64 && *kind != CP_POLICY_LINEAR_PER_ENV &&
+        *kind != CP_POLICY_MLP_DEEP)
         return fail(CP_EINVAL, "unknown policy kind %d", *kind);
     if (*kind != CP_POLICY_RANDOM && !policy->weights) return fail(CP_EINVAL, "policy weights are NULL");
     if (*kind == CP_POLICY_LINEAR_PER_ENV && !is_aligned(policy->weights, 4))
@@ -166,6 +167,7 @@ int rollout_impl(uint32_t env_offset, int64_t n_envs, int64_t T, uint32_t seed, 
     if (kind == CP_POLICY_MLP) memcpy(p.w, policy->weights, 114 * sizeof(float));
     if (kind == CP_POLICY_MLP32) memcpy(p.w, policy->weights, 226 * sizeof(float));
     if (kind == CP_POLICY_MLP64) memcpy(p.w, policy->weights, 450 * sizeof(float));
+    if (kind == CP_POLICY_MLP_DEEP) memcpy(p.w, policy->weights, 386 * sizeof(float));
     if (kind == CP_POLICY_LINEAR_PER_ENV) p.env_weights = policy->weights;  // DEVICE [10][n_envs]
     const bool streams = p.reward_stream || p.done_bits || p.action_bits || p.trajectory;
     cudaError_t e = cp::launch_rollout(p, kind, streams, arithmetic == CP_ARITH_CONTRACTED, tl_stream);

@@ -392,4 +392,37 @@ __device__ __forceinline__ uint32_t mlp_action(const MlpWT<H> &p, const State &z
     return (l1 > l0) ? 0x80000000u : 0u;
 }
 
+// Two hidden layers, 4 -> 16 (tanh) -> 16 (tanh) -> 2. The sixteen first-layer activations stay
+// in registers; second-layer units are consumed by the two logit chains as they are produced
+// (ascending unit order, the chains start from the biases: the order of the definition).
+struct MlpDeepW {
+    float w1[16][4], b1[16];
+    float w2[16][16], b2[16];
+    float w3[2][16], b3[2];
+};
+template <bool FAST_TANH = false>
+__device__ __forceinline__ uint32_t mlp_deep_action(const MlpDeepW &p, const State &z) {
+    float h1[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        float acc = p.b1[j];
+        acc = __fmaf_rn(p.w1[j][0], z.x, acc);
+        acc = __fmaf_rn(p.w1[j][1], z.xd, acc);
+        acc = __fmaf_rn(p.w1[j][2], z.th, acc);
+        acc = __fmaf_rn(p.w1[j][3], z.thd, acc);
+        h1[j] = FAST_TANH ? tanh_contracted(acc) : tanhf(acc);
+    }
+    float l0 = p.b3[0], l1 = p.b3[1];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+        float acc = p.b2[k];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) acc = __fmaf_rn(p.w2[k][j], h1[j], acc);
+        const float h2 = FAST_TANH ? tanh_contracted(acc) : tanhf(acc);
+        l0 = __fmaf_rn(p.w3[0][k], h2, l0);
+        l1 = __fmaf_rn(p.w3[1][k], h2, l1);
+    }
+    return (l1 > l0) ? 0x80000000u : 0u;
+}
+
 }  // namespace cp

@@ -26,7 +26,8 @@ namespace cp {
 
 // POLICY: 0 hashed random action, 1 linear, 2 MLP with 16 hidden units, 3 action bits supplied by
 // the caller, 4 / 5 MLP with 32 / 64 hidden units, 6 one linear policy per environment (its ten
-// parameters are loaded into registers before the time loop; handled in the kernel body).
+// parameters are loaded into registers before the time loop; handled in the kernel body), 7 MLP
+// with two hidden layers of 16 units.
 template <int POLICY, bool CONTRACT>
 __device__ __forceinline__ uint32_t policy_signbit(const RolloutParams &p, const FoldedKeys &ka,
                                                    uint32_t folded_t, const State &z) {
@@ -38,6 +39,8 @@ __device__ __forceinline__ uint32_t policy_signbit(const RolloutParams &p, const
         return mlp_action<16, CONTRACT>(*reinterpret_cast<const MlpWT<16> *>(p.w), z);
     } else if (POLICY == 4) {
         return mlp_action<32, CONTRACT>(*reinterpret_cast<const MlpWT<32> *>(p.w), z);
+    } else if (POLICY == 7) {
+        return mlp_deep_action<CONTRACT>(*reinterpret_cast<const MlpDeepW *>(p.w), z);
     } else {
         return mlp_action<64, CONTRACT>(*reinterpret_cast<const MlpWT<64> *>(p.w), z);
     }
@@ -395,7 +398,7 @@ cudaError_t launch_rollout_arith(RolloutParams &p, int policy, bool streams, cud
     // Per-environment linear policies keep ten weights per env in registers: 89 registers with
     // two envs per thread, 63 with one, which is 8 % faster.
     const bool small = (p.n + 63) / 64 < (int64_t)sm_count() * 16;
-    const bool heavy = policy == 2 || policy == 4 || policy == 5 || policy == 6;
+    const bool heavy = policy == 2 || policy == 4 || policy == 5 || policy == 6 || policy == 7;
     int ept = g_tuning.rollout_ept;      // 0 auto, 1, 2
     int coop = g_tuning.rollout_coop;    // 0 auto, 1 cooperative, 2 per lane, 3 per lane and ahead
     if (ept == 0) ept = (small || heavy || coop >= 2) ? 1 : 2;
@@ -415,6 +418,7 @@ cudaError_t launch_rollout_arith(RolloutParams &p, int policy, bool streams, cud
         case 3: return launch_mode<3, CONTRACT>(p, mode, shape, s);
         case 4: return launch_mode<4, CONTRACT>(p, mode, shape, s);
         case 5: return launch_mode<5, CONTRACT>(p, mode, shape, s);
+        case 7: return launch_mode<7, CONTRACT>(p, mode, shape, s);
         default: return launch_mode<6, CONTRACT>(p, mode, shape, s);
     }
 }

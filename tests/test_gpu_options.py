@@ -230,10 +230,11 @@ def test_general_call_argument_checks(cp):
     assert cp.cp_launch_count() == before
 
 
-@pytest.mark.parametrize("kind", [inputs.POLICY_MLP32, inputs.POLICY_MLP64])
-def test_wider_mlp_policies_against_oracle(cp, oracle, kind):
+@pytest.mark.parametrize("kind,pseed", [(inputs.POLICY_MLP32, 3), (inputs.POLICY_MLP64, 3), (inputs.POLICY_MLP_DEEP, 7),
+                                        (inputs.POLICY_MLP_DEEP, 11)])
+def test_wider_and_deeper_mlp_policies_against_oracle(cp, oracle, kind, pseed):
     n, T, seed = 20000, 150, 1
-    w = inputs.policy_weights(kind, 3)  # a draw for which both networks use both actions
+    w = inputs.policy_weights(kind, pseed)  # draws for which the networks use both actions
     out = outputs(n, T)
     cp.cp_rollout(n, T, seed, cp.policy(kind, w), **out)
     r = fetch(out)
