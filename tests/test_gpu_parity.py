@@ -484,6 +484,25 @@ def test_work_shapes_agree_bitwise_and_survive_mass_termination(cp):
             assert np.all(results[0]["ep_count"] == T) and np.all(results[0]["ep_return_sum"] == T)
 
 
+def test_launch_geometry_does_not_change_results(cp):
+    """Persistent grids (warps looping over several tasks, re-using their shared-memory restart
+    list), small CTAs and every work shape give the bits of the default launch."""
+    n, T = 70001, 45
+    want = run_rollout(cp, n, T, 7, streams=True)
+    try:
+        for per_sm, block in ((1, 256), (2, 64), (1, 32), (0, 96)):
+            cp.cp_tune("rollout_ctas_per_sm", per_sm)
+            cp.cp_tune("rollout_block", block)
+            for shape in H.SHAPES:
+                with H.rollout_shape(cp, *shape):
+                    got = run_rollout(cp, n, T, 7, streams=True)
+                for k in want:
+                    assert np.array_equal(want[k], got[k]), (k, per_sm, block, shape)
+    finally:
+        cp.cp_tune("rollout_ctas_per_sm", 0)
+        cp.cp_tune("rollout_block", 0)
+
+
 def test_shards_compose(cp):
     n, T = 10000, 80
     whole = run_rollout(cp, n, T, 3)
