@@ -372,6 +372,9 @@ typedef struct {
     float *min_gap;          /* [n] or NULL: smallest |logit1-logit0| seen */
     uint32_t max_steps;      /* episode step limit (CartPole-v1 uses 500); 0 = none */
     const uint32_t *action_bits_in; /* [T][ceil(n/32)] supplied actions (bit i%32 of word i/32) or NULL */
+    const float *start_states_in;   /* [T][4][n] supplied start states or NULL: an env that finishes at
+                                       the k-th step of this call continues from row k (the paper's
+                                       baseline feeds all its random values as data, Sec. V-A) */
     int64_t lo, hi;          /* env sub-range handled by this worker */
     uint64_t tot_ret, tot_cnt;
 } co_rollout_job;
@@ -421,7 +424,11 @@ static void co_rollout_range(co_rollout_job *J)
                 ret_sum += ep_len;
                 ep_cnt += 1u;
                 ep_len = 0u;
-                co_reset_state(J->seed, env, t + 1u, zn);
+                if (J->start_states_in)
+                    for (int p = 0; p < 4; ++p)
+                        zn[p] = J->start_states_in[(k * 4 + p) * n + i];
+                else
+                    co_reset_state(J->seed, env, t + 1u, zn);
             }
             memcpy(z, zn, sizeof z);
             if (J->reward_stream) J->reward_stream[k * n + i] = 1.0f;
@@ -458,7 +465,8 @@ void co_rollout_ex(uint32_t env_offset, int64_t n, int64_t T, uint32_t seed, uin
                    const float *weights, const float *init_state, uint32_t *ep_len_io,
                    float *ep_return_sum, uint32_t *ep_count, uint64_t *totals, float *reward_stream,
                    uint32_t *done_bits, uint32_t *action_bits, float *final_state, float *trajectory,
-                   float *min_gap, int nthreads, uint32_t max_steps, const uint32_t *action_bits_in)
+                   float *min_gap, int nthreads, uint32_t max_steps, const uint32_t *action_bits_in,
+                   const float *start_states_in)
 {
     if (nthreads < 1) nthreads = 1;
     if (nthreads > 256) nthreads = 256;
@@ -473,7 +481,8 @@ void co_rollout_ex(uint32_t env_offset, int64_t n, int64_t T, uint32_t seed, uin
         if (hi > n) hi = n;
         co_rollout_job J = {env_offset, n, T, seed, t0, kind, weights, init_state, ep_len_io,
                             ep_return_sum, ep_count, reward_stream, done_bits, action_bits,
-                            final_state, trajectory, min_gap, max_steps, action_bits_in, lo, hi, 0, 0};
+                            final_state, trajectory, min_gap, max_steps, action_bits_in, start_states_in,
+                            lo, hi, 0, 0};
         jobs[used++] = J;
     }
     if (used == 1) {
@@ -500,7 +509,7 @@ void co_rollout(uint32_t env_offset, int64_t n, int64_t T, uint32_t seed, uint32
 {
     co_rollout_ex(env_offset, n, T, seed, t0, kind, weights, init_state, ep_len_io, ep_return_sum, ep_count,
                   totals, reward_stream, done_bits, action_bits, final_state, trajectory, min_gap, nthreads,
-                  0u, NULL);
+                  0u, NULL, NULL);
 }
 
 /* co_step with an episode step limit: ep_len [n] holds the steps already taken in each

@@ -83,7 +83,7 @@ def lib() -> C.CDLL:
         L.co_rollout.restype = None
         L.co_rollout.argtypes = [u32, i64, i64, u32, u32, i32, p, p, p, p, p, p, p, p, p, p, p, p, i32]
         L.co_rollout_ex.restype = None
-        L.co_rollout_ex.argtypes = [u32, i64, i64, u32, u32, i32, p, p, p, p, p, p, p, p, p, p, p, p, i32, u32, p]
+        L.co_rollout_ex.argtypes = [u32, i64, i64, u32, u32, i32, p, p, p, p, p, p, p, p, p, p, p, p, i32, u32, p, p]
         L.co_step_limited.restype = None
         L.co_step_limited.argtypes = [u32, i64, i64, i64, u32, u32, p, p, p, p, p, p, u32]
         _lib = L
@@ -221,11 +221,13 @@ def rollout(n: int, T: int, seed: int, policy_kind: int = POLICY_RANDOM, weights
             reward_stream: bool = False, done_bits: bool = False,
             action_bits: bool = False, final_state: bool = False, trajectory: bool = False,
             min_gap: bool = False, nthreads: int = 1, max_episode_steps: int = 0,
-            action_bits_in: np.ndarray | None = None) -> dict:
+            action_bits_in: np.ndarray | None = None, start_states_in: np.ndarray | None = None) -> dict:
     """Rollout of n envs for T steps. Returns a dict of the requested outputs.
 
     max_episode_steps > 0 cuts episodes off at that length; action_bits_in ([T, ceil(n/32)]
-    uint32, bit i%32 of word i//32) supplies the actions instead of the policy."""
+    uint32, bit i%32 of word i//32) supplies the actions instead of the policy;
+    start_states_in (float32 [T, 4, n]) supplies the start states: an env that finishes at the
+    k-th step of the call continues from row k instead of the hashed start state."""
     w = None
     if policy_kind != POLICY_RANDOM:
         w = np.ascontiguousarray(weights, np.float32).ravel()
@@ -253,11 +255,14 @@ def rollout(n: int, T: int, seed: int, policy_kind: int = POLICY_RANDOM, weights
     if action_bits_in is not None:
         action_bits_in = np.ascontiguousarray(action_bits_in).view(np.uint32)
         assert action_bits_in.shape == (T, words)
+    if start_states_in is not None:
+        start_states_in = np.ascontiguousarray(start_states_in, np.float32)
+        assert start_states_in.shape == (T, 4, n)
     lib().co_rollout_ex(env_offset, n, T, seed, t0, policy_kind, _ptr(w), _ptr(init_state), _ptr(ep_len),
                         _ptr(res["ep_return_sum"]), _ptr(res["ep_count"]), _ptr(res["totals"]),
                         _ptr(res["reward_stream"]), _ptr(res["done_bits"]), _ptr(res["action_bits"]),
                         _ptr(res["final_state"]), _ptr(res["trajectory"]), _ptr(res["min_gap"]),
-                        int(nthreads), int(max_episode_steps), _ptr(action_bits_in))
+                        int(nthreads), int(max_episode_steps), _ptr(action_bits_in), _ptr(start_states_in))
     return res
 
 

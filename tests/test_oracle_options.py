@@ -150,6 +150,45 @@ def test_supplied_action_stream(oracle):
     assert np.all((first >= 6) & (first <= 12))
 
 
+def test_supplied_start_states(oracle):
+    """All randomness as data (the paper's baseline, Sec. V-A): start states read from an array."""
+    n, T, seed, off = 37, 60, 3, 500
+    # (1) feeding the hashed start states of times t0+1 .. t0+T back in reproduces the hashed rollout
+    t0 = 11
+    pool = np.stack([oracle.initial_state(n, seed, t0 + k + 1, off) for k in range(T)])
+    h = oracle.rollout(n, T, seed, env_offset=off, t0=t0, trajectory=True, done_bits=True)
+    g = oracle.rollout(n, T, seed, env_offset=off, t0=t0, start_states_in=pool, trajectory=True, done_bits=True)
+    for k in ("ep_return_sum", "ep_count", "trajectory", "done_bits", "totals"):
+        assert np.array_equal(h[k], g[k]), k
+    # (2) arbitrary supplied states: after every done the state is exactly row k of the array, and
+    # between restarts the trajectory is the one-step dynamics (brute force with co_step's pieces)
+    rng = np.random.default_rng(4)
+    pool = (0.05 * rng.uniform(-1, 1, (T, 4, n))).astype(np.float32)
+    pool[:, 2, ::3] = np.float32(0.2)      # some start states sit right at the edge: very short episodes
+    acts = rng.integers(0, 2, (T, n)).astype(np.uint8)
+    r = oracle.rollout(n, T, seed, action_bits_in=pack_bits(acts), start_states_in=pool, trajectory=True,
+                       done_bits=True)
+    done = unpack_bits(r["done_bits"], n)
+    z = oracle.initial_state(n, seed)
+    ep_len = np.zeros(n, np.int64)
+    ret = np.zeros(n, np.int64)
+    cnt = np.zeros(n, np.int64)
+    for k in range(T):
+        for i in range(n):
+            zn, d = oracle.dynamics_f32(z[:, i], int(acts[k, i]))
+            ep_len[i] += 1
+            assert int(d) == done[k, i]
+            if d:
+                ret[i] += ep_len[i]
+                cnt[i] += 1
+                ep_len[i] = 0
+                zn = pool[k, :, i]
+            assert np.array_equal(np.asarray(zn, np.float32).view(np.uint32), r["trajectory"][k, :, i].view(np.uint32))
+            z[:, i] = zn
+    assert np.array_equal(r["ep_return_sum"], ret.astype(np.float32)) and np.array_equal(r["ep_count"], cnt.astype(np.uint32))
+    assert cnt[::3].min() >= 3 and done.sum() > 0
+
+
 @pytest.mark.parametrize("kind,hidden", [(inputs.POLICY_MLP32, 32), (inputs.POLICY_MLP64, 64)])
 def test_wider_mlp_policies(oracle, kind, hidden):
     w = inputs.policy_weights(kind, 7)
