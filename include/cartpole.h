@@ -219,6 +219,11 @@ int cp_rollout_from(cp_state *state, int64_t T, uint32_t *ep_len, const cp_polic
  *   - actions given as data instead of drawn by a policy (the paper's baseline, Sec. V-A, feeds
  *     precomputed random values): action_bits_in DEVICE [T][ceil(n_envs/32)], bit (i%32) of word
  *     (i/32) of row k = action of env i at the k-th step of this call; overrides `policy`;
+ *   - start states given as data too (the other half of that baseline's randomness; also the way
+ *     to evaluate a policy from chosen start states): start_states_in DEVICE [T][4][n_envs], an
+ *     environment that finishes at the k-th step of this call continues from row k (planes x,
+ *     x_dot, theta, theta_dot) instead of the hashed start state. The first states still come
+ *     from `state`, or from the hash of time t0;
  *   - a choice of arithmetic. CP_ARITH_EXACT (0, what every other entry point uses): each operation
  *     of the step rounded once, in the order of the per-op ladder, so that ladder, fused step and
  *     rollout give the same bits. CP_ARITH_CONTRACTED: the step as a contracting compiler would
@@ -254,6 +259,7 @@ typedef struct cp_rollout_args {
     uint32_t max_episode_steps;    /* 0 = no limit */
     uint32_t arithmetic;           /* CP_ARITH_EXACT or CP_ARITH_CONTRACTED */
     const uint32_t *action_bits_in; /* DEVICE or NULL */
+    const float *start_states_in;   /* DEVICE or NULL */
 } cp_rollout_args;
 int cp_rollout_ex(const cp_rollout_args *args);
 

@@ -48,7 +48,8 @@ class cp_rollout_args(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("env_offset", C.c_uint32), ("n_envs", C.c_int64), ("T", C.c_int64),
                 ("seed", C.c_uint32), ("t0", C.c_uint32), ("policy", C.POINTER(cp_policy)),
                 ("returns", C.POINTER(cp_returns)), ("state", C.c_void_p), ("ep_len", C.c_void_p),
-                ("max_episode_steps", C.c_uint32), ("arithmetic", C.c_uint32), ("action_bits_in", C.c_void_p)]
+                ("max_episode_steps", C.c_uint32), ("arithmetic", C.c_uint32), ("action_bits_in", C.c_void_p),
+                ("start_states_in", C.c_void_p)]
 
 
 CP_ARITH_EXACT, CP_ARITH_CONTRACTED = 0, 1
@@ -334,10 +335,10 @@ def cp_rollout_from(state: State, T: int, ep_len=None, policy: _Policy | None = 
 def cp_rollout_ex(*, n_envs: int = 0, T: int, seed: int = 0, t0: int = 0, env_offset: int = 0,
                   policy: _Policy | None = None, state: State | None = None, ep_len=None,
                   max_episode_steps: int = 0, action_bits_in=None, arithmetic: int = CP_ARITH_EXACT,
-                  **returns) -> None:
-    """General rollout: optional episode step limit, optional supplied action bit stream, choice
-    of arithmetic, either from start states (n_envs, seed, t0, env_offset) or advancing `state`
-    in place."""
+                  start_states_in=None, **returns) -> None:
+    """General rollout: optional episode step limit, optional supplied action bit stream and
+    start states ([T, 4, n] float32), choice of arithmetic, either from start states (n_envs,
+    seed, t0, env_offset) or advancing `state` in place."""
     import torch
     _use_current_stream()
     r = _returns_struct(**returns)
@@ -351,6 +352,10 @@ def cp_rollout_ex(*, n_envs: int = 0, T: int, seed: int = 0, t0: int = 0, env_of
     a.max_episode_steps = max_episode_steps
     a.arithmetic = arithmetic
     a.action_bits_in = _dptr(action_bits_in, torch.int32)
+    if start_states_in is not None:
+        n = state.info()["n_envs"] if state is not None else n_envs
+        assert tuple(start_states_in.shape) == (T, 4, n), "start_states_in must be [T, 4, n_envs]"
+    a.start_states_in = _dptr(start_states_in, torch.float32)
     _check(lib().cp_rollout_ex(C.byref(a)))
 
 

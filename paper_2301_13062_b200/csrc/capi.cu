@@ -131,8 +131,10 @@ void advance(cp_state *state, cp_state *out_state, uint32_t steps) {
 int rollout_impl(uint32_t env_offset, int64_t n_envs, int64_t T, uint32_t seed, uint32_t t0, const cp_policy *policy,
                  const cp_returns *ret, const float *init_planes, int64_t init_stride, float *out_planes,
                  int64_t out_stride, uint32_t *ep_len, uint32_t max_steps = 0,
-                 const uint32_t *action_bits_in = nullptr, uint32_t arithmetic = CP_ARITH_EXACT) {
+                 const uint32_t *action_bits_in = nullptr, uint32_t arithmetic = CP_ARITH_EXACT,
+                 const float *start_states_in = nullptr) {
     int kind, rc;
+    if (start_states_in && !is_aligned(start_states_in, 4)) return fail(CP_EINVAL, "start_states_in is misaligned");
     if (arithmetic != CP_ARITH_EXACT && arithmetic != CP_ARITH_CONTRACTED)
         return fail(CP_EINVAL, "arithmetic must be CP_ARITH_EXACT or CP_ARITH_CONTRACTED (got %u)", arithmetic);
     if ((rc = check_range(n_envs, env_offset)) != CP_OK) return rc;
@@ -163,6 +165,7 @@ int rollout_impl(uint32_t env_offset, int64_t n_envs, int64_t T, uint32_t seed, 
     p.trajectory = ret->trajectory;
     p.max_steps = max_steps;
     p.action_bits_in = action_bits_in;
+    p.start_in = start_states_in;
     if (kind == CP_POLICY_LINEAR) memcpy(p.w, policy->weights, 10 * sizeof(float));
     if (kind == CP_POLICY_MLP) memcpy(p.w, policy->weights, 114 * sizeof(float));
     if (kind == CP_POLICY_MLP32) memcpy(p.w, policy->weights, 226 * sizeof(float));
@@ -456,14 +459,15 @@ int cp_rollout_ex(const cp_rollout_args *a) {
         if (rc != CP_OK) return rc;
         cp_state *st = a->state;
         rc = rollout_impl(st->env_offset, st->n, a->T, st->seed, st->t, a->policy, a->returns, st->planes, st->stride,
-                          st->planes, st->stride, a->ep_len, a->max_episode_steps, a->action_bits_in, a->arithmetic);
+                          st->planes, st->stride, a->ep_len, a->max_episode_steps, a->action_bits_in, a->arithmetic,
+                          a->start_states_in);
         if (rc != CP_OK) return rc;
         st->t += (uint32_t)a->T;
         return CP_OK;
     }
     return rollout_impl(a->env_offset, a->n_envs, a->T, a->seed, a->t0, a->policy, a->returns, nullptr, 0,
                         a->returns->final_state, a->n_envs, a->ep_len, a->max_episode_steps, a->action_bits_in,
-                        a->arithmetic);
+                        a->arithmetic, a->start_states_in);
 }
 
 int cp_rollout_host(int64_t n_envs, int64_t T, uint32_t seed, const cp_policy *policy, float *h_ep_return_sum,

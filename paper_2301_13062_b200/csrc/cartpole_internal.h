@@ -43,6 +43,7 @@ struct RolloutParams {
     float *trajectory;
     uint32_t max_steps;              // episode step limit, 0 = none
     const uint32_t *action_bits_in;  // [T][words] supplied actions or nullptr
+    const float *start_in;           // [T][4][n] supplied start states or nullptr
     const float *env_weights;        // [10][n] one linear policy per env (policy kind 6) or nullptr
     float w[450];  // largest policy: MLP with 64 hidden units, 7*64 + 2 floats
 };

@@ -195,7 +195,17 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
                 if (!COOP && done[j]) {
                     cnt[j] += 1u;
                     begin[j] = t1;
-                    z[j] = AHEAD ? fresh : start_state_folded(kr[j], folded_4t1);
+                    if (AHEAD) {
+                        z[j] = fresh;
+                    } else if (p.start_in) {  // start states supplied as data: row (t - t0) of [T][4][n]
+                        const float *row = p.start_in + (int64_t)(t - p.t0) * 4 * p.n + idx[j];
+                        z[j].x = __ldg(row);
+                        z[j].xd = __ldg(row + p.n);
+                        z[j].th = __ldg(row + 2 * p.n);
+                        z[j].thd = __ldg(row + 3 * p.n);
+                    } else {
+                        z[j] = start_state_folded(kr[j], folded_4t1);
+                    }
                 }
             }
 
@@ -407,8 +417,9 @@ cudaError_t launch_rollout_arith(RolloutParams &p, int policy, bool streams, cud
     // and with the linear policy, whose episodes are long)
     const bool tiny = (p.n + 31) / 32 <= (int64_t)sm_count() * 4 * 2;
     if (coop == 0) coop = (small && ept == 1) ? ((tiny && (policy == 0 || policy == 3)) ? 3 : 2) : 1;
-    // two envs per thread are always cooperative
-    const int shape = ept == 2 ? 2 : (coop == 2 ? 0 : coop == 3 ? 3 : 1);
+    // two envs per thread are always cooperative; supplied start states are read by the lane that
+    // needs them, so they always take the plain per-lane shape
+    const int shape = p.start_in ? 0 : ept == 2 ? 2 : (coop == 2 ? 0 : coop == 3 ? 3 : 1);
     // 0: no per-step output; 1: reward plane + done bitmask only; 2: any other combination
     const int mode = !streams ? 0 : (p.reward_stream && p.done_bits && !p.action_bits && !p.trajectory) ? 1 : 2;
     switch (policy) {

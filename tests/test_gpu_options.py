@@ -316,3 +316,49 @@ def test_reset_through_the_host_program_allocator(cp, oracle):
         cp.cp_free(st2)
     finally:
         cp.use_torch_allocator(False)
+
+
+def test_supplied_start_states(cp, oracle):
+    """Start states read from a caller's [T][4][n] array instead of the hash."""
+    n, T, seed, off, t0 = 5003, 90, 3, 70, 11
+    # (1) GPU-internal: the hashed start states fed back as data reproduce the hashed rollout
+    pool = torch.zeros(T, 4, n, device="cuda")
+    for k in range(T):
+        st = cp.cp_wrap(pool[k], n, seed, t0 + k + 1, off)
+        cp.cp_fill_start(st)
+    a, b = outputs(n, T), outputs(n, T)
+    cp.cp_rollout_ex(n_envs=n, T=T, seed=seed, env_offset=off, t0=t0, **a)
+    cp.cp_rollout_ex(n_envs=n, T=T, seed=seed, env_offset=off, t0=t0, start_states_in=pool, **b)
+    ra, rb = fetch(a), fetch(b)
+    for k in ra:
+        assert np.array_equal(ra[k], rb[k]), k
+    # (2) against the oracle: arbitrary start states (some at the edge: very short episodes),
+    # with supplied actions (all randomness as data), the hashed actions, and a linear policy
+    rng = np.random.default_rng(5)
+    states = (0.05 * rng.uniform(-1, 1, (T, 4, n))).astype(np.float32)
+    states[:, 2, ::3] = np.float32(0.2)
+    d_states = torch.from_numpy(states).cuda()
+    acts = rng.integers(0, 2, (T, n)).astype(np.uint8)
+    d_bits = torch.from_numpy(pack_bits(acts).view(np.int32)).cuda()
+    w = inputs.policy_weights(1, 4)
+    for gpu_kw, ora_kw, kind, wts in (({"action_bits_in": d_bits}, {"action_bits_in": pack_bits(acts)}, 0, None),
+                                      ({}, {}, 0, None), ({}, {}, 1, w)):
+        out = outputs(n, T)
+        cp.cp_rollout_ex(n_envs=n, T=T, seed=seed, env_offset=off, start_states_in=d_states,
+                         policy=cp.policy(kind, wts) if kind else None, **gpu_kw, **out)
+        r = fetch(out)
+        o = oracle.rollout(n, T, seed, kind, wts, env_offset=off, start_states_in=states, done_bits=True,
+                           min_gap=True, nthreads=4, **ora_kw)
+        H.assert_returns_match(r["ep_return_sum"], r["ep_count"], o["ep_return_sum"], o["ep_count"],
+                               o["min_gap"] < 1e-5)
+        same = r["ep_return_sum"] == o["ep_return_sum"]
+        assert np.array_equal(H.unpack_bits(r["done_bits"], n)[:, same], H.unpack_bits(o["done_bits"], n)[:, same])
+        assert r["ep_count"].sum() > n and (kind or np.median(r["ep_count"][::3]) >= 3)
+    # (3) the contracted arithmetic and chunked calls on a batch take the option too
+    st = cp.cp_reset(n, seed)
+    ret = torch.empty(n, device="cuda")
+    cp.cp_rollout_ex(state=st, T=T, start_states_in=d_states, arithmetic=cp.CP_ARITH_CONTRACTED, ep_return_sum=ret)
+    torch.cuda.synchronize()
+    assert st.info()["t"] == T and float(ret.sum()) > 0
+    with pytest.raises(AssertionError):
+        cp.cp_rollout_ex(n_envs=n, T=T - 1, seed=seed, start_states_in=d_states, ep_return_sum=ret)
