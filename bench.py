@@ -513,7 +513,19 @@ def measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args) -> dict:
     ms /= 10
     out["c3_rollout_per_env_linear"] = {"n_envs": n, "T": T, "ms_per_launch": ms,
                                         "env_steps_per_sec": n * T / (ms * 1e-3)}
-    del outs, act, pop
+    # every random value as data, as in the paper's baseline (Sec. V-A): the action bits of above
+    # and the start states (here the hashed ones of each time step: [T][4][n] floats = 8.4 GB)
+    starts = torch.empty(T, 4, n, device="cuda")
+    for k in range(T):
+        cp.cp_fill_start(cp.cp_wrap(starts[k], n, w3.seed, k + 1))
+
+    def data_fn():
+        cp.cp_rollout_ex(n_envs=n, T=T, seed=w3.seed, action_bits_in=act, start_states_in=starts, **outs)
+    ms, _ = timed(data_fn, 10, 3)
+    ms /= 10
+    out["c3_rollout_all_randomness_supplied"] = {"n_envs": n, "T": T, "ms_per_launch": ms,
+                                                 "env_steps_per_sec": n * T / (ms * 1e-3)}
+    del outs, act, pop, starts
     torch.cuda.empty_cache()
 
     # wider in-kernel policies on config 5's shape (16,777,216 envs x 200 steps)
