@@ -287,12 +287,14 @@ def main() -> None:
                    "counts land in pinned host memory (stored there by the kernel over PCIe while it runs), "
                    "totals copied back, stream synchronised, every step"}
 
+    # side measurements and the CPU baseline belong to the one-GPU run (under torchrun they would
+    # only keep the other ranks waiting in the final reduction)
     paths = {}
-    if not args.no_paths and rank == 0:
+    if not args.no_paths and world == 1:
         paths = measure_paths(cp, inputs, torch, lambda *a, **k: timed(*a, all_ranks=False, **k), peaks, peak_inst, args)
 
     cpu = None
-    if not args.no_cpu and rank == 0:
+    if not args.no_cpu and world == 1:
         from oracle import cartpole_oracle as oracle
         cores = min(host_cores(), 256)
         sample = min(n, 1 << 20)
