@@ -75,6 +75,10 @@ cudaError_t launch_actions(uint8_t *out, int64_t n, uint32_t env_offset, uint32_
                            cudaStream_t s);
 cudaError_t launch_rollout(RolloutParams &p, int policy, bool streams, bool contracted, cudaStream_t s);
 cudaError_t launch_rollout_contracted(RolloutParams &p, int policy, bool streams, cudaStream_t s);
+// the MLP policies (kinds 2, 4, 5, 7), canonical and contracted arithmetic; mode and shape as
+// chosen by launch_rollout_arith
+cudaError_t launch_rollout_networks(RolloutParams &p, int policy, int mode, int shape, cudaStream_t s);
+cudaError_t launch_rollout_networks_contracted(RolloutParams &p, int policy, int mode, int shape, cudaStream_t s);
 cudaError_t launch_sincos_selftest(uint32_t lo_bits, uint32_t hi_bits, unsigned long long *mismatches,
                                    cudaStream_t s);
 

@@ -427,15 +427,25 @@ cudaError_t launch_rollout_arith(RolloutParams &p, int policy, bool streams, cud
     const int shape = p.start_in ? 0 : ept == 2 ? 2 : (coop == 2 ? 0 : coop == 3 ? 3 : 1);
     // 0: no per-step output; 1: reward plane + done bitmask only; 2: any other combination
     const int mode = !streams ? 0 : (p.reward_stream && p.done_bits && !p.action_bits && !p.trajectory) ? 1 : 2;
+    // the network policies are instantiated in translation units of their own (build time)
+    if (policy == 2 || policy == 4 || policy == 5 || policy == 7)
+        return CONTRACT ? launch_rollout_networks_contracted(p, policy, mode, shape, s)
+                        : launch_rollout_networks(p, policy, mode, shape, s);
     switch (policy) {
         case 0: return launch_mode<0, CONTRACT>(p, mode, shape, s);
         case 1: return launch_mode<1, CONTRACT>(p, mode, shape, s);
-        case 2: return launch_mode<2, CONTRACT>(p, mode, shape, s);
         case 3: return launch_mode<3, CONTRACT>(p, mode, shape, s);
+        default: return launch_mode<6, CONTRACT>(p, mode, shape, s);
+    }
+}
+
+template <bool CONTRACT>
+cudaError_t launch_networks_arith(RolloutParams &p, int policy, int mode, int shape, cudaStream_t s) {
+    switch (policy) {
+        case 2: return launch_mode<2, CONTRACT>(p, mode, shape, s);
         case 4: return launch_mode<4, CONTRACT>(p, mode, shape, s);
         case 5: return launch_mode<5, CONTRACT>(p, mode, shape, s);
-        case 7: return launch_mode<7, CONTRACT>(p, mode, shape, s);
-        default: return launch_mode<6, CONTRACT>(p, mode, shape, s);
+        default: return launch_mode<7, CONTRACT>(p, mode, shape, s);
     }
 }
 
