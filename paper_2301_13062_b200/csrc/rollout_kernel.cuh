@@ -15,9 +15,10 @@
 // only synchronisation is __syncwarp() around a warp's own 192 bytes of shared memory in the
 // cooperative restart.
 //
-// This header holds the kernel template and its dispatch; rollout_kernel.cu instantiates it
-// for the canonical (one rounding per op) arithmetic, rollout_contracted.cu for the
-// contracted arithmetic, so that the two sets of kernels compile side by side.
+// This header holds the kernel template and its dispatch; rollout_kernel.cu and
+// rollout_networks.cu instantiate it for the canonical (one rounding per op) arithmetic,
+// rollout_contracted.cu and rollout_networks_contracted.cu for the contracted arithmetic (the
+// *_networks files hold the MLP policies), so that the kernel families compile side by side.
 #pragma once
 #include "cartpole_device.cuh"
 #include "cartpole_internal.h"
