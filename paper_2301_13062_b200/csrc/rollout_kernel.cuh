@@ -149,8 +149,10 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
             word_off[j] = task * EPT + j;
             const bool in_range = word_off[j] < words;
             word_ok[j] = lane == 0 && in_range;
-            rew_ptr[j] = STREAMS == 1 ? p.reward_stream + idx[j] : nullptr;
-            done_ptr[j] = STREAMS == 1 ? p.done_bits + (word_ok[j] ? word_off[j] : 0) : nullptr;
+            // STREAMS == 1 keeps ONE running pointer per stream: slot j's element lies a constant
+            // 32 floats / 1 word behind slot 0's (never dereferenced where the slot has no env)
+            rew_ptr[j] = STREAMS == 1 ? p.reward_stream + (base + lane) : nullptr;
+            done_ptr[j] = STREAMS == 1 ? p.done_bits + task * EPT : nullptr;
             act_ptr[j] = POLICY == 3 ? p.action_bits_in + (in_range ? word_off[j] : 0) : nullptr;
             vmask[j] = __ballot_sync(0xffffffffu, valid[j]);
         }
@@ -276,10 +278,12 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
             for (int j = 0; j < EPT; ++j) {
                 if (STREAMS == 1) {
                     const uint32_t m = COOP ? (dmask[j] & vmask[j]) : __ballot_sync(0xffffffffu, done[j] && valid[j]);
-                    if (word_ok[j]) *done_ptr[j] = m;
-                    if (valid[j]) *rew_ptr[j] = 1.0f;
-                    done_ptr[j] += words;
-                    rew_ptr[j] += p.n;
+                    if (word_ok[j]) done_ptr[0][j] = m;
+                    if (valid[j]) rew_ptr[0][32 * j] = 1.0f;
+                    if (j == EPT - 1) {
+                        done_ptr[0] += words;
+                        rew_ptr[0] += p.n;
+                    }
                 }
                 if (STREAMS == 2) {
                     if (want_done) {
