@@ -40,12 +40,12 @@ SMS = 148
 ROLLOUT_OPS = {
     "random": {"thread": 69.6, "slot": 89.8},
     "linear": {"thread": 73.8, "slot": 80.5},
-    "linear+streams": {"thread": 91.9, "slot": 95.6},
+    "linear+streams": {"thread": 91.9, "slot": 94.0},
     "mlp": {"thread": 438.3, "slot": 467.2},
     "random+contracted": {"thread": 53.6, "slot": 72.4},
 }
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch in the same captures.
-ROLLOUT_DRAM_BYTES = {"random": 24.3e3, "linear": 24.6e3, "linear+streams": 382.3e6, "mlp": 22.5e3}
+ROLLOUT_DRAM_BYTES = {"random": 24.3e3, "linear": 24.6e3, "linear+streams": 382.1e6, "mlp": 22.5e3}
 STEP_DRAM_BYTES_16M = 566.9e6  # step_kernel at 16,777,216 envs, same kind of capture
 # Algorithmic HBM bytes per env-step of the step paths.
 STEP_BYTES = 37.0      # 16 in + 16 out + 4 reward + 1 done, hashed action
