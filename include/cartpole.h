@@ -343,7 +343,9 @@ int cp_selftest_tanh(uint32_t lo_bits, uint32_t hi_bits, uint64_t *out);
  * they are used. out DEVICE [4] uint64, caller zeroes; every count must come back 0. */
 int cp_selftest_arith(uint64_t *out);
 
-/* Diagnostics: for states inside the range episodes visit (|theta| <= 0.22, |theta_dot| <= 20) the
+/* Diagnostics: for states with |theta| <= 0.22 (every angle an episode visits; such a state only
+ * survives its step if |theta_dot| < 21.5, and the accelerations of a state that does not survive
+ * are never observed) the
  * kernels compute the angular acceleration's quotient with the hardware reciprocal plus one exact
  * correction instead of the general division. This compares the two over the whole operand domain
  * of such states: every den_step-th float32 denominator in [0.6210, 0.6242] (53,688 values at
