@@ -65,7 +65,10 @@ constexpr int kMaxWarpsPerCta = 8;  // __launch_bounds__(256)
 //      and a finished env just takes it (instantiated for the hashed and the supplied actions,
 //      whose episodes are short: for at most two warps per scheduler the four hashes fill
 //      issue slots the dynamics' dependency chain leaves empty, which is quicker than a restart
-//      branch on 77 % of the steps; with more warps, or rare restarts, it is wasted issue).
+//      branch on 77 % of the steps; with more warps, or rare restarts, it is wasted issue);
+//   4: as 0, with the start states read from the caller's array instead of hashed (a shape of
+//      its own because even a never-taken run-time test in the restart path cost shape 0
+//      4-6 %).
 // STREAMS: 0 no per-step output; 1 exactly the reward plane and the done bitmask (no run-time
 // tests in the loop); 2 any combination, tested per step.
 // LIMIT: episodes are cut off after p.max_steps steps.
@@ -76,6 +79,7 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
     constexpr int EPT = SHAPE == 2 ? 2 : 1;
     constexpr bool COOP = SHAPE == 1 || SHAPE == 2;
     constexpr bool AHEAD = SHAPE == 3;
+    constexpr bool START_IN = SHAPE == 4;
     const uint32_t lane = threadIdx.x & 31u;
     // Per warp: key pairs of up to 8 finished envs, and their 8 x 4 start-state components.
     __shared__ uint2 s_keys[COOP ? kMaxWarpsPerCta : 1][8];
@@ -218,7 +222,7 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
                     begin[j] = t1;
                     if (AHEAD) {
                         z[j] = fresh;
-                    } else if (p.start_in) {  // start states supplied as data: row (t - t0) of [T][4][n]
+                    } else if (START_IN) {  // start states supplied as data: row (t - t0) of [T][4][n]
                         const float *row = p.start_in + (int64_t)(t - p.t0) * 4 * p.n + idx[j];
                         z[j].x = __ldg(row);
                         z[j].xd = __ldg(row + p.n);
@@ -322,7 +326,7 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
                     word_off[j] += words;
                 }
             }
-            small_all = p.start_in == nullptr;
+            small_all = true;  // only read by the warp-restart shapes, which always restart from the hash
         }
 
 #pragma unroll
@@ -399,6 +403,7 @@ cudaError_t launch_shape(RolloutParams &p, int shape, cudaStream_t s) {
         case 0:
         case 3: return launch_one<POLICY, 0, STREAMS, LIMIT, CONTRACT>(p, s);
         case 1: return launch_one<POLICY, 1, STREAMS, LIMIT, CONTRACT>(p, s);
+        case 4: return launch_one<POLICY, 4, STREAMS, LIMIT, CONTRACT>(p, s);
         default: return launch_one<POLICY, 2, STREAMS, LIMIT, CONTRACT>(p, s);
     }
 }
@@ -442,8 +447,8 @@ cudaError_t launch_rollout_arith(RolloutParams &p, int policy, bool streams, cud
     const bool tiny = (p.n + 31) / 32 <= (int64_t)sm_count() * 4 * 2;
     if (coop == 0) coop = (small && ept == 1) ? ((tiny && (policy == 0 || policy == 3)) ? 3 : 2) : 1;
     // two envs per thread are always cooperative; supplied start states are read by the lane that
-    // needs them, so they always take the plain per-lane shape
-    const int shape = p.start_in ? 0 : ept == 2 ? 2 : (coop == 2 ? 0 : coop == 3 ? 3 : 1);
+    // needs them, so they always take the per-lane shape that reads them (4)
+    const int shape = p.start_in ? 4 : ept == 2 ? 2 : (coop == 2 ? 0 : coop == 3 ? 3 : 1);
     // 0: no per-step output; 1: reward plane + done bitmask only; 2: any other combination
     const int mode = !streams ? 0 : (p.reward_stream && p.done_bits && !p.action_bits && !p.trajectory) ? 1 : 2;
     // the network policies are instantiated in translation units of their own (build time)
