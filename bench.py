@@ -38,15 +38,17 @@ SMS = 148
 # smsp__inst_executed.sum / (N*T) of the kernel the library launches by default at this size
 # (restarts by the whole warp): the issue slots it really occupies.
 ROLLOUT_OPS = {
-    "random": {"thread": 69.6, "slot": 89.8},
-    "linear": {"thread": 73.8, "slot": 80.5},
-    "linear+streams": {"thread": 91.9, "slot": 94.0},
-    "mlp": {"thread": 438.3, "slot": 467.2},
-    "random+contracted": {"thread": 53.6, "slot": 72.4},
+    "random": {"thread": 68.6, "slot": 84.5},
+    "linear": {"thread": 73.8, "slot": 76.8},
+    # here the default kernel's own thread count (88.2) is below the per-lane formulation's (91.9:
+    # one running stream pointer per env instead of one per two envs), so it is the algorithmic one
+    "linear+streams": {"thread": 88.2, "slot": 88.5},
+    "mlp": {"thread": 440.3, "slot": 463.7},
+    "random+contracted": {"thread": 55.6, "slot": 70.5},
 }
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch in the same captures.
-ROLLOUT_DRAM_BYTES = {"random": 24.3e3, "linear": 24.6e3, "linear+streams": 382.1e6, "mlp": 22.5e3}
-STEP_DRAM_BYTES_16M = 566.9e6  # step_kernel at 16,777,216 envs, same kind of capture
+ROLLOUT_DRAM_BYTES = {"random": 24.6e3, "linear": 24.3e3, "linear+streams": 381.0e6, "mlp": 65.5e3}
+STEP_DRAM_BYTES_16M = 568.2e6  # step_kernel at 16,777,216 envs, same kind of capture
 # Algorithmic HBM bytes per env-step of the step paths.
 STEP_BYTES = 37.0      # 16 in + 16 out + 4 reward + 1 done, hashed action
 LADDER_BYTES = 375.0   # sum over the 46 one-op kernels of their input and output planes
