@@ -333,6 +333,23 @@ def measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args) -> dict:
     out = {}
     hbm = peaks["hbm_gbs"] * 1e9
 
+    # what the pipes sustain on this GPU: single-kind instruction streams (float32 fused
+    # multiply-add, 32-bit integer multiply-add, special-function reciprocal), beside the issue
+    # peak the rollout's roofline is derived from
+    seed = torch.linspace(0.5, 1.5, 10, device="cuda")
+    sink = torch.empty(cp.CP_CALIBRATE_THREADS_PER_SM * torch.cuda.get_device_properties(0).multi_processor_count,
+                       device="cuda")
+    calib = {"issue_peak_tinst_per_s": peak_inst / 1e12}
+    for name, kind, iters in (("ffma", 0, 20000), ("imad", 1, 20000), ("mufu_rcp", 2, 5000)):
+        count = {"n": 0}
+
+        def fn():
+            count["n"] = cp.cp_calibrate_pipe(kind, seed, sink, iters)
+        ms, _ = timed(fn, 3, 2, flush=False)
+        calib[name + "_tinst_per_s"] = 3 * count["n"] / (ms * 1e-3) / 1e12
+    out["pipe_calibration"] = calib
+    del seed, sink
+
     def step_setup(n):
         stride = (n + 3) // 4 * 4
         a = torch.zeros(4, stride, device="cuda")

@@ -354,6 +354,16 @@ int cp_selftest_arith(uint64_t *out);
  * out[0] += mismatching quotients (must stay 0), out[1] += (denominator, |numerator|) pairs tested. */
 int cp_selftest_tame_div(uint32_t den_step, uint64_t *out);
 
+/* Calibration of the roofline denominators: enqueue one launch in which every thread executes
+ * iters rounds of eight independent chains of one instruction kind — 0: float32 fused
+ * multiply-add, 1: 32-bit integer multiply-add, 2: the special-function reciprocal — on a grid of
+ * 8 CTAs x 256 threads per SM. seed DEVICE [10] floats (ordinary magnitudes, e.g. 0.5 .. 1.5),
+ * sink DEVICE [CP_CALIBRATE_THREADS_PER_SM x SM count] floats, overwritten. Returns the number of
+ * thread-instructions of the measured kind the launch executes (the caller times the launch), or
+ * a negative error code. */
+#define CP_CALIBRATE_THREADS_PER_SM 2048
+int64_t cp_calibrate_pipe(int kind, const float *seed, float *sink, int iters);
+
 const char *cp_last_error(void);
 const char *cp_version(void);
 

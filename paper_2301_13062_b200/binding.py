@@ -31,7 +31,9 @@ EXPORTS = [
     "cp_launch_count", "cp_selftest_sincos", "cp_last_error", "cp_version", "cp_step_unfused_noalloc",
     "cp_selftest_sincos_accuracy", "cp_selftest_arith", "cp_step_repeat", "cp_selftest_tame_div",
     "cp_rollout_ex", "cp_step_ex", "cp_rollout_host_shard", "cp_selftest_tanh", "cp_set_allocator",
+    "cp_calibrate_pipe",
 ]
+CP_CALIBRATE_THREADS_PER_SM = 2048
 CP_NOALLOC_MAX_ENVS = 65536
 
 
@@ -106,6 +108,7 @@ def lib() -> C.CDLL:
             "cp_selftest_sincos": (i32, [u32, u32, p]),
             "cp_selftest_sincos_accuracy": (i32, [u32, u32, p]),
             "cp_selftest_tanh": (i32, [u32, u32, p]),
+            "cp_calibrate_pipe": (i64, [i32, p, p, i32]),
             "cp_selftest_arith": (i32, [p]),
             "cp_selftest_tame_div": (i32, [u32, p]),
             "cp_last_error": (C.c_char_p, []),
@@ -411,6 +414,16 @@ def cp_selftest_tanh(lo_bits: int, hi_bits: int, out) -> None:
     import torch
     _use_current_stream()
     _check(lib().cp_selftest_tanh(lo_bits, hi_bits, _dptr(out, torch.int64)))
+
+
+def cp_calibrate_pipe(kind: int, seed, sink, iters: int) -> int:
+    """Enqueue the calibration launch; returns the thread-instructions it executes."""
+    import torch
+    _use_current_stream()
+    n = lib().cp_calibrate_pipe(kind, _dptr(seed, torch.float32), _dptr(sink, torch.float32), iters)
+    if n < 0:
+        _check(int(n))
+    return int(n)
 
 
 def cp_selftest_arith(out) -> None:

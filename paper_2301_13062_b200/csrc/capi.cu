@@ -622,6 +622,16 @@ int cp_selftest_tame_div(uint32_t den_step, uint64_t *out) {
     return e == cudaSuccess ? CP_OK : cuda_fail(e, "self-test launch");
 }
 
+int64_t cp_calibrate_pipe(int kind, const float *seed, float *sink, int iters) {
+    if (kind < 0 || kind > 2) return fail(CP_EINVAL, "kind must be 0 (FFMA), 1 (IMAD) or 2 (MUFU)");
+    if (!seed || !sink || !is_aligned(seed, 4) || !is_aligned(sink, 4)) return fail(CP_EINVAL, "seed or sink is NULL or misaligned");
+    if (iters < 1 || iters > (1 << 24)) return fail(CP_EINVAL, "iters must be in [1, 2^24]");
+    int threads = 0;
+    cudaError_t e = cp::launch_pipe_rate(kind, seed, sink, iters, &threads, tl_stream);
+    if (e != cudaSuccess) return cuda_fail(e, "calibration launch");
+    return (int64_t)threads * iters * 8;
+}
+
 const char *cp_last_error(void) { return tl_error; }
 const char *cp_version(void) { return "cartpole-b200 0.1 (sm_100a)"; }
 

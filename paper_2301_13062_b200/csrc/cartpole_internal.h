@@ -84,6 +84,7 @@ cudaError_t launch_sincos_selftest(uint32_t lo_bits, uint32_t hi_bits, unsigned 
 
 cudaError_t launch_sincos_accuracy(uint32_t lo_bits, uint32_t hi_bits, unsigned long long *out, cudaStream_t s);
 cudaError_t launch_tanh_accuracy(uint32_t lo_bits, uint32_t hi_bits, unsigned long long *out, cudaStream_t s);
+cudaError_t launch_pipe_rate(int kind, const float *seed, float *sink, int iters, int *threads, cudaStream_t s);
 cudaError_t launch_arith_selftest(unsigned long long *out, cudaStream_t s);
 cudaError_t launch_tame_div_selftest(uint32_t den_step, unsigned long long *out, cudaStream_t s);
 

@@ -382,6 +382,51 @@ cudaError_t launch_tame_div_selftest(uint32_t den_step, unsigned long long *out,
     return cudaGetLastError();
 }
 
+// ---- calibration: what one pipe sustains, for the roofline denominators ----
+// Every thread runs `iters` rounds of eight independent chains of one instruction kind
+// (0: FFMA, 1: IMAD, 2: MUFU reciprocal), sixteen resident warps per scheduler. The host times
+// the launch; instructions = threads * iters * 8. The seeds come from memory so that nothing
+// folds at compile time, and the results are stored so that nothing is dead.
+template <int KIND>
+__global__ void __launch_bounds__(256) pipe_rate_kernel(const float *seed, float *sink, int iters) {
+    float a[8];
+    uint32_t u[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        a[k] = seed[k] + (float)threadIdx.x * 1e-3f;
+        u[k] = __float_as_uint(a[k]) | 1u;
+    }
+    const float m = seed[8], c = seed[9];
+    const uint32_t um = __float_as_uint(m) | 1u, uc = __float_as_uint(c);
+    for (int i = 0; i < iters; ++i) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            if (KIND == 0) a[k] = __fmaf_rn(a[k], m, c);
+            if (KIND == 1) u[k] = u[k] * um + uc;
+            if (KIND == 2) {  // the add keeps the assembler from cancelling a reciprocal of a reciprocal
+                asm volatile("rcp.approx.ftz.f32 %0, %0;" : "+f"(a[k]));
+                a[k] = __fadd_rn(a[k], c);
+            }
+        }
+    }
+    float acc = 0.0f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) acc += KIND == 1 ? __uint_as_float(u[k] & 0x3fffffffu) : a[k];
+    sink[(size_t)blockIdx.x * blockDim.x + threadIdx.x] = acc;
+}
+
+cudaError_t launch_pipe_rate(int kind, const float *seed, float *sink, int iters, int *threads, cudaStream_t s) {
+    const int grid = sm_count() * 8, block = 256;  // 64 warps per SM = 16 per scheduler
+    *threads = grid * block;
+    switch (kind) {
+        case 0: pipe_rate_kernel<0><<<grid, block, 0, s>>>(seed, sink, iters); break;
+        case 1: pipe_rate_kernel<1><<<grid, block, 0, s>>>(seed, sink, iters); break;
+        default: pipe_rate_kernel<2><<<grid, block, 0, s>>>(seed, sink, iters); break;
+    }
+    count_launch();
+    return cudaGetLastError();
+}
+
 cudaError_t launch_arith_selftest(unsigned long long *out, cudaStream_t s) {
     arith_selftest_kernel<<<sm_count() * 8, 256, 0, s>>>(out);
     count_launch();
