@@ -281,7 +281,10 @@ def test_per_env_linear_policies_against_oracle(cp, oracle):
 def test_reset_through_the_host_program_allocator(cp, oracle):
     """cp_set_allocator: cp_reset takes its batch from torch's caching allocator (visible in torch's
     accounting, returned on cp_free) and the batch behaves like any other."""
+    import gc
     n = 200_003
+    gc.collect()               # tensors of earlier tests must not be freed between the readings
+    gc.disable()
     torch.cuda.synchronize()
     before = torch.cuda.memory_allocated()
     cp.use_torch_allocator(True)
@@ -315,6 +318,7 @@ def test_reset_through_the_host_program_allocator(cp, oracle):
         assert torch.cuda.memory_allocated() == with_batch - held
         cp.cp_free(st2)
     finally:
+        gc.enable()
         cp.use_torch_allocator(False)
 
 
@@ -354,6 +358,14 @@ def test_supplied_start_states(cp, oracle):
         same = r["ep_return_sum"] == o["ep_return_sum"]
         assert np.array_equal(H.unpack_bits(r["done_bits"], n)[:, same], H.unpack_bits(o["done_bits"], n)[:, same])
         assert r["ep_count"].sum() > n and (kind or np.median(r["ep_count"][::3]) >= 3)
+    # with an episode step limit on top (the two options meet in one kernel)
+    out = outputs(n, T)
+    cp.cp_rollout_ex(n_envs=n, T=T, seed=seed, env_offset=off, start_states_in=d_states, max_episode_steps=7, **out)
+    r = fetch(out)
+    o = oracle.rollout(n, T, seed, env_offset=off, start_states_in=states, max_episode_steps=7, done_bits=True, nthreads=4)
+    H.assert_returns_match(r["ep_return_sum"], r["ep_count"], o["ep_return_sum"], o["ep_count"])
+    same = r["ep_return_sum"] == o["ep_return_sum"]
+    assert np.array_equal(H.unpack_bits(r["done_bits"], n)[:, same], H.unpack_bits(o["done_bits"], n)[:, same])
     # (3) the contracted arithmetic and chunked calls on a batch take the option too
     st = cp.cp_reset(n, seed)
     ret = torch.empty(n, device="cuda")
