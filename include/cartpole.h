@@ -292,7 +292,8 @@ void cp_shutdown(void);
 /* Stream used by this thread's later calls (a cudaStream_t; NULL = legacy default stream). */
 void cp_set_stream(void *cuda_stream);
 
-/* Device allocator used by cp_reset for the batches it owns, process-wide: alloc(bytes) returns a
+/* Device allocator used by cp_reset for the batches it owns, process-wide (plumbing; the paper
+ * has no counterpart): alloc(bytes) returns a
  * DEVICE pointer aligned to at least 16 bytes or NULL, release(ptr) takes it back (a handle keeps
  * the release function it was created under, so the allocator may change while handles live).
  * Both NULL (the default) = cudaMalloc / cudaFree. A host program that runs its own caching
@@ -354,7 +355,8 @@ int cp_selftest_arith(uint64_t *out);
  * out[0] += mismatching quotients (must stay 0), out[1] += (denominator, |numerator|) pairs tested. */
 int cp_selftest_tame_div(uint32_t den_step, uint64_t *out);
 
-/* Calibration of the roofline denominators: enqueue one launch in which every thread executes
+/* Calibration of the roofline denominators (a measurement aid; the paper has no counterpart):
+ * enqueue one launch in which every thread executes
  * iters rounds of eight independent chains of one instruction kind — 0: float32 fused
  * multiply-add, 1: 32-bit integer multiply-add, 2: the special-function reciprocal — on a grid of
  * 8 CTAs x 256 threads per SM. seed DEVICE [10] floats (ordinary magnitudes, e.g. 0.5 .. 1.5),
