@@ -72,6 +72,23 @@ def test_rollout_beyond_4_gib(cp, oracle):
     torch.cuda.empty_cache()
 
 
+def test_last_environment_ids(cp, oracle):
+    """The top of the 32-bit env-id space: the range that ends at id 2^32 - 1 is accepted and
+    matches the oracle, one id further is refused on the host."""
+    n, T, seed = 1000, 60, 2
+    off = (1 << 32) - n
+    ret = torch.empty(n, device="cuda")
+    cnt = torch.empty(n, dtype=torch.int32, device="cuda")
+    done = torch.zeros(T, (n + 31) // 32, dtype=torch.int32, device="cuda")
+    cp.cp_rollout_shard(off, n, T, seed, None, ep_return_sum=ret, ep_count=cnt, done_bits=done)
+    torch.cuda.synchronize()
+    o = oracle.rollout(n, T, seed, env_offset=off, done_bits=True)
+    assert np.array_equal(ret.cpu().numpy(), o["ep_return_sum"])
+    assert np.array_equal(H.unpack_bits(done.cpu().numpy(), n), H.unpack_bits(o["done_bits"], n))
+    with pytest.raises(cp.CartpoleError):
+        cp.cp_rollout_shard(off + 1, n, T, seed, None, ep_return_sum=ret, ep_count=cnt)
+
+
 def test_fused_step_beyond_4_gib(cp, oracle):
     n, seed = N_BIG, 5
     stride = (n + 3) // 4 * 4
