@@ -1,0 +1,119 @@
+"""Randomised (but seeded) combinations of everything the general rollout call takes — batch size,
+horizon, start time, env offset, policy, work shape, step limit, supplied actions, supplied start
+states, output streams, arithmetic — each compared with the oracle run on the same arguments.
+Catches interactions that the per-feature tests do not cross."""
+import numpy as np
+import pytest
+
+from paper_2301_13062_b200 import inputs
+from tests import gpu_helpers as H
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def cp():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2301_13062_b200 import binding, build
+    build.build()
+    binding.lib()
+    torch.cuda.set_device(0)
+    return binding
+
+
+def pack_bits(bits):
+    T, n = bits.shape
+    words = (n + 31) // 32
+    padded = np.zeros((T, words * 32), np.uint8)
+    padded[:, :n] = bits
+    return np.packbits(padded, axis=1, bitorder="little").view(np.uint32).reshape(T, words)
+
+
+# weight draws for which the policy uses both actions (checked on the oracle)
+POLICY_SEEDS = {1: 4, 2: 6, 4: 3, 5: 3, 7: 7}
+
+
+@pytest.mark.parametrize("case", range(36))
+def test_random_combination_against_oracle(cp, oracle, case):
+    rng = np.random.default_rng(1000 + case)
+    n = int(rng.choice([1, 31, 32, 33, 97, 1000, 4097, 20011]))
+    T = int(rng.integers(1, 90))
+    seed = int(rng.integers(0, 1 << 31))
+    t0 = int(rng.choice([0, 1, 17, 100000]))
+    off = int(rng.choice([0, 5, 1 << 20]))
+    kind = int(rng.choice([0, 0, 1, 2, 4, 5, 6, 7]))
+    shape = H.SHAPES[int(rng.integers(0, len(H.SHAPES)))]
+    limit = int(rng.choice([0, 0, 1, 5, 40]))
+    supplied_actions = kind == 0 and rng.random() < 0.35
+    supplied_starts = rng.random() < 0.3
+    contracted = rng.random() < 0.25
+    streams = rng.choice(["none", "done", "reward+done", "all"])
+    words = (n + 31) // 32
+
+    if kind == 6:
+        weights = inputs.per_env_linear_weights(n, 11 + case)
+        pol = cp.policy(kind, torch.from_numpy(weights).cuda())
+    elif kind:
+        weights = inputs.policy_weights(kind, POLICY_SEEDS[kind])
+        pol = cp.policy(kind, weights)
+    else:
+        weights, pol = None, None
+    gpu_kw, ora_kw = {}, {}
+    if supplied_actions:
+        acts = rng.integers(0, 2, (T, n)).astype(np.uint8)
+        gpu_kw["action_bits_in"] = torch.from_numpy(pack_bits(acts).view(np.int32)).cuda()
+        ora_kw["action_bits_in"] = pack_bits(acts)
+    if supplied_starts:
+        starts = (0.05 * rng.uniform(-1, 1, (T, 4, n))).astype(np.float32)
+        starts[:, 2, ::5] = np.float32(0.19)
+        gpu_kw["start_states_in"] = torch.from_numpy(starts).cuda()
+        ora_kw["start_states_in"] = starts
+    out = {"ep_return_sum": torch.full((n,), -1.0, device="cuda"),
+           "ep_count": torch.full((n,), -1, dtype=torch.int32, device="cuda"),
+           "totals": torch.zeros(2, dtype=torch.int64, device="cuda"),
+           "final_state": torch.zeros(4, n, device="cuda")}
+    if streams in ("done", "reward+done", "all"):
+        out["done_bits"] = torch.zeros(T, words, dtype=torch.int32, device="cuda")
+    if streams in ("reward+done", "all"):
+        out["reward_stream"] = torch.zeros(T, n, device="cuda")
+    if streams == "all":
+        out["action_bits"] = torch.zeros(T, words, dtype=torch.int32, device="cuda")
+
+    with H.rollout_shape(cp, *shape):
+        cp.cp_rollout_ex(n_envs=n, T=T, seed=seed, t0=t0, env_offset=off, policy=pol, max_episode_steps=limit,
+                         arithmetic=cp.CP_ARITH_CONTRACTED if contracted else cp.CP_ARITH_EXACT, **gpu_kw, **out)
+    torch.cuda.synchronize()
+    r = {k: v.cpu().numpy() for k, v in out.items()}
+    o = oracle.rollout(n, T, seed, kind, weights, env_offset=off, t0=t0, max_episode_steps=limit,
+                       done_bits=True, action_bits=True, final_state=True, min_gap=True, **ora_kw)
+
+    ret, cnt = r["ep_return_sum"], r["ep_count"].view(np.uint32)
+    same = (ret == o["ep_return_sum"]) & (cnt == o["ep_count"])
+    feedback = kind != 0 and not supplied_actions
+    if contracted and feedback:
+        # statistics only (per-step differences feed back through the action choice)
+        assert same.mean() >= 0.9 or n < 100
+    else:
+        excused = same | (o["min_gap"] < 1e-5)
+        # a last-bit sine/cosine difference may flip a done flag inside the 1e-5 band: rare
+        assert excused.sum() >= n - max(1, n // 500), (n, int((~excused).sum()))
+    assert int(r["totals"][0]) == int(ret.astype(np.int64).sum())
+    assert int(r["totals"][1]) == int(cnt.astype(np.int64).sum())
+    if "done_bits" in r:
+        gd, od = H.unpack_bits(r["done_bits"], n), H.unpack_bits(o["done_bits"], n)
+        assert np.array_equal(gd.sum(axis=0), cnt)
+        assert np.array_equal(gd[:, same], od[:, same]) or (contracted and feedback)
+        if n % 32:
+            assert not np.any(r["done_bits"].view(np.uint32)[:, -1] >> (n % 32))
+    if "reward_stream" in r:
+        assert np.all(r["reward_stream"] == 1.0)
+    if "action_bits" in r and not (contracted and feedback):
+        ga, oa = H.unpack_bits(r["action_bits"], n), H.unpack_bits(o["action_bits"], n)
+        assert np.array_equal(ga[:, same], oa[:, same])
+    if not contracted:
+        live = same & np.isfinite(o["final_state"]).all(axis=0)
+        err = np.abs(r["final_state"][:, live].astype(np.float64) - o["final_state"][:, live])
+        assert err.size == 0 or err.max() < 1e-3   # trajectories that agree on every done flag stay together
