@@ -307,8 +307,11 @@ int cp_set_allocator(void *(*alloc)(size_t), void (*release)(void *));
  * batches except with the MLP policies), "rollout_coop" (how finished environments get their
  * start state: 1 = by the whole warp through shared memory, 2 = each lane its own when its env
  * finishes, 3 = each lane computes it every step ahead of the dynamics (hashed or supplied
- * actions only, otherwise as 2), 2 and 3 only with one environment per thread; 0 = default: per
- * lane for batches too small to fill the GPU (ahead for the very small), by the warp otherwise;
+ * actions only, otherwise as 2), 4 = a helper warp per stepping warp hashes every step's action
+ * and start state ahead into shared memory (hashed actions, hashed start states, canonical
+ * arithmetic, no per-step streams; otherwise as 2), 2, 3 and 4 only with one environment per
+ * thread; 0 = default: helper warps for up to six warps of environments per SM, per lane for
+ * other batches too small to fill the GPU (ahead for the smaller ones), by the warp otherwise;
  * every choice gives the same bits), "rollout_ctas_per_sm" (0 = default: one 32*ept-environment task per warp and as many
  * CTAs as that takes; k > 0 = persistent grid of k CTAs per SM looping over tasks), "step_block"
  * (32..256, default 64), "step_vec_min_envs" (batches smaller than this use the one-env-per-thread

@@ -565,7 +565,7 @@ int cp_tune(const char *key, int value) {
         if (value != 0 && value != 1 && value != 2) return fail(CP_EINVAL, "rollout_ept must be 0, 1 or 2");
         cp::g_tuning.rollout_ept = value;
     } else if (!strcmp(key, "rollout_coop")) {
-        if (value < 0 || value > 3) return fail(CP_EINVAL, "rollout_coop must be 0, 1, 2 or 3");
+        if (value < 0 || value > 4) return fail(CP_EINVAL, "rollout_coop must be 0..4");
         cp::g_tuning.rollout_coop = value;
     } else if (!strcmp(key, "rollout_ctas_per_sm")) {
         if (value < 0 || value > 1024) return fail(CP_EINVAL, "rollout_ctas_per_sm must be 0..1024");

@@ -51,7 +51,8 @@ struct RolloutParams {
 struct LaunchTuning {
     int rollout_block = 0;        // 0: 128 for very small batches, 256 otherwise
     int rollout_ept = 0;          // 0: chosen per policy and batch size
-    int rollout_coop = 0;         // 0: chosen per batch size; 1 restarts by the warp; 2 per lane (ept 1)
+    int rollout_coop = 0;         // 0: chosen per batch size; 1 restarts by the warp; 2 per lane (ept 1);
+                                  // 3 per lane, computed ahead; 4 handed over by a producer warp
     int rollout_ctas_per_sm = 0;  // 0: one task per warp (non-persistent grid)
     int step_block = 64;
     // Below this many envs the one-env-per-thread kernel is used: a small batch is latency-bound,
@@ -75,6 +76,9 @@ cudaError_t launch_actions(uint8_t *out, int64_t n, uint32_t env_offset, uint32_
                            cudaStream_t s);
 cudaError_t launch_rollout(RolloutParams &p, int policy, bool streams, bool contracted, cudaStream_t s);
 cudaError_t launch_rollout_contracted(RolloutParams &p, int policy, bool streams, cudaStream_t s);
+// the producer-assisted kernel for very small batches, and whether a call is one it covers
+bool rollout_assisted_applies(const RolloutParams &p, int policy, bool streams);
+cudaError_t launch_rollout_assisted(RolloutParams &p, cudaStream_t s);
 // the MLP policies (kinds 2, 4, 5, 7), canonical and contracted arithmetic; mode and shape as
 // chosen by launch_rollout_arith
 cudaError_t launch_rollout_networks(RolloutParams &p, int policy, int mode, int shape, cudaStream_t s);

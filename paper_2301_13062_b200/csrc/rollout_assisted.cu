@@ -1,0 +1,197 @@
+// Rollout for batches far too small to fill the chip (the paper's own shape, 2,048 environments
+// x 10,000 steps, Sec. V-A, is 64 warps on 592 warp schedulers): there a step's LATENCY is what
+// is paid, and every instruction the stepping warp does not have to issue shortens it.
+//
+// Everything random in a rollout depends on (seed, env, time) only, never on the trajectory. So
+// each stepping warp ("consumer") gets a helper warp ("producer") on another scheduler of the
+// same SM that hashes, a chunk of steps ahead, the action force and the start state of every
+// step for the consumer's 32 environments into shared memory. The consumer's step is then two
+// shared-memory loads, the dynamics, the termination test and four selects: about 60 instead
+// of 110 instructions, with no integer hashing in its dependency chain. Same hashes, same
+// dynamics function, same bits as the general kernel.
+//
+// Synchronisation: one hardware barrier per consumer/producer pair (bar.sync with the pair's own
+// id, 64 threads), once per chunk, double-buffered. Both warps of a pair execute exactly
+// 1 + ceil(T / kChunk) barriers, a number fixed by the launch parameters alone; there is no flag,
+// no spin and no dependence on data, so neither warp can wait for an arrival that does not come.
+//
+// Scope: hashed actions, canonical arithmetic, hashed start states, no per-step streams (with or
+// without an episode step limit). Every other call takes the general kernel.
+#include "cartpole_device.cuh"
+#include "cartpole_internal.h"
+
+namespace cp {
+
+namespace {
+
+// Steps per hand-over: 40 KB of static shared memory per CTA either way (640 bytes per step, two
+// buffers). Measured on 2,048 x 10,000: 8 steps 0.543 ms, 16 steps 0.512 ms.
+template <int PAIRS>
+constexpr int kChunkOf = PAIRS == 1 ? 32 : 16;
+
+template <int CHUNK>
+struct PairBuffers {
+    float4 start[2][CHUNK][32];  // start state of time t + 1, for the env of each lane
+    float force[2][CHUNK][32];   // +-F of the action at time t
+};
+
+// Barrier 1 for pair 0, barrier 2 for pair 1 (immediates: a register id makes the kernel claim
+// all sixteen barriers).
+template <int PAIRS>
+__device__ __forceinline__ void pair_barrier(uint32_t pair) {
+    __syncwarp();
+    if (PAIRS == 1 || pair == 0u)
+        asm volatile("bar.sync 1, 64;" ::: "memory");
+    else
+        asm volatile("bar.sync 2, 64;" ::: "memory");
+}
+
+template <bool KNOWN_SMALL, bool LIMIT, int CHUNK>
+__device__ __forceinline__ void consume_step(const PairBuffers<CHUNK> &buf, uint32_t b, int s, uint32_t lane,
+                                             uint32_t t1, uint32_t max_steps, State &z, uint32_t &cnt,
+                                             uint32_t &begin) {
+    const float4 fresh = buf.start[b][s][lane];
+    const float force = buf.force[b][s][lane];
+    bool done = euler_step<KNOWN_SMALL>(z, force);
+    if (LIMIT) done |= (t1 - begin) >= max_steps;
+    // selects, not a branch: nothing diverges in the stepping warp (measured equal or up to 4 % faster)
+    cnt += done ? 1u : 0u;
+    begin = done ? t1 : begin;
+    z.x = done ? fresh.x : z.x;
+    z.xd = done ? fresh.y : z.xd;
+    z.th = done ? fresh.z : z.th;
+    z.thd = done ? fresh.w : z.thd;
+}
+
+template <int PAIRS, bool LIMIT>
+__global__ void __launch_bounds__(64 * PAIRS) rollout_assisted_kernel(const __grid_constant__ RolloutParams p) {
+    constexpr int kChunk = kChunkOf<PAIRS>;
+    __shared__ PairBuffers<kChunk> s_buf[PAIRS];
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const bool producer = warp >= (uint32_t)PAIRS;
+    const uint32_t pair = producer ? warp - PAIRS : warp;
+    const int64_t task = (int64_t)blockIdx.x * PAIRS + pair;
+    if (task >= p.n_tasks) return;  // both warps of the pair leave; no other pair uses their barrier
+    PairBuffers<kChunk> &buf = s_buf[pair];
+    const uint32_t n_chunks = (p.T + kChunk - 1) / kChunk;
+
+    int64_t idx = task * 32 + lane;
+    const bool valid = idx < p.n;
+    if (!valid) idx = p.n - 1;  // idle lanes shadow the last environment and store nothing
+    const uint32_t env = p.env_offset + (uint32_t)idx;
+    const FoldedKeys kr = fold_keys(make_keys(p.salt_r, env));
+
+    if (producer) {
+        const FoldedKeys ka = fold_keys(make_keys(p.salt_a, env));
+        for (uint32_t c = 0; c <= n_chunks; ++c) {
+            // chunk c is written while the consumer works on chunk c - 1 (other buffer); the
+            // buffer written here was last read in chunk c - 2, which the barrier before closed
+            if (c < n_chunks) {
+                const uint32_t b = c & 1u, tc = p.t0 + c * kChunk;
+#pragma unroll 4
+                for (int s = 0; s < kChunk; ++s) {
+                    const uint32_t t = tc + s;
+                    const State f = start_state_folded(kr, fold16(4u * (t + 1u)));
+                    buf.start[b][s][lane] = make_float4(f.x, f.xd, f.th, f.thd);
+                    buf.force[b][s][lane] = force_from_signbit(action_signbit_folded(ka, fold16(t)));
+                }
+            }
+            pair_barrier<PAIRS>(pair);
+        }
+        return;
+    }
+
+    State z;
+    if (p.init_planes) {
+        z.x = p.init_planes[idx];
+        z.xd = p.init_planes[p.init_stride + idx];
+        z.th = p.init_planes[2 * p.init_stride + idx];
+        z.thd = p.init_planes[3 * p.init_stride + idx];
+    } else {
+        z = start_state_folded(kr, fold16(4u * p.t0));
+    }
+    // as in the general kernel: the returns follow from the time of the last termination, and
+    // only the step limit needs the carried-in episode length inside the loop
+    uint32_t cnt = 0u, begin = p.t0 - ((LIMIT && p.ep_len_io) ? p.ep_len_io[idx] : 0u);
+    const uint32_t t_end = p.t0 + p.T;
+    pair_barrier<PAIRS>(pair);  // chunk 0 is there
+    for (uint32_t c = 0; c < n_chunks; ++c) {
+        const uint32_t b = c & 1u, tc = p.t0 + c * kChunk;
+        const int steps = (int)min((uint32_t)kChunk, t_end - tc);
+        if (c == 0u) {
+            // the caller's initial state may hold any angle: the first chunk tests it per lane
+            for (int s = 0; s < steps; ++s)
+                consume_step<false, LIMIT>(buf, b, s, lane, tc + s + 1u, p.max_steps, z, cnt, begin);
+        } else if (steps == kChunk) {
+            // from the second step on every angle is a survivor's (<= 0.2095) or a start state's
+#pragma unroll
+            for (int s = 0; s < kChunk; ++s)
+                consume_step<true, LIMIT>(buf, b, s, lane, tc + s + 1u, p.max_steps, z, cnt, begin);
+        } else {
+            for (int s = 0; s < steps; ++s)
+                consume_step<true, LIMIT>(buf, b, s, lane, tc + s + 1u, p.max_steps, z, cnt, begin);
+        }
+        pair_barrier<PAIRS>(pair);
+    }
+
+    unsigned long long tot_ret = 0, tot_cnt = 0;
+    if (valid) {
+        const uint32_t carried = p.ep_len_io ? p.ep_len_io[idx] : 0u;
+        const uint32_t first_begin = p.t0 - carried;
+        const uint32_t ret = cnt ? begin - first_begin : 0u;
+        const uint32_t running = t_end - begin + ((!LIMIT && cnt == 0u) ? carried : 0u);
+        if (p.ep_return_sum) p.ep_return_sum[idx] = (float)ret;
+        if (p.ep_count) p.ep_count[idx] = cnt;
+        if (p.ep_len_io) p.ep_len_io[idx] = running;
+        if (p.out_planes) {
+            p.out_planes[idx] = z.x;
+            p.out_planes[p.out_stride + idx] = z.xd;
+            p.out_planes[2 * p.out_stride + idx] = z.th;
+            p.out_planes[3 * p.out_stride + idx] = z.thd;
+        }
+        tot_ret = ret;
+        tot_cnt = cnt;
+    }
+    if (p.totals) {
+        for (int o = 16; o > 0; o >>= 1) {
+            tot_ret += __shfl_down_sync(0xffffffffu, tot_ret, o);
+            tot_cnt += __shfl_down_sync(0xffffffffu, tot_cnt, o);
+        }
+        if (lane == 0 && (tot_ret | tot_cnt)) {
+            atomicAdd(p.totals, tot_ret);
+            atomicAdd(p.totals + 1, tot_cnt);
+        }
+    }
+}
+
+}  // namespace
+
+bool rollout_assisted_applies(const RolloutParams &p, int policy, bool streams) {
+    if (policy != 0 || streams || p.action_bits_in || p.start_in) return false;
+    if (g_tuning.rollout_coop == 4) return true;
+    if (g_tuning.rollout_coop != 0 || g_tuning.rollout_ept != 0) return false;
+    // up to six pairs per SM, three warps per scheduler. Measured against the general kernel's
+    // best shape, x 5,000 steps: 9,472 envs 0.26 / 0.61 ms, 18,944 envs 0.48 / 0.61 ms,
+    // 28,416 envs 0.65 / 0.74 ms, 33,152 envs (seven pairs per SM) 0.83 / 0.74 ms.
+    return (p.n + 31) / 32 <= (int64_t)sm_count() * 6;
+}
+
+cudaError_t launch_rollout_assisted(RolloutParams &p, cudaStream_t s) {
+    p.n_tasks = (p.n + 31) / 32;
+    // one pair per CTA spreads the pairs over the SMs; beyond one pair per SM, two pairs per CTA
+    // put the four warps of a CTA on the four schedulers of one SM
+    const bool two = g_tuning.rollout_block ? g_tuning.rollout_block >= 128 : p.n_tasks > sm_count();
+    const unsigned grid = (unsigned)(two ? (p.n_tasks + 1) / 2 : p.n_tasks);
+    if (two && p.max_steps)
+        rollout_assisted_kernel<2, true><<<grid, 128, 0, s>>>(p);
+    else if (two)
+        rollout_assisted_kernel<2, false><<<grid, 128, 0, s>>>(p);
+    else if (p.max_steps)
+        rollout_assisted_kernel<1, true><<<grid, 64, 0, s>>>(p);
+    else
+        rollout_assisted_kernel<1, false><<<grid, 64, 0, s>>>(p);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace cp

@@ -448,7 +448,9 @@ cudaError_t launch_rollout_arith(RolloutParams &p, int policy, bool streams, cud
     if (coop == 0) coop = (small && ept == 1) ? ((tiny && (policy == 0 || policy == 3)) ? 3 : 2) : 1;
     // two envs per thread are always cooperative; supplied start states are read by the lane that
     // needs them, so they always take the per-lane shape that reads them (4)
-    const int shape = p.start_in ? 4 : ept == 2 ? 2 : (coop == 2 ? 0 : coop == 3 ? 3 : 1);
+    // (coop 4 asks for the producer-assisted kernel of rollout_assisted.cu; a call it does not
+    // cover lands here and takes the plain per-lane shape)
+    const int shape = p.start_in ? 4 : ept == 2 ? 2 : ((coop == 2 || coop == 4) ? 0 : coop == 3 ? 3 : 1);
     // 0: no per-step output; 1: reward plane + done bitmask only; 2: any other combination
     const int mode = !streams ? 0 : (p.reward_stream && p.done_bits && !p.action_bits && !p.trajectory) ? 1 : 2;
     // the network policies are instantiated in translation units of their own (build time)

@@ -24,9 +24,11 @@ REL_TOL = 2e-6
 
 # The rollout kernel's work shapes as (rollout_ept, rollout_coop) tuning values: one env per
 # thread with per-lane restarts, the same with start states computed ahead every step, one env
-# per thread with restarts by the whole warp, two envs per thread (always by the warp). The
+# per thread with restarts by the whole warp, two envs per thread (always by the warp), and the
+# kernel whose helper warps hash actions and start states ahead of the stepping warps (it covers
+# hashed actions without streams or step limit; other calls fall to the first shape). The
 # library picks one by batch size and policy; tests force each of them on small batches.
-SHAPES = [(1, 2), (1, 3), (1, 1), (2, 1)]
+SHAPES = [(1, 2), (1, 3), (1, 1), (2, 1), (1, 4)]
 
 
 @contextlib.contextmanager

@@ -1,0 +1,125 @@
+"""The producer-assisted rollout kernel (very small batches: a helper warp hashes actions and start
+states ahead of each stepping warp). It must give the same bits as the general kernel, which the
+other files pin to the oracle, and it is compared with the oracle directly as well. Cases: ragged
+batch sizes, horizons around the 16- and 32-step hand-overs, both CTA forms with an odd number of warp
+tasks, a caller's initial state with angles outside the polynomial range, carried episode lengths
+and the step limit."""
+import contextlib
+
+import numpy as np
+import pytest
+
+from tests import gpu_helpers as H
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+ASSISTED, PER_LANE = 4, 2
+
+
+@pytest.fixture(scope="module")
+def cp():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2301_13062_b200 import binding, build
+    build.build()
+    binding.lib()
+    torch.cuda.set_device(0)
+    return binding
+
+
+@contextlib.contextmanager
+def kernel(cp, coop, block=0):
+    cp.cp_tune("rollout_block", block)
+    try:
+        with H.rollout_shape(cp, 1, coop):
+            yield
+    finally:
+        cp.cp_tune("rollout_block", 0)
+
+
+def rollout(cp, coop, n, T, seed, block=0, **kw):
+    out = {"ep_return_sum": torch.full((n,), -1.0, device="cuda"),
+           "ep_count": torch.full((n,), -1, dtype=torch.int32, device="cuda"),
+           "totals": torch.zeros(2, dtype=torch.int64, device="cuda"),
+           "final_state": torch.zeros(4, n, device="cuda")}
+    with kernel(cp, coop, block):
+        cp.cp_rollout_ex(n_envs=n, T=T, seed=seed, **kw, **out)
+    torch.cuda.synchronize()
+    return {k: v.cpu().numpy() for k, v in out.items()}
+
+
+def assert_same_bits(a, b):
+    for k in a:
+        assert np.array_equal(a[k].view(np.uint32) if a[k].dtype == np.float32 else a[k],
+                              b[k].view(np.uint32) if b[k].dtype == np.float32 else b[k]), k
+
+
+@pytest.mark.parametrize("n", [1, 33, 1000, 4737])
+@pytest.mark.parametrize("T", [1, 15, 16, 17, 32, 33, 100])
+def test_same_bits_as_general_kernel_and_oracle(cp, oracle, n, T):
+    seed, t0, off = 12, 5, 77
+    general = rollout(cp, PER_LANE, n, T, seed, t0=t0, env_offset=off)
+    for block in (64, 128):                      # one pair and two pairs per CTA (4737 envs: 149 tasks, odd)
+        got = rollout(cp, ASSISTED, n, T, seed, block, t0=t0, env_offset=off)
+        assert_same_bits(got, general)
+    auto = rollout(cp, 0, n, T, seed, t0=t0, env_offset=off)      # what a caller gets
+    assert_same_bits(auto, general)
+    o = oracle.rollout(n, T, seed, env_offset=off, t0=t0, min_gap=True)
+    H.assert_returns_match(auto["ep_return_sum"], auto["ep_count"].view(np.uint32), o["ep_return_sum"],
+                           o["ep_count"], excuse=o["min_gap"] < 1e-5,
+                           min_identical=0.999 if n >= 1000 else 0.0)
+    assert int(auto["totals"][1]) == int(auto["ep_count"].astype(np.int64).sum())
+
+
+def test_callers_state_with_large_angles(cp, oracle):
+    """Angles beyond the polynomial range in the initial state (some survive the first step): the
+    first hand-over chunk must take the full-range sine and cosine."""
+    n, seed, T = 2000, 4, 40
+    rng = np.random.default_rng(3)
+    z0 = np.stack([rng.uniform(-2, 2, n), rng.uniform(-1, 1, n), rng.uniform(-0.3, 0.3, n),
+                   rng.uniform(-3, 3, n)]).astype(np.float32)
+    z0[2, :8] = [0.25, -0.25, 0.2201, -0.2201, 0.5, 3.0, -40.0, 0.2199]
+    z0[3, :8] = [-3.0, 3.0, -1.0, 1.0, -20.0, 0.0, 0.0, 0.0]
+    res = {}
+    for coop in (PER_LANE, ASSISTED):
+        planes = torch.zeros(4, (n + 3) // 4 * 4, device="cuda")
+        planes[:, :n] = torch.from_numpy(z0).cuda()
+        st = cp.cp_wrap(planes, n, seed, 9)
+        ret = torch.empty(n, device="cuda")
+        cnt = torch.empty(n, dtype=torch.int32, device="cuda")
+        with kernel(cp, coop):
+            cp.cp_rollout_from(st, T, None, None, ep_return_sum=ret, ep_count=cnt)
+        torch.cuda.synchronize()
+        res[coop] = {"ret": ret.cpu().numpy(), "cnt": cnt.cpu().numpy(), "z": planes[:, :n].cpu().numpy()}
+    assert_same_bits(res[ASSISTED], res[PER_LANE])
+    o = oracle.rollout(n, T, seed, t0=9, init_state=z0, final_state=True, min_gap=True)
+    H.assert_returns_match(res[ASSISTED]["ret"], res[ASSISTED]["cnt"].view(np.uint32), o["ep_return_sum"],
+                           o["ep_count"], excuse=o["min_gap"] < 1e-5)
+    survived_wide = (np.abs(z0[2]) > 0.22) & (np.abs(z0[2] + np.float32(0.02) * z0[3]) < 0.2)
+    assert survived_wide.sum() >= 2        # the case the test is about occurs
+
+
+def test_step_limit_and_carried_lengths_in_chunks(cp, oracle):
+    n, seed, limit = 1500, 21, 25
+    whole = oracle.rollout(n, 63, seed, max_episode_steps=limit, final_state=True, min_gap=True)
+    res = {}
+    for coop in (PER_LANE, ASSISTED):
+        st = cp.cp_reset(n, seed)
+        ep_len = torch.zeros(n, dtype=torch.int32, device="cuda")
+        ret, cnt = np.zeros(n, np.float32), np.zeros(n, np.uint32)
+        for T in (7, 16, 40):
+            rs = torch.zeros(n, device="cuda")
+            ct = torch.zeros(n, dtype=torch.int32, device="cuda")
+            with kernel(cp, coop):
+                cp.cp_rollout_ex(T=T, state=st, ep_len=ep_len, max_episode_steps=limit, ep_return_sum=rs, ep_count=ct)
+            torch.cuda.synchronize()
+            ret += rs.cpu().numpy()
+            cnt += ct.cpu().numpy().view(np.uint32)
+        res[coop] = {"ret": ret, "cnt": cnt, "len": ep_len.cpu().numpy()}
+        cp.cp_free(st)
+    assert_same_bits(res[ASSISTED], res[PER_LANE])
+    H.assert_returns_match(res[ASSISTED]["ret"], res[ASSISTED]["cnt"], whole["ep_return_sum"], whole["ep_count"],
+                           excuse=whole["min_gap"] < 1e-5)
+    assert res[ASSISTED]["len"].max() < limit
