@@ -310,7 +310,7 @@ int cp_set_allocator(void *(*alloc)(size_t), void (*release)(void *));
  * actions only, otherwise as 2), 4 = a helper warp per stepping warp hashes every step's action
  * and start state ahead into shared memory (hashed actions, hashed start states, canonical
  * arithmetic, no per-step streams; otherwise as 2), 2, 3 and 4 only with one environment per
- * thread; 0 = default: helper warps for up to six warps of environments per SM, per lane for
+ * thread; 0 = default: helper warps for up to ten warps of environments per SM, per lane for
  * other batches too small to fill the GPU (ahead for the smaller ones), by the warp otherwise;
  * every choice gives the same bits), "rollout_ctas_per_sm" (0 = default: one 32*ept-environment task per warp and as many
  * CTAs as that takes; k > 0 = persistent grid of k CTAs per SM looping over tasks), "step_block"

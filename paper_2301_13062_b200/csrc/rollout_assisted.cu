@@ -29,6 +29,10 @@ namespace {
 template <int PAIRS>
 constexpr int kChunkOf = PAIRS == 1 ? 32 : 16;
 
+// Steps per trip of the consumer's loop over a chunk. Measured on 2,048 x 10,000 (ms per launch):
+// 1: 0.666, 2: 0.481, 3: 0.487, 4: 0.503, 8: 0.504, 16: 0.506, whole chunk: 0.506.
+constexpr int kStepUnroll = 2;
+
 template <int CHUNK>
 struct PairBuffers {
     float4 start[2][CHUNK][32];  // start state of time t + 1, for the env of each lane
@@ -124,7 +128,7 @@ __global__ void __launch_bounds__(64 * PAIRS) rollout_assisted_kernel(const __gr
                 consume_step<false, LIMIT>(buf, b, s, lane, tc + s + 1u, p.max_steps, z, cnt, begin);
         } else if (steps == kChunk) {
             // from the second step on every angle is a survivor's (<= 0.2095) or a start state's
-#pragma unroll
+#pragma unroll kStepUnroll
             for (int s = 0; s < kChunk; ++s)
                 consume_step<true, LIMIT>(buf, b, s, lane, tc + s + 1u, p.max_steps, z, cnt, begin);
         } else {
@@ -170,10 +174,12 @@ bool rollout_assisted_applies(const RolloutParams &p, int policy, bool streams) 
     if (policy != 0 || streams || p.action_bits_in || p.start_in) return false;
     if (g_tuning.rollout_coop == 4) return true;
     if (g_tuning.rollout_coop != 0 || g_tuning.rollout_ept != 0) return false;
-    // up to six pairs per SM, three warps per scheduler. Measured against the general kernel's
-    // best shape, x 5,000 steps: 9,472 envs 0.26 / 0.61 ms, 18,944 envs 0.48 / 0.61 ms,
-    // 28,416 envs 0.65 / 0.74 ms, 33,152 envs (seven pairs per SM) 0.83 / 0.74 ms.
-    return (p.n + 31) / 32 <= (int64_t)sm_count() * 6;
+    // up to ten pairs per SM (five CTAs of two pairs: 200 KB of shared memory; a sixth CTA would
+    // wait for a second wave). Measured against the general kernel's best shape, ms per launch:
+    // x 5,000 steps 9,472 envs 0.25 / 0.61, 18,944 envs 0.45 / 0.61, 28,416 envs 0.57 / 0.74,
+    // 37,888 envs 0.70 / 0.74; x 4,000 steps 47,360 envs (ten pairs per SM) 0.72 / 0.83,
+    // 56,832 envs (twelve) 0.88 / 0.82.
+    return (p.n + 31) / 32 <= (int64_t)sm_count() * 10;
 }
 
 cudaError_t launch_rollout_assisted(RolloutParams &p, cudaStream_t s) {
