@@ -122,17 +122,21 @@ __global__ void __launch_bounds__(64 * PAIRS) rollout_assisted_kernel(const __gr
     for (uint32_t c = 0; c < n_chunks; ++c) {
         const uint32_t b = c & 1u, tc = p.t0 + c * kChunk;
         const int steps = (int)min((uint32_t)kChunk, t_end - tc);
-        if (c == 0u) {
-            // the caller's initial state may hold any angle: the first chunk tests it per lane
-            for (int s = 0; s < steps; ++s)
-                consume_step<false, LIMIT>(buf, b, s, lane, tc + s + 1u, p.max_steps, z, cnt, begin);
-        } else if (steps == kChunk) {
-            // from the second step on every angle is a survivor's (<= 0.2095) or a start state's
+        if (c != 0u && steps == kChunk) {
 #pragma unroll kStepUnroll
             for (int s = 0; s < kChunk; ++s)
                 consume_step<true, LIMIT>(buf, b, s, lane, tc + s + 1u, p.max_steps, z, cnt, begin);
         } else {
-            for (int s = 0; s < steps; ++s)
+            // The caller's initial state may hold any angle: the very first step tests it per
+            // lane. From the second step on every angle is a survivor's (<= 0.2095) or a start
+            // state's (<= 0.05).
+            int s = 0;
+            if (c == 0u) {
+                consume_step<false, LIMIT>(buf, b, 0, lane, tc + 1u, p.max_steps, z, cnt, begin);
+                s = 1;
+            }
+#pragma unroll kStepUnroll
+            for (; s < steps; ++s)
                 consume_step<true, LIMIT>(buf, b, s, lane, tc + s + 1u, p.max_steps, z, cnt, begin);
         }
         pair_barrier<PAIRS>(pair);
