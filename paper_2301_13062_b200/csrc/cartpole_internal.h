@@ -78,7 +78,7 @@ cudaError_t launch_rollout(RolloutParams &p, int policy, bool streams, bool cont
 cudaError_t launch_rollout_contracted(RolloutParams &p, int policy, bool streams, cudaStream_t s);
 // the producer-assisted kernel for very small batches, and whether a call is one it covers
 bool rollout_assisted_applies(const RolloutParams &p, int policy, bool streams);
-cudaError_t launch_rollout_assisted(RolloutParams &p, cudaStream_t s);
+cudaError_t launch_rollout_assisted(RolloutParams &p, bool contracted, cudaStream_t s);
 // the MLP policies (kinds 2, 4, 5, 7), canonical and contracted arithmetic; mode and shape as
 // chosen by launch_rollout_arith
 cudaError_t launch_rollout_networks(RolloutParams &p, int policy, int mode, int shape, cudaStream_t s);

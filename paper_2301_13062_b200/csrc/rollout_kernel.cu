@@ -5,9 +5,9 @@
 namespace cp {
 
 cudaError_t launch_rollout(RolloutParams &p, int policy, bool streams, bool contracted, cudaStream_t s) {
-    if (contracted) return launch_rollout_contracted(p, policy, streams, s);
     // very small batches with hashed actions: a helper warp per stepping warp (rollout_assisted.cu)
-    if (rollout_assisted_applies(p, policy, streams)) return launch_rollout_assisted(p, s);
+    if (rollout_assisted_applies(p, policy, streams)) return launch_rollout_assisted(p, contracted, s);
+    if (contracted) return launch_rollout_contracted(p, policy, streams, s);
     return launch_rollout_arith<false>(p, policy, streams, s);
 }
 

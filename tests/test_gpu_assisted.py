@@ -73,6 +73,21 @@ def test_same_bits_as_general_kernel_and_oracle(cp, oracle, n, T):
     assert int(auto["totals"][1]) == int(auto["ep_count"].astype(np.int64).sum())
 
 
+@pytest.mark.parametrize("limit", [0, 30])
+def test_contracted_arithmetic_same_bits_as_general_kernel(cp, oracle, limit):
+    n, T, seed = 3001, 150, 5
+    kw = {"arithmetic": cp.CP_ARITH_CONTRACTED, "max_episode_steps": limit, "t0": 3}
+    general = rollout(cp, PER_LANE, n, T, seed, **kw)
+    for block in (64, 128):
+        assert_same_bits(rollout(cp, ASSISTED, n, T, seed, block, **kw), general)
+    auto = rollout(cp, 0, n, T, seed, **kw)
+    assert_same_bits(auto, general)
+    canonical = rollout(cp, 0, n, T, seed, max_episode_steps=limit, t0=3)
+    assert not np.array_equal(auto["final_state"], canonical["final_state"])    # the variant really ran
+    o = oracle.rollout(n, T, seed, t0=3, max_episode_steps=limit)
+    H.assert_returns_match(auto["ep_return_sum"], auto["ep_count"].view(np.uint32), o["ep_return_sum"], o["ep_count"])
+
+
 def test_callers_state_with_large_angles(cp, oracle):
     """Angles beyond the polynomial range in the initial state (some survive the first step): the
     first hand-over chunk must take the full-range sine and cosine."""
