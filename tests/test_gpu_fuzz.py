@@ -2,6 +2,8 @@
 horizon, start time, env offset, policy, work shape, step limit, supplied actions, supplied start
 states, output streams, arithmetic — each compared with the oracle run on the same arguments.
 Catches interactions that the per-feature tests do not cross."""
+import os
+
 import numpy as np
 import pytest
 
@@ -36,7 +38,7 @@ def pack_bits(bits):
 POLICY_SEEDS = {1: 4, 2: 6, 4: 3, 5: 3, 7: 7}
 
 
-@pytest.mark.parametrize("case", range(36))
+@pytest.mark.parametrize("case", range(int(os.environ.get("CARTPOLE_FUZZ_CASES", "36"))))   # more for a soak run
 def test_random_combination_against_oracle(cp, oracle, case):
     rng = np.random.default_rng(1000 + case)
     n = int(rng.choice([1, 31, 32, 33, 97, 1000, 4097, 20011]))
