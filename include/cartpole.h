@@ -308,8 +308,8 @@ int cp_set_allocator(void *(*alloc)(size_t), void (*release)(void *));
  * start state: 1 = by the whole warp through shared memory, 2 = each lane its own when its env
  * finishes, 3 = each lane computes it every step ahead of the dynamics (hashed or supplied
  * actions only, otherwise as 2), 4 = a helper warp per stepping warp hashes every step's action
- * and start state ahead into shared memory (hashed actions, hashed start states, no per-step
- * streams; otherwise as 2), 2, 3 and 4 only with one environment per
+ * and start state ahead into shared memory (hashed or supplied actions and hashed start
+ * states; otherwise as 2), 2, 3 and 4 only with one environment per
  * thread; 0 = default: helper warps for up to ten warps of environments per SM, per lane for
  * other batches too small to fill the GPU (ahead for the smaller ones), by the warp otherwise;
  * every choice gives the same bits), "rollout_ctas_per_sm" (0 = default: one 32*ept-environment task per warp and as many

@@ -15,8 +15,9 @@
 // 1 + ceil(T / kChunk) barriers, a number fixed by the launch parameters alone; there is no flag,
 // no spin and no dependence on data, so neither warp can wait for an arrival that does not come.
 //
-// Scope: hashed actions, hashed start states, no per-step streams (either arithmetic, with or
-// without an episode step limit). Every other call takes the general kernel.
+// Scope: hashed or supplied actions (the producer turns the caller's action words into forces),
+// hashed start states, either arithmetic, with or without an episode step limit and per-step
+// output streams. Calls with a feedback policy or supplied start states take the general kernel.
 #include "cartpole_device.cuh"
 #include "cartpole_internal.h"
 
@@ -50,14 +51,21 @@ __device__ __forceinline__ void pair_barrier(uint32_t pair) {
         asm volatile("bar.sync 2, 64;" ::: "memory");
 }
 
-template <bool KNOWN_SMALL, bool LIMIT, bool CONTRACT, int CHUNK>
-__device__ __forceinline__ void consume_step(const PairBuffers<CHUNK> &buf, uint32_t b, int s, uint32_t lane,
-                                             uint32_t t1, uint32_t max_steps, State &z, uint32_t &cnt,
-                                             uint32_t &begin) {
+// Where the consumer's per-step outputs go (only read when STREAMS): offsets into the [T][n]
+// planes and the [T][words] bit planes advance by one row per step.
+struct StreamCursor {
+    int64_t env_off, word_off, idx, words;
+    bool valid, want_done, want_act, want_rew, want_traj;
+};
+
+template <bool KNOWN_SMALL, bool LIMIT, bool CONTRACT, int STREAMS, int CHUNK>
+__device__ __forceinline__ void consume_step(const RolloutParams &p, const PairBuffers<CHUNK> &buf, uint32_t b,
+                                             int s, uint32_t lane, uint32_t t1, StreamCursor &sc, State &z,
+                                             uint32_t &cnt, uint32_t &begin) {
     const float4 fresh = buf.start[b][s][lane];
     const float force = buf.force[b][s][lane];
     bool done = CONTRACT ? euler_step_contracted<KNOWN_SMALL>(z, force) : euler_step<KNOWN_SMALL>(z, force);
-    if (LIMIT) done |= (t1 - begin) >= max_steps;
+    if (LIMIT) done |= (t1 - begin) >= p.max_steps;
     // selects, not a branch: nothing diverges in the stepping warp (measured equal or up to 4 % faster)
     cnt += done ? 1u : 0u;
     begin = done ? t1 : begin;
@@ -65,9 +73,41 @@ __device__ __forceinline__ void consume_step(const PairBuffers<CHUNK> &buf, uint
     z.xd = done ? fresh.y : z.xd;
     z.th = done ? fresh.z : z.th;
     z.thd = done ? fresh.w : z.thd;
+    // Same layout and meaning as the general kernel's streams. STREAMS 1: exactly the reward plane
+    // and the done bits, no tests (each run-time test is a branch in the one warp whose latency
+    // is the launch's time); 2: any combination.
+    if (STREAMS == 1) {
+        const uint32_t m = __ballot_sync(0xffffffffu, done && sc.valid);
+        if (lane == 0u) p.done_bits[sc.word_off] = m;
+        if (sc.valid) p.reward_stream[sc.env_off] = 1.0f;
+        sc.env_off += p.n;
+        sc.word_off += sc.words;
+    }
+    if (STREAMS == 2) {
+        if (sc.want_done) {
+            const uint32_t m = __ballot_sync(0xffffffffu, done && sc.valid);
+            if (lane == 0u) p.done_bits[sc.word_off] = m;
+        }
+        if (sc.want_act) {
+            const uint32_t m = __ballot_sync(0xffffffffu, force > 0.0f && sc.valid);
+            if (lane == 0u) p.action_bits[sc.word_off] = m;
+        }
+        if (sc.valid) {
+            if (sc.want_rew) p.reward_stream[sc.env_off] = 1.0f;
+            if (sc.want_traj) {
+                float *tr = p.trajectory + 4 * sc.env_off - 3 * sc.idx;  // row 4k, column idx
+                tr[0] = z.x;
+                tr[p.n] = z.xd;
+                tr[2 * p.n] = z.th;
+                tr[3 * p.n] = z.thd;
+            }
+        }
+        sc.env_off += p.n;
+        sc.word_off += sc.words;
+    }
 }
 
-template <int PAIRS, bool LIMIT, bool CONTRACT>
+template <int PAIRS, bool LIMIT, bool CONTRACT, int STREAMS>
 __global__ void __launch_bounds__(64 * PAIRS) rollout_assisted_kernel(const __grid_constant__ RolloutParams p) {
     constexpr int kChunk = kChunkOf<PAIRS>;
     __shared__ PairBuffers<kChunk> s_buf[PAIRS];
@@ -87,17 +127,35 @@ __global__ void __launch_bounds__(64 * PAIRS) rollout_assisted_kernel(const __gr
 
     if (producer) {
         const FoldedKeys ka = fold_keys(make_keys(p.salt_a, env));
+        const int64_t words = (p.n + 31) >> 5;
         for (uint32_t c = 0; c <= n_chunks; ++c) {
             // chunk c is written while the consumer works on chunk c - 1 (other buffer); the
             // buffer written here was last read in chunk c - 2, which the barrier before closed
             if (c < n_chunks) {
                 const uint32_t b = c & 1u, tc = p.t0 + c * kChunk;
+                // The caller's actions: row (t - t0) of [T][words], one word per warp task. Lane s
+                // fetches the word of the chunk's step s, all in one load issued before the
+                // hashing below and used after it, when it has long arrived.
+                uint32_t my_word = 0u;
+                if (p.action_bits_in) {
+                    const uint32_t row = c * kChunk + lane;
+                    if (lane < (uint32_t)kChunk && row < p.T)
+                        my_word = __ldg(p.action_bits_in + (int64_t)row * words + task);
+                }
 #pragma unroll 4
                 for (int s = 0; s < kChunk; ++s) {
                     const uint32_t t = tc + s;
                     const State f = start_state_folded(kr, fold16(4u * (t + 1u)));
                     buf.start[b][s][lane] = make_float4(f.x, f.xd, f.th, f.thd);
-                    buf.force[b][s][lane] = force_from_signbit(action_signbit_folded(ka, fold16(t)));
+                    if (!p.action_bits_in)
+                        buf.force[b][s][lane] = force_from_signbit(action_signbit_folded(ka, fold16(t)));
+                }
+                if (p.action_bits_in) {
+#pragma unroll 4
+                    for (int s = 0; s < kChunk; ++s) {
+                        const uint32_t word = __shfl_sync(0xffffffffu, my_word, s);
+                        buf.force[b][s][lane] = force_from_signbit((word << (31u - lane)) & 0x80000000u);
+                    }
                 }
             }
             pair_barrier<PAIRS>(pair);
@@ -118,6 +176,15 @@ __global__ void __launch_bounds__(64 * PAIRS) rollout_assisted_kernel(const __gr
     // only the step limit needs the carried-in episode length inside the loop
     uint32_t cnt = 0u, begin = p.t0 - ((LIMIT && p.ep_len_io) ? p.ep_len_io[idx] : 0u);
     const uint32_t t_end = p.t0 + p.T;
+    StreamCursor sc;
+    sc.env_off = sc.idx = idx;
+    sc.word_off = task;  // one 32-env word per warp task
+    sc.words = (p.n + 31) >> 5;
+    sc.valid = valid;
+    sc.want_done = STREAMS == 2 && p.done_bits;
+    sc.want_act = STREAMS == 2 && p.action_bits;
+    sc.want_rew = STREAMS == 2 && p.reward_stream;
+    sc.want_traj = STREAMS == 2 && p.trajectory;
     pair_barrier<PAIRS>(pair);  // chunk 0 is there
     for (uint32_t c = 0; c < n_chunks; ++c) {
         const uint32_t b = c & 1u, tc = p.t0 + c * kChunk;
@@ -125,19 +192,19 @@ __global__ void __launch_bounds__(64 * PAIRS) rollout_assisted_kernel(const __gr
         if (c != 0u && steps == kChunk) {
 #pragma unroll kStepUnroll
             for (int s = 0; s < kChunk; ++s)
-                consume_step<true, LIMIT, CONTRACT>(buf, b, s, lane, tc + s + 1u, p.max_steps, z, cnt, begin);
+                consume_step<true, LIMIT, CONTRACT, STREAMS>(p, buf, b, s, lane, tc + s + 1u, sc, z, cnt, begin);
         } else {
             // The caller's initial state may hold any angle: the very first step tests it per
             // lane. From the second step on every angle is a survivor's (<= 0.2095) or a start
             // state's (<= 0.05).
             int s = 0;
             if (c == 0u) {
-                consume_step<false, LIMIT, CONTRACT>(buf, b, 0, lane, tc + 1u, p.max_steps, z, cnt, begin);
+                consume_step<false, LIMIT, CONTRACT, STREAMS>(p, buf, b, 0, lane, tc + 1u, sc, z, cnt, begin);
                 s = 1;
             }
 #pragma unroll kStepUnroll
             for (; s < steps; ++s)
-                consume_step<true, LIMIT, CONTRACT>(buf, b, s, lane, tc + s + 1u, p.max_steps, z, cnt, begin);
+                consume_step<true, LIMIT, CONTRACT, STREAMS>(p, buf, b, s, lane, tc + s + 1u, sc, z, cnt, begin);
         }
         pair_barrier<PAIRS>(pair);
     }
@@ -175,7 +242,9 @@ __global__ void __launch_bounds__(64 * PAIRS) rollout_assisted_kernel(const __gr
 }  // namespace
 
 bool rollout_assisted_applies(const RolloutParams &p, int policy, bool streams) {
-    if (policy != 0 || streams || p.action_bits_in || p.start_in) return false;
+    (void)streams;
+    // supplied actions replace whatever policy was named
+    if ((policy != 0 && !p.action_bits_in) || p.start_in) return false;
     if (g_tuning.rollout_coop == 4) return true;
     if (g_tuning.rollout_coop != 0 || g_tuning.rollout_ept != 0) return false;
     // up to ten pairs per SM (five CTAs of two pairs: 200 KB of shared memory; a sixth CTA would
@@ -187,12 +256,21 @@ bool rollout_assisted_applies(const RolloutParams &p, int policy, bool streams) 
 }
 
 namespace {
+template <int PAIRS, bool CONTRACT, int STREAMS>
+void launch_limit(const RolloutParams &p, unsigned grid, cudaStream_t s) {
+    if (p.max_steps)
+        rollout_assisted_kernel<PAIRS, true, CONTRACT, STREAMS><<<grid, 64 * PAIRS, 0, s>>>(p);
+    else
+        rollout_assisted_kernel<PAIRS, false, CONTRACT, STREAMS><<<grid, 64 * PAIRS, 0, s>>>(p);
+}
 template <int PAIRS, bool CONTRACT>
 void launch_pairs(const RolloutParams &p, unsigned grid, cudaStream_t s) {
-    if (p.max_steps)
-        rollout_assisted_kernel<PAIRS, true, CONTRACT><<<grid, 64 * PAIRS, 0, s>>>(p);
+    if (p.reward_stream && p.done_bits && !p.action_bits && !p.trajectory)
+        launch_limit<PAIRS, CONTRACT, 1>(p, grid, s);
+    else if (p.reward_stream || p.done_bits || p.action_bits || p.trajectory)
+        launch_limit<PAIRS, CONTRACT, 2>(p, grid, s);
     else
-        rollout_assisted_kernel<PAIRS, false, CONTRACT><<<grid, 64 * PAIRS, 0, s>>>(p);
+        launch_limit<PAIRS, CONTRACT, 0>(p, grid, s);
 }
 }  // namespace
 

@@ -39,11 +39,16 @@ def kernel(cp, coop, block=0):
         cp.cp_tune("rollout_block", 0)
 
 
-def rollout(cp, coop, n, T, seed, block=0, **kw):
+def rollout(cp, coop, n, T, seed, block=0, streams=(), **kw):
+    words = (n + 31) // 32
     out = {"ep_return_sum": torch.full((n,), -1.0, device="cuda"),
            "ep_count": torch.full((n,), -1, dtype=torch.int32, device="cuda"),
            "totals": torch.zeros(2, dtype=torch.int64, device="cuda"),
            "final_state": torch.zeros(4, n, device="cuda")}
+    shapes = {"done_bits": ((T, words), torch.int32), "action_bits": ((T, words), torch.int32),
+              "reward_stream": ((T, n), torch.float32), "trajectory": ((T, 4, n), torch.float32)}
+    for name in streams:
+        out[name] = torch.full(shapes[name][0], 7, dtype=shapes[name][1], device="cuda")
     with kernel(cp, coop, block):
         cp.cp_rollout_ex(n_envs=n, T=T, seed=seed, **kw, **out)
     torch.cuda.synchronize()
@@ -86,6 +91,37 @@ def test_contracted_arithmetic_same_bits_as_general_kernel(cp, oracle, limit):
     assert not np.array_equal(auto["final_state"], canonical["final_state"])    # the variant really ran
     o = oracle.rollout(n, T, seed, t0=3, max_episode_steps=limit)
     H.assert_returns_match(auto["ep_return_sum"], auto["ep_count"].view(np.uint32), o["ep_return_sum"], o["ep_count"])
+
+
+@pytest.mark.parametrize("streams", [("done_bits",), ("reward_stream", "done_bits"),
+                                     ("done_bits", "action_bits", "reward_stream", "trajectory")])
+@pytest.mark.parametrize("supplied", [False, True])
+def test_streams_and_supplied_actions(cp, oracle, streams, supplied):
+    n, T, seed, limit = 2101, 70, 8, 40
+    words = (n + 31) // 32
+    kw, ora_kw = {"t0": 2, "env_offset": 9, "max_episode_steps": limit}, {}
+    if supplied:
+        rng = np.random.default_rng(5)
+        bits = rng.integers(0, 1 << 32, (T, words), dtype=np.uint64).astype(np.uint32)
+        kw["action_bits_in"] = torch.from_numpy(bits.view(np.int32)).cuda()
+        ora_kw["action_bits_in"] = bits
+    general = rollout(cp, PER_LANE, n, T, seed, streams=streams, **kw)
+    for block in (64, 128):
+        assert_same_bits(rollout(cp, ASSISTED, n, T, seed, block, streams=streams, **kw), general)
+    auto = rollout(cp, 0, n, T, seed, streams=streams, **kw)
+    assert_same_bits(auto, general)
+    o = oracle.rollout(n, T, seed, t0=2, env_offset=9, max_episode_steps=limit, done_bits=True, action_bits=True,
+                       min_gap=True, **ora_kw)
+    same = (auto["ep_return_sum"] == o["ep_return_sum"]) & (auto["ep_count"].view(np.uint32) == o["ep_count"])
+    assert (same | (o["min_gap"] < 1e-5)).mean() >= 0.999
+    gd, od = H.unpack_bits(auto["done_bits"], n), H.unpack_bits(o["done_bits"], n)
+    assert np.array_equal(gd[:, same], od[:, same])
+    if "action_bits" in streams:
+        assert np.array_equal(H.unpack_bits(auto["action_bits"], n), H.unpack_bits(o["action_bits"], n))
+    if "reward_stream" in streams:
+        assert np.all(auto["reward_stream"] == 1.0)
+    if "trajectory" in streams:
+        assert np.array_equal(auto["trajectory"][-1], auto["final_state"])
 
 
 def test_callers_state_with_large_angles(cp, oracle):
