@@ -124,6 +124,27 @@ def test_streams_and_supplied_actions(cp, oracle, streams, supplied):
         assert np.array_equal(auto["trajectory"][-1], auto["final_state"])
 
 
+def test_forced_on_a_large_batch_and_at_the_end_of_time(cp, oracle):
+    """Far more pairs than fit on the chip at once (CTAs in waves), and the last steps the
+    32-bit step counter allows (the counter 4 * (t + 1) of the last start state wraps to 0 on
+    both sides)."""
+    n, T, seed = 300007, 20, 3
+    general = rollout(cp, PER_LANE, n, T, seed)
+    assert_same_bits(rollout(cp, ASSISTED, n, T, seed), general)
+    n, T = 5000, 45
+    t0 = (1 << 30) - T
+    general = rollout(cp, PER_LANE, n, T, seed, t0=t0, streams=("done_bits",))
+    got = rollout(cp, 0, n, T, seed, t0=t0, streams=("done_bits",))
+    assert_same_bits(got, general)
+    o = oracle.rollout(n, T, seed, t0=t0, done_bits=True, final_state=True)
+    H.assert_returns_match(got["ep_return_sum"], got["ep_count"].view(np.uint32), o["ep_return_sum"], o["ep_count"])
+    last_done = H.unpack_bits(o["done_bits"], n)[-1].astype(bool)
+    assert last_done.sum() > 50     # envs that restart at time 2^30 itself
+    assert np.array_equal(got["final_state"][:, last_done], o["final_state"][:, last_done])
+    with pytest.raises(cp.CartpoleError):
+        rollout(cp, 0, n, T + 1, seed, t0=t0)
+
+
 def test_callers_state_with_large_angles(cp, oracle):
     """Angles beyond the polynomial range in the initial state (some survive the first step): the
     first hand-over chunk must take the full-range sine and cosine."""
