@@ -605,6 +605,14 @@ def measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args) -> dict:
         if w.streams:
             entry["stream_write_gbs"] = rate * 4.125 / 1e9
             entry["stream_write_frac_of_hbm"] = rate * 4.125 / hbm
+        if name in ("c1", "paper"):
+            # a few warps on the whole chip: one warp's per-step latency is what is paid, so the
+            # fractions above say nothing; the figure to read is the time per step against the
+            # step's dependency chain (14 dependent float operations, about 60 SM cycles)
+            entry["kernel"] = "rollout_assisted_kernel"
+            entry["bound"] = "latency"
+            entry["ns_per_step"] = ms * 1e6 / T
+            entry["sm_cycles_per_step"] = ms * 1e-3 / T * peaks["sm_max_mhz"] * 1e6
         out[f"{name}_rollout"] = entry
         del outs
         torch.cuda.empty_cache()
