@@ -276,7 +276,21 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
                     __syncwarp();
 #pragma unroll
                     for (int j = 0; j < EPT; ++j) {
-                        if (listed[j]) {
+                        if (STREAMS == 0) {
+                            // A listed lane takes its four components with one predicated 16-byte
+                            // load straight into the state registers, written as such: the
+                            // compiler's form loads into temporaries and moves them (1,048,576 x
+                            // 500: 1.320 -> 1.302 ms; with the reward and done streams this form
+                            // costs six registers and 1.4 %, so those instances keep the other).
+                            const uint32_t out_addr = (uint32_t)__cvta_generic_to_shared(out_w) + slot[j] * 16u;
+                            asm volatile(
+                                "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %4, 0;\n\t"
+                                "@p ld.shared.v4.f32 {%0, %1, %2, %3}, [%5];\n\t}"
+                                : "+f"(z[j].x), "+f"(z[j].xd), "+f"(z[j].th), "+f"(z[j].thd)
+                                : "r"((uint32_t)listed[j]), "r"(out_addr)
+                                : "memory");
+                            if (done[j] && !listed[j]) z[j] = start_state_folded(kr[j], folded_4t1);
+                        } else if (listed[j]) {
                             const float4 s = reinterpret_cast<const float4 *>(out_w)[slot[j]];
                             z[j].x = s.x;
                             z[j].xd = s.y;
