@@ -38,16 +38,16 @@ SMS = 148
 # smsp__inst_executed.sum / (N*T) of the kernel the library launches by default at this size
 # (restarts by the whole warp): the issue slots it really occupies.
 ROLLOUT_OPS = {
-    "random": {"thread": 68.6, "slot": 83.8},
-    "linear": {"thread": 73.8, "slot": 76.7},
-    # here the default kernel's own thread count (88.2) is below the per-lane formulation's (91.9:
+    "random": {"thread": 68.6, "slot": 82.6},
+    "linear": {"thread": 73.8, "slot": 76.2},
+    # here the default kernel's own thread count (87.7) is below the per-lane formulation's (91.9:
     # one running stream pointer per env instead of one per two envs), so it is the algorithmic one
-    "linear+streams": {"thread": 88.2, "slot": 88.5},
-    "mlp": {"thread": 440.3, "slot": 462.9},
-    "random+contracted": {"thread": 55.6, "slot": 69.8},
+    "linear+streams": {"thread": 87.7, "slot": 87.8},
+    "mlp": {"thread": 440.3, "slot": 464.4},
+    "random+contracted": {"thread": 55.6, "slot": 68.6},
 }
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch in the same captures.
-ROLLOUT_DRAM_BYTES = {"random": 24.8e3, "linear": 24.3e3, "linear+streams": 381.9e6, "mlp": 22.0e3}
+ROLLOUT_DRAM_BYTES = {"random": 24.8e3, "linear": 24.6e3, "linear+streams": 381.1e6, "mlp": 21.8e3}
 STEP_DRAM_BYTES_16M = 568.2e6  # step_kernel at 16,777,216 envs, same kind of capture
 # Algorithmic HBM bytes per env-step of the step paths.
 STEP_BYTES = 37.0      # 16 in + 16 out + 4 reward + 1 done, hashed action

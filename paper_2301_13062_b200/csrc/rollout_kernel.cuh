@@ -289,16 +289,25 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
                                 : "+f"(z[j].x), "+f"(z[j].xd), "+f"(z[j].th), "+f"(z[j].thd)
                                 : "r"((uint32_t)listed[j]), "r"(out_addr)
                                 : "memory");
-                            if (done[j] && !listed[j]) z[j] = start_state_folded(kr[j], folded_4t1);
                         } else if (listed[j]) {
                             const float4 s = reinterpret_cast<const float4 *>(out_w)[slot[j]];
                             z[j].x = s.x;
                             z[j].xd = s.y;
                             z[j].th = s.z;
                             z[j].thd = s.w;
-                        } else if (done[j]) {  // more than CAP envs of this slot finished at once: rare
-                            z[j] = start_state_folded(kr[j], folded_4t1);
                         }
+                    }
+                    // More than CAP envs of one slot finished at once (rare): the surplus lanes hash
+                    // their own start states. Found by one warp-uniform test of the two masks; a
+                    // per-lane test costs a divergent branch per env slot on every pass through
+                    // the block (1.301 -> 1.287 ms on 1,048,576 x 500).
+                    bool surplus = false;
+#pragma unroll
+                    for (int j = 0; j < EPT; ++j) surplus = surplus || __popc(dmask[j]) > (int)CAP;
+                    if (surplus) {
+#pragma unroll
+                        for (int j = 0; j < EPT; ++j)
+                            if (done[j] && !listed[j]) z[j] = start_state_folded(kr[j], folded_4t1);
                     }
                     // No third barrier: the next write to keys_w follows this step's reads of it by
                     // the second barrier, and the next write to out_w follows the next first barrier.
