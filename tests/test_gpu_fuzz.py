@@ -104,18 +104,21 @@ def test_random_combination_against_oracle(cp, oracle, case):
         assert excused.sum() >= n - max(1, n // 500), (n, int((~excused).sum()))
     assert int(r["totals"][0]) == int(ret.astype(np.int64).sum())
     assert int(r["totals"][1]) == int(cnt.astype(np.int64).sum())
+    # An env that came within 1e-5 of a threshold or of a logit tie may have taken the other branch
+    # once and still show the same returns: per-step bits and states are compared on the others.
+    sure = same & (o["min_gap"] >= 1e-5)
     if "done_bits" in r:
         gd, od = H.unpack_bits(r["done_bits"], n), H.unpack_bits(o["done_bits"], n)
         assert np.array_equal(gd.sum(axis=0), cnt)
-        assert np.array_equal(gd[:, same], od[:, same]) or (contracted and feedback)
+        assert np.array_equal(gd[:, sure], od[:, sure]) or (contracted and feedback)
         if n % 32:
             assert not np.any(r["done_bits"].view(np.uint32)[:, -1] >> (n % 32))
     if "reward_stream" in r:
         assert np.all(r["reward_stream"] == 1.0)
     if "action_bits" in r and not (contracted and feedback):
         ga, oa = H.unpack_bits(r["action_bits"], n), H.unpack_bits(o["action_bits"], n)
-        assert np.array_equal(ga[:, same], oa[:, same])
+        assert np.array_equal(ga[:, sure], oa[:, sure])
     if not contracted:
-        live = same & np.isfinite(o["final_state"]).all(axis=0)
+        live = sure & np.isfinite(o["final_state"]).all(axis=0)
         err = np.abs(r["final_state"][:, live].astype(np.float64) - o["final_state"][:, live])
         assert err.size == 0 or err.max() < 1e-3   # trajectories that agree on every done flag stay together
