@@ -31,7 +31,7 @@ EXPORTS = [
     "cp_launch_count", "cp_selftest_sincos", "cp_last_error", "cp_version", "cp_step_unfused_noalloc",
     "cp_selftest_sincos_accuracy", "cp_selftest_arith", "cp_step_repeat", "cp_selftest_tame_div",
     "cp_rollout_ex", "cp_step_ex", "cp_rollout_host_shard", "cp_selftest_tanh", "cp_set_allocator",
-    "cp_calibrate_pipe",
+    "cp_calibrate_pipe", "cp_selftest_pair",
 ]
 CP_CALIBRATE_THREADS_PER_SM = 2048
 CP_NOALLOC_MAX_ENVS = 65536
@@ -111,6 +111,7 @@ def lib() -> C.CDLL:
             "cp_calibrate_pipe": (i64, [i32, p, p, i32]),
             "cp_selftest_arith": (i32, [p]),
             "cp_selftest_tame_div": (i32, [u32, p]),
+            "cp_selftest_pair": (i32, [C.c_uint64, u32, p]),
             "cp_last_error": (C.c_char_p, []),
             "cp_version": (C.c_char_p, []),
         }
@@ -436,6 +437,12 @@ def cp_selftest_tame_div(den_step: int, out) -> None:
     import torch
     _use_current_stream()
     _check(lib().cp_selftest_tame_div(den_step, _dptr(out, torch.int64)))
+
+
+def cp_selftest_pair(count: int, seed: int, out) -> None:
+    import torch
+    _use_current_stream()
+    _check(lib().cp_selftest_pair(count, seed, _dptr(out, torch.int64)))
 
 
 def cp_version() -> str:

@@ -22,7 +22,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcartpole.so")
 STAMP = os.path.join(HERE, "libcartpole.so.stamp")
 SOURCES = ["rollout_networks.cu", "rollout_networks_contracted.cu", "rollout_kernel.cu", "rollout_contracted.cu",
-           "rollout_assisted.cu", "capi.cu", "step_kernel.cu", "ladder_kernels.cu", "ladder_noalloc.cu"]
+           "rollout_assisted.cu", "rollout_deferred.cu", "capi.cu", "step_kernel.cu", "ladder_kernels.cu", "ladder_noalloc.cu"]
 HEADERS = ["cartpole_device.cuh", "cartpole_internal.h", "rollout_kernel.cuh", os.path.join("..", "..", "include", "cartpole.h")]
 
 NVCC_FLAGS = [

@@ -565,8 +565,12 @@ int cp_tune(const char *key, int value) {
         if (value != 0 && value != 1 && value != 2) return fail(CP_EINVAL, "rollout_ept must be 0, 1 or 2");
         cp::g_tuning.rollout_ept = value;
     } else if (!strcmp(key, "rollout_coop")) {
-        if (value < 0 || value > 4) return fail(CP_EINVAL, "rollout_coop must be 0..4");
+        if (value < 0 || value > 5) return fail(CP_EINVAL, "rollout_coop must be 0..5");
         cp::g_tuning.rollout_coop = value;
+    } else if (!strcmp(key, "rollout_defer")) {
+        if (value != 0 && value != 2 && value != 4 && value != 8)
+            return fail(CP_EINVAL, "rollout_defer must be 0, 2, 4 or 8");
+        cp::g_tuning.rollout_defer = value;
     } else if (!strcmp(key, "rollout_ctas_per_sm")) {
         if (value < 0 || value > 1024) return fail(CP_EINVAL, "rollout_ctas_per_sm must be 0..1024");
         cp::g_tuning.rollout_ctas_per_sm = value;
@@ -612,6 +616,13 @@ int cp_selftest_tanh(uint32_t lo_bits, uint32_t hi_bits, uint64_t *out) {
 int cp_selftest_arith(uint64_t *out) {
     if (!out || !is_aligned(out, 8)) return fail(CP_EINVAL, "out is NULL or misaligned");
     cudaError_t e = cp::launch_arith_selftest(reinterpret_cast<unsigned long long *>(out), tl_stream);
+    return e == cudaSuccess ? CP_OK : cuda_fail(e, "self-test launch");
+}
+
+int cp_selftest_pair(uint64_t count, uint32_t seed, uint64_t *out) {
+    if (!out || !is_aligned(out, 8)) return fail(CP_EINVAL, "out is NULL or misaligned");
+    if (count == 0) return fail(CP_EINVAL, "count must be >= 1");
+    cudaError_t e = cp::launch_pair_selftest(count, seed, reinterpret_cast<unsigned long long *>(out), tl_stream);
     return e == cudaSuccess ? CP_OK : cuda_fail(e, "self-test launch");
 }
 

@@ -309,6 +309,132 @@ __device__ __forceinline__ bool euler_step(State &z, float force) {
     return (fabsf(nx) > kXT) | (fabsf(nth) > kTT);
 }
 
+// ---- two environments per instruction (packed float32 arithmetic of sm_100a) ----
+// Blackwell issues mul / add / sub / fma on a PAIR of float32 values held in a 64-bit register
+// (mul.rn.f32x2 and friends). Each half is rounded exactly like the scalar .rn operation, so a
+// thread that owns two independent environments can run both dependency chains with one
+// instruction stream: the bits do not change, the issue slots of the float arithmetic halve.
+// Low half = environment slot 0, high half = slot 1.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 splat2(float c) { return pack2(c, c); }
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+
+struct StatePair {
+    f32x2 x, xd, th, thd;
+};
+__device__ __forceinline__ StatePair pack_states(const State &a, const State &b) {
+    StatePair z;
+    z.x = pack2(a.x, b.x);
+    z.xd = pack2(a.xd, b.xd);
+    z.th = pack2(a.th, b.th);
+    z.thd = pack2(a.thd, b.thd);
+    return z;
+}
+__device__ __forceinline__ void unpack_states(const StatePair &z, State &a, State &b) {
+    unpack2(z.x, a.x, b.x);
+    unpack2(z.xd, a.xd, b.xd);
+    unpack2(z.th, a.th, b.th);
+    unpack2(z.thd, a.thd, b.thd);
+}
+
+// div_mtot_core on both halves; -q * M + x is written q * (-M) + x (the product's sign flip is
+// exact, so the fused operation rounds the same real number).
+__device__ __forceinline__ f32x2 div_mtot_core2(f32x2 x) {
+    const f32x2 r = splat2(kRcpMTot);
+    const f32x2 q = mul2(x, r);
+    const f32x2 rem = fma2(q, splat2(-kMTot), x);
+    return fma2(rem, r, q);
+}
+
+// A product that feeds an addition. The assembler of CUDA 12.9 contracts a packed multiply whose
+// only use is a packed add / sub into one fused multiply-add even though both carry an explicit
+// .rn (which forbids exactly that for the scalar forms) and --fmad=false is given — measured on
+// the GPU: 13 % of random operand pairs then differ from the separately rounded result. It does
+// not touch a product that enters a fused multiply-add as the multiplicand, so such sums are
+// written  c + a*b  ==  fma(RN(-a*b), -1, c): negating a product is exact, and the fma adds
+// exactly RN(a*b). cp_selftest_pair compares the packed step with the scalar one bit for bit.
+__device__ __forceinline__ f32x2 add_product2(f32x2 c, f32x2 neg_product) {
+    return fma2(neg_product, splat2(-1.0f), c);
+}
+
+// euler_step<true> (both angles within the polynomial range) for two environments at once:
+// the same operations in the same order on each half, hence the same bits. Rewrites that keep
+// negations out of the packed instructions: see div_mtot_core2; the denominator of the
+// angular acceleration is formed with its sign flipped (RN(a - b) == -RN(b - a)), which is the
+// operand the remainder step of div_tame needs, while the reciprocal takes the positive value.
+__device__ __forceinline__ void euler_step_pair(StatePair &z, f32x2 force, bool &done0, bool &done1) {
+    const f32x2 zz = mul2(z.th, z.th);
+    const f32x2 sp = fma2(splat2(8.319973014e-03f), zz, splat2(-1.666664630e-01f));
+    const f32x2 s = fma2(mul2(sp, zz), z.th, z.th);
+    f32x2 cq = fma2(splat2(-1.387019176e-03f), zz, splat2(4.166663438e-02f));
+    cq = fma2(cq, zz, splat2(-0.5f));
+    const f32x2 c = fma2(cq, zz, splat2(1.0f));
+    // accel<true>
+    const f32x2 t0 = mul2(z.thd, z.thd);
+    const f32x2 nt1 = mul2(splat2(-kPML), t0);
+    const f32x2 nt2 = mul2(nt1, s);
+    const f32x2 t3 = add_product2(force, nt2);  // force + t2
+    const f32x2 temp = div_mtot_core2(t3);
+    const f32x2 n0 = mul2(splat2(kG), s);
+    const f32x2 n1 = mul2(c, temp);
+    const f32x2 num = add_product2(n0, n1);  // n0 - n1
+    const f32x2 d0 = mul2(c, c);
+    const f32x2 h1 = mul2(splat2(0.5f * kMPole), d0);
+    const f32x2 nden = sub2(div_mtot_core2(h1), splat2(0.5f * kFT));  // -den
+    float nd0, nd1, r0, r1;
+    unpack2(nden, nd0, nd1);
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r0) : "f"(-nd0));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r1) : "f"(-nd1));
+    const f32x2 r = pack2(r0, r1);
+    const f32x2 q = mul2(num, r);
+    const f32x2 rem = fma2(nden, q, num);
+    const f32x2 thacc = fma2(rem, r, q);
+    const f32x2 p0 = mul2(splat2(kPML), thacc);
+    const f32x2 p1 = mul2(p0, c);
+    const f32x2 xacc = sub2(temp, div_mtot_core2(p1));
+    const f32x2 ntau = splat2(-kTau);
+    const f32x2 nx = add_product2(z.x, mul2(ntau, z.xd));
+    const f32x2 nxd = add_product2(z.xd, mul2(ntau, xacc));
+    const f32x2 nth = add_product2(z.th, mul2(ntau, z.thd));
+    const f32x2 nthd = add_product2(z.thd, mul2(ntau, thacc));
+    z.x = nx;
+    z.xd = nxd;
+    z.th = nth;
+    z.thd = nthd;
+    float x0, x1, a0, a1;
+    unpack2(nx, x0, x1);
+    unpack2(nth, a0, a1);
+    done0 = (fabsf(x0) > kXT) | (fabsf(a0) > kTT);
+    done1 = (fabsf(x1) > kXT) | (fabsf(a1) > kTT);
+}
+
 // ---- contracted arithmetic (an optional, separately reported rollout variant) ----
 // The same step with the roundings a compiler allowed to contract would drop (the paper's
 // fused kernels are generated without a one-rounding-per-op promise, Sec. V-B/V-G): fused

@@ -52,8 +52,10 @@ struct LaunchTuning {
     int rollout_block = 0;        // 0: 128 for very small batches, 256 otherwise
     int rollout_ept = 0;          // 0: chosen per policy and batch size
     int rollout_coop = 0;         // 0: chosen per batch size; 1 restarts by the warp; 2 per lane (ept 1);
-                                  // 3 per lane, computed ahead; 4 handed over by a producer warp
+                                  // 3 per lane, computed ahead; 4 handed over by a producer warp;
+                                  // 5 deferred (two envs per thread, own clock per env, restarts every few trips)
     int rollout_ctas_per_sm = 0;  // 0: one task per warp (non-persistent grid)
+    int rollout_defer = 0;        // deferred-restart kernel: trips between restart passes (0: 4; 2, 4 or 8)
     int step_block = 64;
     // Below this many envs the one-env-per-thread kernel is used: a small batch is latency-bound,
     // and four envs in sequence per thread take longer than four times as many threads
@@ -79,6 +81,9 @@ cudaError_t launch_rollout_contracted(RolloutParams &p, int policy, bool streams
 // the producer-assisted kernel for very small batches, and whether a call is one it covers
 bool rollout_assisted_applies(const RolloutParams &p, int policy, bool streams);
 cudaError_t launch_rollout_assisted(RolloutParams &p, bool contracted, cudaStream_t s);
+// the deferred-restart kernel (large batches, no per-step streams), and whether a call is one it covers
+bool rollout_deferred_applies(const RolloutParams &p, int policy, bool streams);
+cudaError_t launch_rollout_deferred(RolloutParams &p, int policy, cudaStream_t s);
 // the MLP policies (kinds 2, 4, 5, 7), canonical and contracted arithmetic; mode and shape as
 // chosen by launch_rollout_arith
 cudaError_t launch_rollout_networks(RolloutParams &p, int policy, int mode, int shape, cudaStream_t s);
@@ -90,6 +95,7 @@ cudaError_t launch_sincos_accuracy(uint32_t lo_bits, uint32_t hi_bits, unsigned 
 cudaError_t launch_tanh_accuracy(uint32_t lo_bits, uint32_t hi_bits, unsigned long long *out, cudaStream_t s);
 cudaError_t launch_pipe_rate(int kind, const float *seed, float *sink, int iters, int *threads, cudaStream_t s);
 cudaError_t launch_arith_selftest(unsigned long long *out, cudaStream_t s);
+cudaError_t launch_pair_selftest(unsigned long long count, uint32_t seed, unsigned long long *out, cudaStream_t s);
 cudaError_t launch_tame_div_selftest(uint32_t den_step, unsigned long long *out, cudaStream_t s);
 
 // The per-op ladder. Workspace layout is private to ladder_kernels.cu.

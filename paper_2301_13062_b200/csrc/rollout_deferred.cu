@@ -1,0 +1,243 @@
+// Fused rollout with deferred restarts (paper Sec. V-D / V-G: all steps in one launch; Sec. V-A:
+// the random values must not stand in the step's way).
+//
+// The general rollout kernel restarts finished environments after every step, and with the
+// random policy some environment of a warp finishes on 95 % of the steps, so the restart
+// machinery (ballots, ranks, shared-memory exchange, or four hashes issued for the whole warp) is
+// paid on practically every step although 4.5 % of the environments need it. Nothing forces an
+// environment to restart in the same loop trip it finished in: every random value is a function
+// of (seed, env, global time), so an environment that waits keeps its own clock and simply
+// continues later from the start state of the time it finished at. Here
+//
+//   * a thread owns two environments ("slots"), stepped together by the packed float32
+//     instructions of sm_100a (euler_step_pair: one instruction, two independent roundings);
+//   * every slot has its own global time t; a slot whose episode ended stops counting and idles
+//     (its half of the packed arithmetic computes values nobody reads);
+//   * every K trips the idle slots hash their start state of time t and go on. A slot therefore
+//     lags behind the trip counter by the trips it idled (about (K-1)/2 per episode), and the
+//     loop runs until the slowest slot of the warp has done its T steps.
+//
+// Every environment still takes exactly the steps t0 .. t0+T-1 with the actions and start states
+// of those times: the results are bit for bit those of the other work shapes (the tests compare
+// them). What changes is the issue count: restart work drops from every trip to every K-th, and
+// the price is idle slots (about 7 % at K = 4 with the random policy's 22-step episodes) and a
+// ragged end.
+//
+// Scope: no per-step output streams (they are rows of global time) and no episode step limit;
+// hashed actions, the shared linear policy or one linear policy per environment; canonical
+// arithmetic. Everything else takes the general kernel.
+//
+// No warp waits for another one and nothing spins: the loop's trip count is bounded by the
+// launch parameters (every trip block advances every unfinished slot by at least one step).
+#include <type_traits>
+
+#include "cartpole_device.cuh"
+#include "cartpole_internal.h"
+
+namespace cp {
+
+namespace {
+
+template <int POLICY>
+__device__ __forceinline__ uint32_t deferred_action(const RolloutParams &p, const FoldedKeys &ka, const LinearW &own,
+                                                    uint32_t t, const State &z) {
+    if (POLICY == 0) return action_signbit_folded(ka, fold16(t));
+    if (POLICY == 1) return linear_action(*reinterpret_cast<const LinearW *>(p.w), z);
+    return linear_action(own, z);
+}
+
+// POLICY: 0 hashed actions, 1 shared linear policy, 6 one linear policy per environment.
+// K: trips between restart passes.
+template <int POLICY, int K>
+__global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_constant__ RolloutParams p) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const int64_t task = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    unsigned long long tot_ret = 0, tot_cnt = 0;
+    if (task < p.n_tasks) {  // warp-uniform
+        const int64_t base = task * 64;
+        const uint32_t t_end = p.t0 + p.T;
+        FoldedKeys ka[2], kr[2];
+        LinearW own[POLICY == 6 ? 2 : 1];
+        uint32_t t[2], cnt[2], begin[2];
+        bool act[2];
+        State z0[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            int64_t idx = base + j * 32 + lane;
+            if (idx >= p.n) idx = p.n - 1;  // idle lanes shadow the last environment and store nothing
+            const uint32_t env = p.env_offset + (uint32_t)idx;
+            if (POLICY == 0) ka[j] = fold_keys(make_keys(p.salt_a, env));
+            kr[j] = fold_keys(make_keys(p.salt_r, env));
+            if (p.init_planes) {
+                z0[j].x = p.init_planes[idx];
+                z0[j].xd = p.init_planes[p.init_stride + idx];
+                z0[j].th = p.init_planes[2 * p.init_stride + idx];
+                z0[j].thd = p.init_planes[3 * p.init_stride + idx];
+            } else {
+                z0[j] = start_state_folded(kr[j], fold16(4u * p.t0));
+            }
+            if (POLICY == 6) {
+                LinearW &o = own[POLICY == 6 ? j : 0];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) o.w[q / 4][q % 4] = p.env_weights[(int64_t)q * p.n + idx];
+                o.b[0] = p.env_weights[8 * p.n + idx];
+                o.b[1] = p.env_weights[9 * p.n + idx];
+            }
+            t[j] = p.t0;
+            cnt[j] = 0u;
+            begin[j] = p.t0;
+            act[j] = true;
+        }
+        StatePair zz = pack_states(z0[0], z0[1]);
+
+        // Slot j has done its last step (its clock reached t_end): results out, slot retired.
+        auto finalize = [&](int j, bool done_now) {
+            State a, b;
+            unpack_states(zz, a, b);
+            State &mine = j ? b : a;
+            // an episode that ended on the very last step hands over the start state of t_end
+            if (done_now) mine = start_state_folded(kr[j], fold16(4u * t_end));
+            zz = pack_states(a, b);
+            const int64_t idx = base + j * 32 + lane;
+            if (idx < p.n) {
+                // sum of the returns of the completed episodes = last termination time - time the
+                // first of them began (every step earns reward 1)
+                const uint32_t carried = p.ep_len_io ? p.ep_len_io[idx] : 0u;
+                const uint32_t ret = cnt[j] ? begin[j] - (p.t0 - carried) : 0u;
+                const uint32_t running = t_end - begin[j] + (cnt[j] == 0u ? carried : 0u);
+                if (p.ep_return_sum) p.ep_return_sum[idx] = (float)ret;
+                if (p.ep_count) p.ep_count[idx] = cnt[j];
+                if (p.ep_len_io) p.ep_len_io[idx] = running;
+                if (p.out_planes) {
+                    p.out_planes[idx] = mine.x;
+                    p.out_planes[p.out_stride + idx] = mine.xd;
+                    p.out_planes[2 * p.out_stride + idx] = mine.th;
+                    p.out_planes[3 * p.out_stride + idx] = mine.thd;
+                }
+                tot_ret += ret;
+                tot_cnt += cnt[j];
+            }
+        };
+
+        // Bookkeeping of slot j after a trip in which its environment (if it was stepping) either
+        // survived or ended (done_now). TAIL: the slot may have done its last step.
+        auto after_step = [&](auto tail, int j, bool done_now) {
+            constexpr bool TAIL = decltype(tail)::value;
+            const bool live = act[j];
+            if (live) t[j] += 1u;
+            const bool ended = live && done_now;
+            if (ended) {
+                cnt[j] += 1u;
+                begin[j] = t[j];
+            }
+            act[j] = live && !done_now;
+            if (TAIL) {
+                if (live && t[j] == t_end) {
+                    finalize(j, done_now);
+                    act[j] = false;
+                }
+            }
+        };
+
+        // Idle slots that still have steps to do take the start state of their own time.
+        auto restart_pass = [&](auto tail) {
+            constexpr bool TAIL = decltype(tail)::value;
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                if (!act[j] && (!TAIL || t[j] != t_end)) {
+                    State a, b;
+                    unpack_states(zz, a, b);
+                    (j ? b : a) = start_state_folded(kr[j], fold16(4u * t[j]));
+                    zz = pack_states(a, b);
+                    act[j] = true;
+                }
+            }
+        };
+
+        auto trip = [&](auto tail) {
+            State a, b;
+            unpack_states(zz, a, b);
+            const uint32_t sb0 = deferred_action<POLICY>(p, ka[0], own[0], t[0], a);
+            const uint32_t sb1 = deferred_action<POLICY>(p, ka[POLICY == 0 ? 1 : 0], own[POLICY == 6 ? 1 : 0], t[1], b);
+            bool d0, d1;
+            euler_step_pair(zz, pack2(force_from_signbit(sb0), force_from_signbit(sb1)), d0, d1);
+            after_step(tail, 0, d0);
+            after_step(tail, 1, d1);
+        };
+
+        uint32_t trips = 0;  // trips made; no slot's clock is ahead of t0 + trips
+        if (p.init_planes) {
+            // A caller's states may hold any angle: the first trip uses the general scalar step.
+            // From then on every stepping slot is a survivor (|theta| <= 0.2095) or a fresh
+            // start state (|theta| <= 0.05), which is the packed step's domain.
+            State a, b;
+            unpack_states(zz, a, b);
+            const uint32_t sb0 = deferred_action<POLICY>(p, ka[0], own[0], t[0], a);
+            const uint32_t sb1 = deferred_action<POLICY>(p, ka[POLICY == 0 ? 1 : 0], own[POLICY == 6 ? 1 : 0], t[1], b);
+            const bool d0 = euler_step<false>(a, force_from_signbit(sb0));
+            const bool d1 = euler_step<false>(b, force_from_signbit(sb1));
+            zz = pack_states(a, b);
+            after_step(std::true_type{}, 0, d0);
+            after_step(std::true_type{}, 1, d1);
+            restart_pass(std::true_type{});
+            trips = 1;
+        }
+        // Main part: after these trips no clock can have reached t_end yet, so no slot can retire.
+        while (trips + K <= p.T - 1u) {
+#pragma unroll
+            for (int k = 0; k < K; ++k) trip(std::false_type{});
+            restart_pass(std::false_type{});
+            trips += K;
+        }
+        // Tail: slots retire as their clocks reach t_end. Every block of K trips advances every
+        // unretired slot by at least one step, so p.T blocks always suffice.
+        for (uint32_t block = 0; block <= p.T; ++block) {
+            if (__all_sync(0xffffffffu, t[0] == t_end && t[1] == t_end)) break;
+#pragma unroll
+            for (int k = 0; k < K; ++k) trip(std::true_type{});
+            restart_pass(std::true_type{});
+        }
+    }
+
+    if (p.totals) {
+        for (int o = 16; o > 0; o >>= 1) {
+            tot_ret += __shfl_down_sync(0xffffffffu, tot_ret, o);
+            tot_cnt += __shfl_down_sync(0xffffffffu, tot_cnt, o);
+        }
+        if (lane == 0 && (tot_ret | tot_cnt)) {
+            atomicAdd(p.totals, tot_ret);
+            atomicAdd(p.totals + 1, tot_cnt);
+        }
+    }
+}
+
+template <int POLICY>
+cudaError_t launch_k(RolloutParams &p, int k, cudaStream_t s) {
+    p.n_tasks = (p.n + 63) / 64;
+    int64_t grid = (p.n_tasks + 7) / 8;
+    if (grid > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    switch (k) {
+        case 2: rollout_deferred_kernel<POLICY, 2><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        case 8: rollout_deferred_kernel<POLICY, 8><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        default: rollout_deferred_kernel<POLICY, 4><<<(unsigned)grid, 256, 0, s>>>(p); break;
+    }
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool rollout_deferred_applies(const RolloutParams &p, int policy, bool streams) {
+    return !streams && p.max_steps == 0 && !p.action_bits_in && !p.start_in && (policy == 0 || policy == 1 || policy == 6);
+}
+
+cudaError_t launch_rollout_deferred(RolloutParams &p, int policy, cudaStream_t s) {
+    const int k = g_tuning.rollout_defer > 0 ? g_tuning.rollout_defer : 4;
+    switch (policy) {
+        case 0: return launch_k<0>(p, k, s);
+        case 1: return launch_k<1>(p, k, s);
+        default: return launch_k<6>(p, k, s);
+    }
+}
+
+}  // namespace cp

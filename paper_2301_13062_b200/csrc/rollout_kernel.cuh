@@ -80,6 +80,11 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
     constexpr bool COOP = SHAPE == 1 || SHAPE == 2;
     constexpr bool AHEAD = SHAPE == 3;
     constexpr bool START_IN = SHAPE == 4;
+#ifdef CP_EXP_NOPAIR
+    constexpr bool PAIR = false;
+#else
+    constexpr bool PAIR = SHAPE == 2 && !CONTRACT;  // packed two-env arithmetic
+#endif
     const uint32_t lane = threadIdx.x & 31u;
     // Per warp: key pairs of up to 8 finished envs, and their 8 x 4 start-state components.
     __shared__ uint2 s_keys[COOP ? kMaxWarpsPerCta : 1][8];
@@ -209,6 +214,7 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
                     fresh = start_state_folded(kr[j], folded_4t1);
                     asm volatile("" : "+f"(fresh.x), "+f"(fresh.xd), "+f"(fresh.th), "+f"(fresh.thd));
                 }
+                if (PAIR && small_all) continue;  // both envs step together below
                 const float force = force_from_signbit(sb[j]);
                 // warp-uniform; the per-lane shapes and the contracted arithmetic keep the per-lane
                 // test (measured faster there: 2,048 x 10,000 loses 6 % with the flag)
@@ -231,6 +237,19 @@ __global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLL
                     } else {
                         z[j] = start_state_folded(kr[j], folded_4t1);
                     }
+                }
+            }
+
+            if (PAIR && small_all) {
+                // Two envs per thread, canonical arithmetic, every angle in the polynomial range:
+                // one packed instruction steps both envs (same operations, same bits).
+                StatePair zz = pack_states(z[0], z[EPT - 1]);
+                euler_step_pair(zz, pack2(force_from_signbit(sb[0]), force_from_signbit(sb[EPT - 1])), done[0],
+                                done[EPT - 1]);
+                unpack_states(zz, z[0], z[EPT - 1]);
+                if (LIMIT) {
+#pragma unroll
+                    for (int j = 0; j < EPT; ++j) done[j] |= (t1 - begin[j]) >= p.max_steps;
                 }
             }
 
@@ -463,6 +482,7 @@ cudaError_t launch_rollout_arith(RolloutParams &p, int policy, bool streams, cud
     const bool heavy = policy == 2 || policy == 4 || policy == 5 || policy == 6 || policy == 7;
     int ept = g_tuning.rollout_ept;      // 0 auto, 1, 2
     int coop = g_tuning.rollout_coop;    // 0 auto, 1 cooperative, 2 per lane, 3 per lane and ahead
+    if (coop == 5) coop = 0;  // the deferred-restart kernel does not cover this call: default shape
     if (ept == 0) ept = (small || heavy || coop >= 2) ? 1 : 2;
     // at most two warps per scheduler and short episodes: start states computed ahead (measured:
     // 2,048 x 10,000 1.49 vs 1.65 ms, 32,768 x 5,000 0.75 vs 0.83 ms; slower from 65,536 envs on,

@@ -427,6 +427,63 @@ cudaError_t launch_pipe_rate(int kind, const float *seed, float *sink, int iters
     return cudaGetLastError();
 }
 
+// ---- self-test: the packed two-environment step against the scalar step ----
+// count pseudo-random pairs of states from the domain the packed step is used on (|theta| <= 0.22)
+// and a little beyond what an episode visits in the other components; every pair is stepped by
+// euler_step_pair and, half by half, by euler_step<true>. out[0] += pairs whose eight new state
+// components or two termination flags differ in any bit, out[1] += pairs tested.
+__global__ void pair_selftest_kernel(unsigned long long count, uint32_t seed, unsigned long long *out) {
+    unsigned long long bad = 0, seen = 0;
+    const uint32_t s0 = salt(seed, 7u);
+    for (unsigned long long k = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; k < count;
+         k += (unsigned long long)gridDim.x * blockDim.x) {
+        const Keys key = make_keys(s0 ^ (uint32_t)(k >> 32), (uint32_t)k);
+        float u[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) u[i] = (float)(step_hash(key, (uint32_t)i) >> 8) * 1.1920929e-07f - 1.0f;  // [-1, 1)
+        const uint32_t bits = step_hash(key, 8u);
+        // every fourth pair at the scale of start states, the others across the whole live range
+        const float scale = (bits & 3u) ? 1.0f : 0.25f;
+        State a, b;
+        a.x = u[0] * 2.5f * scale;
+        a.xd = u[1] * 4.0f * scale;
+        a.th = u[2] * kSmallAngle * scale;
+        a.thd = u[3] * 22.0f * scale;
+        b.x = u[4] * 2.5f * scale;
+        b.xd = u[5] * 4.0f * scale;
+        b.th = u[6] * kSmallAngle * scale;
+        b.thd = u[7] * 22.0f * scale;
+        const float fa = force_from_signbit((bits << 8) & 0x80000000u), fb = force_from_signbit((bits << 9) & 0x80000000u);
+        StatePair zz = pack_states(a, b);
+        bool pd0, pd1;
+        euler_step_pair(zz, pack2(fa, fb), pd0, pd1);
+        State pa, pb;
+        unpack_states(zz, pa, pb);
+        const bool d0 = euler_step<true>(a, fa), d1 = euler_step<true>(b, fb);
+        const bool same = __float_as_uint(pa.x) == __float_as_uint(a.x) && __float_as_uint(pa.xd) == __float_as_uint(a.xd) &&
+                          __float_as_uint(pa.th) == __float_as_uint(a.th) && __float_as_uint(pa.thd) == __float_as_uint(a.thd) &&
+                          __float_as_uint(pb.x) == __float_as_uint(b.x) && __float_as_uint(pb.xd) == __float_as_uint(b.xd) &&
+                          __float_as_uint(pb.th) == __float_as_uint(b.th) && __float_as_uint(pb.thd) == __float_as_uint(b.thd) &&
+                          pd0 == d0 && pd1 == d1;
+        bad += !same;
+        seen += 1;
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        bad += __shfl_down_sync(0xffffffffu, bad, o);
+        seen += __shfl_down_sync(0xffffffffu, seen, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        if (bad) atomicAdd(out, bad);
+        atomicAdd(out + 1, seen);
+    }
+}
+
+cudaError_t launch_pair_selftest(unsigned long long count, uint32_t seed, unsigned long long *out, cudaStream_t s) {
+    pair_selftest_kernel<<<sm_count() * 8, 256, 0, s>>>(count, seed, out);
+    count_launch();
+    return cudaGetLastError();
+}
+
 cudaError_t launch_arith_selftest(unsigned long long *out, cudaStream_t s) {
     arith_selftest_kernel<<<sm_count() * 8, 256, 0, s>>>(out);
     count_launch();

@@ -28,7 +28,7 @@ REL_TOL = 2e-6
 # kernel whose helper warps hash actions and start states ahead of the stepping warps (it covers
 # hashed actions without streams or step limit; other calls fall to the first shape). The
 # library picks one by batch size and policy; tests force each of them on small batches.
-SHAPES = [(1, 2), (1, 3), (1, 1), (2, 1), (1, 4)]
+SHAPES = [(1, 2), (1, 3), (1, 1), (2, 1), (1, 4), (2, 5)]
 
 
 @contextlib.contextmanager

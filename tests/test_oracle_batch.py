@@ -5,12 +5,11 @@ calls composed in Python), structural invariants of the episode bookkeeping,
 exact-rational evaluation of the policy FMA chains and stored aggregates of the
 smallest benchmark configuration.
 """
-from fractions import Fraction
-
 import numpy as np
 import pytest
 
 from paper_2301_13062_b200 import inputs
+from tests.exact_arith import fma_chain_exact
 
 
 def brute_step(oracle, planes, seed, t, action=None, env_offset=0):
@@ -136,41 +135,13 @@ def test_config1_aggregates(oracle):
 
 
 # ------------------------------------------------------------------ policies
-def _fma_chain_exact(ws, xs, b):
-    """fl32(w*x + acc) with a single rounding per term, via exact rationals."""
-    acc = Fraction(float(b))
-    for w, x in zip(ws, xs):
-        exact = Fraction(float(w)) * Fraction(float(x)) + acc
-        # round-to-nearest-even to float32: float() rounds the rational to f64 first, which could
-        # double-round; use numpy longdouble-free route: scale to an integer significand.
-        acc = Fraction(float(_round_f32(exact)))
-    return np.float32(float(acc))
-
-
-def _round_f32(q: Fraction) -> np.float32:
-    if q == 0:
-        return np.float32(0.0)
-    sign = -1 if q < 0 else 1
-    q = abs(q)
-    e = q.numerator.bit_length() - q.denominator.bit_length()
-    if Fraction(2) ** e > q:
-        e -= 1
-    e = max(e, -126)
-    scaled = q / Fraction(2) ** (e - 23)  # significand as a rational in [2^23, 2^24)
-    fl = scaled.numerator // scaled.denominator
-    rem = scaled - fl
-    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and fl % 2 == 1):
-        fl += 1
-    return np.float32(sign * float(Fraction(fl) * Fraction(2) ** (e - 23)))
-
-
 def test_linear_policy_is_an_fma_chain(oracle):
     w = inputs.policy_weights(inputs.POLICY_LINEAR, 1)
     zs = inputs.random_states(200, seed=2, spread="live")
     for i in range(zs.shape[1]):
         got = oracle.linear_logits(w, zs[:, i])
         for k in range(2):
-            want = _fma_chain_exact(w[4 * k:4 * k + 4], zs[:, i], w[8 + k])
+            want = fma_chain_exact(w[4 * k:4 * k + 4], zs[:, i], w[8 + k])
             assert got[k] == want
 
 
