@@ -369,11 +369,14 @@ int cp_selftest_pair(uint64_t count, uint32_t seed, uint64_t *out);
 /* Calibration of the roofline denominators (a measurement aid; the paper has no counterpart):
  * enqueue one launch in which every thread executes
  * iters rounds of eight independent chains of one instruction kind — 0: float32 fused
- * multiply-add, 1: 32-bit integer multiply-add, 2: the special-function reciprocal — on a grid of
+ * multiply-add, 1: 32-bit integer multiply-add, 2: the special-function reciprocal, 3: the packed
+ * float32 fused multiply-add of sm_100a (two results per instruction) — or of a half-and-half mix:
+ * 4: packed + scalar float, 5: packed float + integer multiply-add, 6: packed float + integer
+ * logic, 7: scalar float + integer multiply-add (which pipes share hardware) — on a grid of
  * 8 CTAs x 256 threads per SM. seed DEVICE [10] floats (ordinary magnitudes, e.g. 0.5 .. 1.5),
  * sink DEVICE [CP_CALIBRATE_THREADS_PER_SM x SM count] floats, overwritten. Returns the number of
- * thread-instructions of the measured kind the launch executes (the caller times the launch), or
- * a negative error code. */
+ * thread-instructions the chains execute (a packed instruction counts once; kind 6 issues two
+ * logic instructions per counted one; the caller times the launch), or a negative error code. */
 #define CP_CALIBRATE_THREADS_PER_SM 2048
 int64_t cp_calibrate_pipe(int kind, const float *seed, float *sink, int iters);
 

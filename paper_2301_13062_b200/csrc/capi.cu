@@ -568,8 +568,8 @@ int cp_tune(const char *key, int value) {
         if (value < 0 || value > 5) return fail(CP_EINVAL, "rollout_coop must be 0..5");
         cp::g_tuning.rollout_coop = value;
     } else if (!strcmp(key, "rollout_defer")) {
-        if (value != 0 && value != 2 && value != 4 && value != 8)
-            return fail(CP_EINVAL, "rollout_defer must be 0, 2, 4 or 8");
+        if (value != 0 && value != 2 && value != 3 && value != 4 && value != 6 && value != 8)
+            return fail(CP_EINVAL, "rollout_defer must be 0, 2, 3, 4, 6 or 8");
         cp::g_tuning.rollout_defer = value;
     } else if (!strcmp(key, "rollout_ctas_per_sm")) {
         if (value < 0 || value > 1024) return fail(CP_EINVAL, "rollout_ctas_per_sm must be 0..1024");
@@ -634,7 +634,7 @@ int cp_selftest_tame_div(uint32_t den_step, uint64_t *out) {
 }
 
 int64_t cp_calibrate_pipe(int kind, const float *seed, float *sink, int iters) {
-    if (kind < 0 || kind > 2) return fail(CP_EINVAL, "kind must be 0 (FFMA), 1 (IMAD) or 2 (MUFU)");
+    if (kind < 0 || kind > 7) return fail(CP_EINVAL, "kind must be 0..7 (FFMA, IMAD, MUFU, FFMA2, and four mixes)");
     if (!seed || !sink || !is_aligned(seed, 4) || !is_aligned(sink, 4)) return fail(CP_EINVAL, "seed or sink is NULL or misaligned");
     if (iters < 1 || iters > (1 << 24)) return fail(CP_EINVAL, "iters must be in [1, 2^24]");
     int threads = 0;

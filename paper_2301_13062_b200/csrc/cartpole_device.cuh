@@ -198,29 +198,26 @@ __device__ __forceinline__ void sin_cos(float th, float &s, float &c) {
 }
 
 // ---- division by the total mass ----
-// x / 1.1f with the correctly rounded result of IEEE division, in three operations instead of
-// the general division sequence: q = x*r, rem = x - q*d (exact, fused), q' = q + rem*r with
-// r = RN(1/d). For d = 1.1f this equals __fdiv_rn(x, d) for EVERY finite x with |x| >= 2^-104
-// and for +0 (checked over all 2^32 bit patterns by cp_selftest_arith); tiny, -0, infinite and
-// NaN inputs take the general division.
-constexpr float kRcpMTot = 0.9090908765792847f;  // RN(1 / 1.1f) = 0x3F68BA2E
+// x / 1.1f with the correctly rounded result of IEEE division, in two operations instead of the
+// general division sequence: with r = RN(1/d) and e = RN(1/d - r) (the reciprocal in two
+// float32 pieces), q = fma(x, r, x*e). The sum x*r + RN(x*e) misses x/d by about 2^-48 of its
+// size, and for d = 1.1f no quotient lies that close to a rounding boundary: the result equals
+// __fdiv_rn(x, d) for EVERY finite x with |x| >= 2^-100, for both zeros, infinities and NaN
+// (checked over all 2^32 bit patterns by cp_selftest_arith); tiny inputs, where x*e underflows,
+// take the general division.
+constexpr float kRcpMTot = 0.9090908765792847f;       // RN(1 / 1.1f) = 0x3F68BA2E
+constexpr float kRcpMTotLo = 1.280761008359832e-08f;  // RN(1 / 1.1f - kRcpMTot) = 0x325C0877
 __device__ __forceinline__ float div_mtot_core(float x) {
-    const float q = __fmul_rn(x, kRcpMTot);
-    const float rem = __fmaf_rn(-q, kMTot, x);
-    return __fmaf_rn(rem, kRcpMTot, q);
+    return __fmaf_rn(x, kRcpMTot, __fmul_rn(x, kRcpMTotLo));
 }
-// x is known to be +0, NaN, infinite, or of magnitude >= 2^-100 (never tiny, never -0).
-__device__ __forceinline__ float div_mtot_not_tiny(float x) {
-    if (fabsf(x) <= 3.402823466e+38f) return div_mtot_core(x);
-    return __fdiv_rn(x, kMTot);
-}
+// x is known to be a zero, NaN, infinite, or of magnitude >= 2^-100 (never tiny).
+__device__ __forceinline__ float div_mtot_not_tiny(float x) { return div_mtot_core(x); }
 // x is known to be NaN or of magnitude in [2^-100, FLT_MAX] (or +0).
 __device__ __forceinline__ float div_mtot_normal(float x) { return div_mtot_core(x); }
 // any x
 __device__ __forceinline__ float div_mtot(float x) {
-    const float ax = fabsf(x);
-    if (ax >= 7.888609052e-31f && ax <= 3.402823466e+38f) return div_mtot_core(x);  // 2^-100 .. FLT_MAX
-    return __fdiv_rn(x, kMTot);
+    if (fabsf(x) >= 7.888609052e-31f) return div_mtot_core(x);  // 2^-100 and up, infinities included
+    return __fdiv_rn(x, kMTot);                                   // tiny, zero, NaN
 }
 
 // Accelerations (canonical op order; one rounding per op).
@@ -232,7 +229,7 @@ __device__ __forceinline__ float div_mtot(float x) {
 // the accelerations are never seen (x' and theta' do not depend on them). For |theta| <= 0.22
 // and |theta_dot| <= 21.5: |s| <= 0.2183, c >= 0.9759, t3 = +-10 + t2 lies in +-[4.95, 15.05],
 // |num| >= 0.9759*4.95/1.1 - 9.8*0.2183 > 2.2, |num| < 16 and |p1| > 0.17: every operand of a
-// division by 1.1 is a normal number far from the range limits, where the three-operation form
+// division by 1.1 is a normal number far from the range limits, where the two-operation form
 // is exact, so no range test is needed. TAME = false makes no assumption and tests each operand.
 // num / den for the operands a tame state produces: den = 0.5*(4/3 - 0.1*c^2/1.1) with
 // c in [0.9689, 1] lies in [0.62121, 0.62400] and |num| in [2.2, 16). On the superset
@@ -364,20 +361,17 @@ __device__ __forceinline__ void unpack_states(const StatePair &z, State &a, Stat
     unpack2(z.thd, a.thd, b.thd);
 }
 
-// div_mtot_core on both halves; -q * M + x is written q * (-M) + x (the product's sign flip is
-// exact, so the fused operation rounds the same real number).
+// div_mtot_core on both halves (a product that enters a fused multiply-add as the addend stays a
+// separate rounding, see add_product2).
 __device__ __forceinline__ f32x2 div_mtot_core2(f32x2 x) {
-    const f32x2 r = splat2(kRcpMTot);
-    const f32x2 q = mul2(x, r);
-    const f32x2 rem = fma2(q, splat2(-kMTot), x);
-    return fma2(rem, r, q);
+    return fma2(x, splat2(kRcpMTot), mul2(x, splat2(kRcpMTotLo)));
 }
 
 // A product that feeds an addition. The assembler of CUDA 12.9 contracts a packed multiply whose
 // only use is a packed add / sub into one fused multiply-add even though both carry an explicit
 // .rn (which forbids exactly that for the scalar forms) and --fmad=false is given — measured on
 // the GPU: 13 % of random operand pairs then differ from the separately rounded result. It does
-// not touch a product that enters a fused multiply-add as the multiplicand, so such sums are
+// not touch a product that enters a fused multiply-add as multiplicand or addend, so such sums are
 // written  c + a*b  ==  fma(RN(-a*b), -1, c): negating a product is exact, and the fma adds
 // exactly RN(a*b). cp_selftest_pair compares the packed step with the scalar one bit for bit.
 __device__ __forceinline__ f32x2 add_product2(f32x2 c, f32x2 neg_product) {
@@ -388,7 +382,9 @@ __device__ __forceinline__ f32x2 add_product2(f32x2 c, f32x2 neg_product) {
 // the same operations in the same order on each half, hence the same bits. Rewrites that keep
 // negations out of the packed instructions: see div_mtot_core2; the denominator of the
 // angular acceleration is formed with its sign flipped (RN(a - b) == -RN(b - a)), which is the
-// operand the remainder step of div_tame needs, while the reciprocal takes the positive value.
+// operand the remainder step of div_tame needs, while the reciprocal takes the positive value;
+// p0 .. p2 are carried with flipped sign (every step is odd in its operand), so that -m_p*l
+// serves both there and in t1.
 __device__ __forceinline__ void euler_step_pair(StatePair &z, f32x2 force, bool &done0, bool &done1) {
     const f32x2 zz = mul2(z.th, z.th);
     const f32x2 sp = fma2(splat2(8.319973014e-03f), zz, splat2(-1.666664630e-01f));
@@ -406,7 +402,7 @@ __device__ __forceinline__ void euler_step_pair(StatePair &z, f32x2 force, bool 
     const f32x2 n1 = mul2(c, temp);
     const f32x2 num = add_product2(n0, n1);  // n0 - n1
     const f32x2 d0 = mul2(c, c);
-    const f32x2 h1 = mul2(splat2(0.5f * kMPole), d0);
+    const f32x2 h1 = mul2(splat2(kPML), d0);  // 0.5 * m_p == m_p * l
     const f32x2 nden = sub2(div_mtot_core2(h1), splat2(0.5f * kFT));  // -den
     float nd0, nd1, r0, r1;
     unpack2(nden, nd0, nd1);
@@ -416,14 +412,13 @@ __device__ __forceinline__ void euler_step_pair(StatePair &z, f32x2 force, bool 
     const f32x2 q = mul2(num, r);
     const f32x2 rem = fma2(nden, q, num);
     const f32x2 thacc = fma2(rem, r, q);
-    const f32x2 p0 = mul2(splat2(kPML), thacc);
-    const f32x2 p1 = mul2(p0, c);
-    const f32x2 xacc = sub2(temp, div_mtot_core2(p1));
-    const f32x2 ntau = splat2(-kTau);
-    const f32x2 nx = add_product2(z.x, mul2(ntau, z.xd));
-    const f32x2 nxd = add_product2(z.xd, mul2(ntau, xacc));
-    const f32x2 nth = add_product2(z.th, mul2(ntau, z.thd));
-    const f32x2 nthd = add_product2(z.thd, mul2(ntau, thacc));
+    const f32x2 np0 = mul2(splat2(-kPML), thacc);
+    const f32x2 np1 = mul2(np0, c);
+    const f32x2 xacc = add2(temp, div_mtot_core2(np1));  // temp - p2
+    const f32x2 nx = add_product2(z.x, mul2(splat2(-kTau), z.xd));
+    const f32x2 nxd = add_product2(z.xd, mul2(splat2(-kTau), xacc));
+    const f32x2 nth = add_product2(z.th, mul2(splat2(-kTau), z.thd));
+    const f32x2 nthd = add_product2(z.thd, mul2(splat2(-kTau), thacc));
     z.x = nx;
     z.xd = nxd;
     z.th = nth;

@@ -38,17 +38,18 @@ namespace cp {
 
 namespace {
 
-template <int POLICY>
+// SHORT: every time of the launch is below 2^16, where fold16(t) == t.
+template <int POLICY, bool SHORT>
 __device__ __forceinline__ uint32_t deferred_action(const RolloutParams &p, const FoldedKeys &ka, const LinearW &own,
                                                     uint32_t t, const State &z) {
-    if (POLICY == 0) return action_signbit_folded(ka, fold16(t));
+    if (POLICY == 0) return action_signbit_folded(ka, SHORT ? t : fold16(t));
     if (POLICY == 1) return linear_action(*reinterpret_cast<const LinearW *>(p.w), z);
     return linear_action(own, z);
 }
 
 // POLICY: 0 hashed actions, 1 shared linear policy, 6 one linear policy per environment.
 // K: trips between restart passes.
-template <int POLICY, int K>
+template <int POLICY, int K, bool SHORT>
 __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_constant__ RolloutParams p) {
     const uint32_t lane = threadIdx.x & 31u;
     const int64_t task = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -91,22 +92,25 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
         StatePair zz = pack_states(z0[0], z0[1]);
 
         // Slot j has done its last step (its clock reached t_end): results out, slot retired.
+        // cnt / begin are brought up to date by the restart pass, so an episode that ended on this
+        // very step (done_now) is added here; it also hands over the start state of t_end.
         auto finalize = [&](int j, bool done_now) {
             State a, b;
             unpack_states(zz, a, b);
             State &mine = j ? b : a;
-            // an episode that ended on the very last step hands over the start state of t_end
             if (done_now) mine = start_state_folded(kr[j], fold16(4u * t_end));
             zz = pack_states(a, b);
             const int64_t idx = base + j * 32 + lane;
             if (idx < p.n) {
                 // sum of the returns of the completed episodes = last termination time - time the
                 // first of them began (every step earns reward 1)
+                const uint32_t n_done = cnt[j] + (done_now ? 1u : 0u);
+                const uint32_t last_begin = done_now ? t_end : begin[j];
                 const uint32_t carried = p.ep_len_io ? p.ep_len_io[idx] : 0u;
-                const uint32_t ret = cnt[j] ? begin[j] - (p.t0 - carried) : 0u;
-                const uint32_t running = t_end - begin[j] + (cnt[j] == 0u ? carried : 0u);
+                const uint32_t ret = n_done ? last_begin - (p.t0 - carried) : 0u;
+                const uint32_t running = t_end - last_begin + (n_done == 0u ? carried : 0u);
                 if (p.ep_return_sum) p.ep_return_sum[idx] = (float)ret;
-                if (p.ep_count) p.ep_count[idx] = cnt[j];
+                if (p.ep_count) p.ep_count[idx] = n_done;
                 if (p.ep_len_io) p.ep_len_io[idx] = running;
                 if (p.out_planes) {
                     p.out_planes[idx] = mine.x;
@@ -115,21 +119,16 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
                     p.out_planes[3 * p.out_stride + idx] = mine.thd;
                 }
                 tot_ret += ret;
-                tot_cnt += cnt[j];
+                tot_cnt += n_done;
             }
         };
 
-        // Bookkeeping of slot j after a trip in which its environment (if it was stepping) either
-        // survived or ended (done_now). TAIL: the slot may have done its last step.
+        // Slot j after a trip: a stepping slot's clock advances, and it goes idle if its episode
+        // ended (done_now). TAIL: the slot may have done its last step.
         auto after_step = [&](auto tail, int j, bool done_now) {
             constexpr bool TAIL = decltype(tail)::value;
             const bool live = act[j];
             if (live) t[j] += 1u;
-            const bool ended = live && done_now;
-            if (ended) {
-                cnt[j] += 1u;
-                begin[j] = t[j];
-            }
             act[j] = live && !done_now;
             if (TAIL) {
                 if (live && t[j] == t_end) {
@@ -139,12 +138,19 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
             }
         };
 
-        // Idle slots that still have steps to do take the start state of their own time.
+        // Idle slots that still have steps to do: their episode ended at their (stopped) clock,
+        // which is also the time the next one begins; they take that time's start state, each
+        // lane hashing its own. (Handing the hashes to the whole warp through shared memory, as
+        // the general kernel does after every step, was measured here too: with a dozen restarts
+        // per pass its ballots, ranks, barriers and rounds cost more instructions than the
+        // divergent per-lane hashes, 1.29 against 1.14 ms on 1,048,576 x 500.)
         auto restart_pass = [&](auto tail) {
             constexpr bool TAIL = decltype(tail)::value;
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
                 if (!act[j] && (!TAIL || t[j] != t_end)) {
+                    cnt[j] += 1u;
+                    begin[j] = t[j];
                     State a, b;
                     unpack_states(zz, a, b);
                     (j ? b : a) = start_state_folded(kr[j], fold16(4u * t[j]));
@@ -157,8 +163,8 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
         auto trip = [&](auto tail) {
             State a, b;
             unpack_states(zz, a, b);
-            const uint32_t sb0 = deferred_action<POLICY>(p, ka[0], own[0], t[0], a);
-            const uint32_t sb1 = deferred_action<POLICY>(p, ka[POLICY == 0 ? 1 : 0], own[POLICY == 6 ? 1 : 0], t[1], b);
+            const uint32_t sb0 = deferred_action<POLICY, SHORT>(p, ka[0], own[0], t[0], a);
+            const uint32_t sb1 = deferred_action<POLICY, SHORT>(p, ka[POLICY == 0 ? 1 : 0], own[POLICY == 6 ? 1 : 0], t[1], b);
             bool d0, d1;
             euler_step_pair(zz, pack2(force_from_signbit(sb0), force_from_signbit(sb1)), d0, d1);
             after_step(tail, 0, d0);
@@ -172,8 +178,8 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
             // start state (|theta| <= 0.05), which is the packed step's domain.
             State a, b;
             unpack_states(zz, a, b);
-            const uint32_t sb0 = deferred_action<POLICY>(p, ka[0], own[0], t[0], a);
-            const uint32_t sb1 = deferred_action<POLICY>(p, ka[POLICY == 0 ? 1 : 0], own[POLICY == 6 ? 1 : 0], t[1], b);
+            const uint32_t sb0 = deferred_action<POLICY, SHORT>(p, ka[0], own[0], t[0], a);
+            const uint32_t sb1 = deferred_action<POLICY, SHORT>(p, ka[POLICY == 0 ? 1 : 0], own[POLICY == 6 ? 1 : 0], t[1], b);
             const bool d0 = euler_step<false>(a, force_from_signbit(sb0));
             const bool d1 = euler_step<false>(b, force_from_signbit(sb1));
             zz = pack_states(a, b);
@@ -211,15 +217,17 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
     }
 }
 
-template <int POLICY>
+template <int POLICY, bool SHORT>
 cudaError_t launch_k(RolloutParams &p, int k, cudaStream_t s) {
     p.n_tasks = (p.n + 63) / 64;
     int64_t grid = (p.n_tasks + 7) / 8;
     if (grid > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     switch (k) {
-        case 2: rollout_deferred_kernel<POLICY, 2><<<(unsigned)grid, 256, 0, s>>>(p); break;
-        case 8: rollout_deferred_kernel<POLICY, 8><<<(unsigned)grid, 256, 0, s>>>(p); break;
-        default: rollout_deferred_kernel<POLICY, 4><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        case 2: rollout_deferred_kernel<POLICY, 2, SHORT><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        case 3: rollout_deferred_kernel<POLICY, 3, SHORT><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        case 6: rollout_deferred_kernel<POLICY, 6, SHORT><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        case 8: rollout_deferred_kernel<POLICY, 8, SHORT><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        default: rollout_deferred_kernel<POLICY, 4, SHORT><<<(unsigned)grid, 256, 0, s>>>(p); break;
     }
     count_launch();
     return cudaGetLastError();
@@ -232,11 +240,13 @@ bool rollout_deferred_applies(const RolloutParams &p, int policy, bool streams) 
 }
 
 cudaError_t launch_rollout_deferred(RolloutParams &p, int policy, cudaStream_t s) {
-    const int k = g_tuning.rollout_defer > 0 ? g_tuning.rollout_defer : 4;
+    const int k = g_tuning.rollout_defer > 0 ? g_tuning.rollout_defer : 6;
+    // the action hash folds the time's upper half into the lower one: nothing to do below 2^16
+    const bool short_times = (uint64_t)p.t0 + p.T <= 65536u;
     switch (policy) {
-        case 0: return launch_k<0>(p, k, s);
-        case 1: return launch_k<1>(p, k, s);
-        default: return launch_k<6>(p, k, s);
+        case 0: return short_times ? launch_k<0, true>(p, k, s) : launch_k<0, false>(p, k, s);
+        case 1: return launch_k<1, false>(p, k, s);
+        default: return launch_k<6, false>(p, k, s);
     }
 }
 

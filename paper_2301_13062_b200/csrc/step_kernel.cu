@@ -383,35 +383,47 @@ cudaError_t launch_tame_div_selftest(uint32_t den_step, unsigned long long *out,
 }
 
 // ---- calibration: what one pipe sustains, for the roofline denominators ----
-// Every thread runs `iters` rounds of eight independent chains of one instruction kind
-// (0: FFMA, 1: IMAD, 2: MUFU reciprocal), sixteen resident warps per scheduler. The host times
-// the launch; instructions = threads * iters * 8. The seeds come from memory so that nothing
-// folds at compile time, and the results are stored so that nothing is dead.
+// Every thread runs `iters` rounds of eight independent chains, sixteen resident warps per
+// scheduler. KIND 0: FFMA, 1: IMAD, 2: MUFU reciprocal, 3: packed FFMA2 (two float32 FMAs per
+// instruction); mixes of four chains each: 4: FFMA2 + FFMA, 5: FFMA2 + IMAD, 6: FFMA2 + integer
+// logic (the ALU pipe), 7: FFMA + IMAD. The host times the launch; instructions = threads *
+// iters * 8. The seeds come from memory so that nothing folds at compile time, and the results
+// are stored so that nothing is dead.
 template <int KIND>
 __global__ void __launch_bounds__(256) pipe_rate_kernel(const float *seed, float *sink, int iters) {
     float a[8];
     uint32_t u[8];
+    f32x2 q[8];
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
         a[k] = seed[k] + (float)threadIdx.x * 1e-3f;
         u[k] = __float_as_uint(a[k]) | 1u;
+        q[k] = pack2(a[k], a[k] + 0.5f);
     }
     const float m = seed[8], c = seed[9];
     const uint32_t um = __float_as_uint(m) | 1u, uc = __float_as_uint(c);
+    const f32x2 qm = pack2(m, m), qc = pack2(c, c);
     for (int i = 0; i < iters; ++i) {
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-            if (KIND == 0) a[k] = __fmaf_rn(a[k], m, c);
-            if (KIND == 1) u[k] = u[k] * um + uc;
+            const bool second = k >= 4;  // the mixes: chains 0-3 packed (7: scalar float), 4-7 the partner
+            if (KIND == 0 || (KIND == 4 && second) || (KIND == 7 && !second)) a[k] = __fmaf_rn(a[k], m, c);
+            if (KIND == 1 || ((KIND == 5 || KIND == 7) && second)) u[k] = u[k] * um + uc;
             if (KIND == 2) {  // the add keeps the assembler from cancelling a reciprocal of a reciprocal
                 asm volatile("rcp.approx.ftz.f32 %0, %0;" : "+f"(a[k]));
                 a[k] = __fadd_rn(a[k], c);
             }
+            if (KIND == 3 || ((KIND == 4 || KIND == 5 || KIND == 6) && !second)) q[k] = fma2(q[k], qm, qc);
+            if (KIND == 6 && second) u[k] = (u[k] ^ um) + (u[k] >> 7);  // two ALU instructions per round
         }
     }
     float acc = 0.0f;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) acc += KIND == 1 ? __uint_as_float(u[k] & 0x3fffffffu) : a[k];
+    for (int k = 0; k < 8; ++k) {
+        float lo, hi;
+        unpack2(q[k], lo, hi);
+        acc += __uint_as_float(u[k] & 0x3fffffffu) + a[k] + lo + hi;
+    }
     sink[(size_t)blockIdx.x * blockDim.x + threadIdx.x] = acc;
 }
 
@@ -421,7 +433,12 @@ cudaError_t launch_pipe_rate(int kind, const float *seed, float *sink, int iters
     switch (kind) {
         case 0: pipe_rate_kernel<0><<<grid, block, 0, s>>>(seed, sink, iters); break;
         case 1: pipe_rate_kernel<1><<<grid, block, 0, s>>>(seed, sink, iters); break;
-        default: pipe_rate_kernel<2><<<grid, block, 0, s>>>(seed, sink, iters); break;
+        case 2: pipe_rate_kernel<2><<<grid, block, 0, s>>>(seed, sink, iters); break;
+        case 3: pipe_rate_kernel<3><<<grid, block, 0, s>>>(seed, sink, iters); break;
+        case 4: pipe_rate_kernel<4><<<grid, block, 0, s>>>(seed, sink, iters); break;
+        case 5: pipe_rate_kernel<5><<<grid, block, 0, s>>>(seed, sink, iters); break;
+        case 6: pipe_rate_kernel<6><<<grid, block, 0, s>>>(seed, sink, iters); break;
+        default: pipe_rate_kernel<7><<<grid, block, 0, s>>>(seed, sink, iters); break;
     }
     count_launch();
     return cudaGetLastError();

@@ -25,7 +25,7 @@ def test_calibration_launches_count_and_order(cp):
     seed = torch.linspace(0.5, 1.5, 10, device="cuda")
     sink = torch.full((threads,), float("nan"), device="cuda")
     rates = {}
-    for kind, iters in ((0, 4000), (1, 4000), (2, 1000)):
+    for kind, iters in ((0, 4000), (1, 4000), (2, 1000), (3, 4000), (4, 4000), (5, 4000), (6, 4000), (7, 4000)):
         n = cp.cp_calibrate_pipe(kind, seed, sink, iters)
         assert n == threads * iters * 8
         torch.cuda.synchronize()
@@ -39,6 +39,6 @@ def test_calibration_launches_count_and_order(cp):
     # the special-function pipe is the narrow one; the float pipe is at least as wide as the integer one
     assert rates[2] < rates[1] <= rates[0] * 1.05
     with pytest.raises(cp.CartpoleError):
-        cp.cp_calibrate_pipe(3, seed, sink, 10)
+        cp.cp_calibrate_pipe(8, seed, sink, 10)
     with pytest.raises(cp.CartpoleError):
         cp.cp_calibrate_pipe(0, seed, sink, 0)

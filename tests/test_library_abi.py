@@ -45,7 +45,8 @@ def test_host_side_argument_errors(cp):
     assert b"unknown tuning key" in L.cp_last_error()
     assert L.cp_tune(b"rollout_block", 100) == cp.CP_EINVAL
     assert L.cp_tune(b"rollout_ept", 3) == cp.CP_EINVAL
-    assert L.cp_tune(b"rollout_coop", 5) == cp.CP_EINVAL
+    assert L.cp_tune(b"rollout_coop", 6) == cp.CP_EINVAL
+    assert L.cp_tune(b"rollout_defer", 5) == cp.CP_EINVAL
     assert L.cp_tune(b"rollout_coop", 0) == cp.CP_OK
     assert L.cp_tune(b"rollout_block", 256) == cp.CP_OK
     assert L.cp_tune(b"rollout_block", 0) == cp.CP_OK
