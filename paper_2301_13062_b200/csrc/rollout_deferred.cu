@@ -23,9 +23,9 @@
 // the price is idle slots (about 7 % at K = 4 with the random policy's 22-step episodes) and a
 // ragged end.
 //
-// Scope: no per-step output streams (they are rows of global time) and no episode step limit;
-// hashed actions, the shared linear policy or one linear policy per environment; canonical
-// arithmetic. Everything else takes the general kernel.
+// Scope: no per-step output streams (they are rows of global time); hashed actions, the shared
+// linear policy or one linear policy per environment; canonical arithmetic; with or without the
+// episode step limit. Everything else takes the general kernel.
 //
 // No warp waits for another one and nothing spins: the loop's trip count is bounded by the
 // launch parameters (every trip block advances every unfinished slot by at least one step).
@@ -48,8 +48,8 @@ __device__ __forceinline__ uint32_t deferred_action(const RolloutParams &p, cons
 }
 
 // POLICY: 0 hashed actions, 1 shared linear policy, 6 one linear policy per environment.
-// K: trips between restart passes.
-template <int POLICY, int K, bool SHORT>
+// K: trips between restart passes. LIMIT: episodes are cut off after p.max_steps steps.
+template <int POLICY, int K, bool SHORT, bool LIMIT>
 __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_constant__ RolloutParams p) {
     const uint32_t lane = threadIdx.x & 31u;
     const int64_t task = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -86,40 +86,34 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
             }
             t[j] = p.t0;
             cnt[j] = 0u;
-            begin[j] = p.t0;
+            begin[j] = p.t0 - ((LIMIT && p.ep_len_io) ? p.ep_len_io[idx] : 0u);
             act[j] = true;
         }
         StatePair zz = pack_states(z0[0], z0[1]);
 
-        // Slot j has done its last step (its clock reached t_end): results out, slot retired.
-        // cnt / begin are brought up to date by the restart pass, so an episode that ended on this
-        // very step (done_now) is added here; it also hands over the start state of t_end.
+        // Slot j has done its last step (its clock reached t_end) and retires. cnt / begin are
+        // brought up to date by the restart pass, so an episode that ended on this very step
+        // (done_now) is added here; it also hands over the start state of t_end. The final state is
+        // stored now (the slot's half of the packed arithmetic goes on computing values nobody
+        // reads); the per-env results wait in cnt / begin and are stored by the whole warp after
+        // the loop, as full lines (a caller may have pointed them at pinned host memory).
         auto finalize = [&](int j, bool done_now) {
-            State a, b;
-            unpack_states(zz, a, b);
-            State &mine = j ? b : a;
-            if (done_now) mine = start_state_folded(kr[j], fold16(4u * t_end));
-            zz = pack_states(a, b);
-            const int64_t idx = base + j * 32 + lane;
-            if (idx < p.n) {
-                // sum of the returns of the completed episodes = last termination time - time the
-                // first of them began (every step earns reward 1)
-                const uint32_t n_done = cnt[j] + (done_now ? 1u : 0u);
-                const uint32_t last_begin = done_now ? t_end : begin[j];
-                const uint32_t carried = p.ep_len_io ? p.ep_len_io[idx] : 0u;
-                const uint32_t ret = n_done ? last_begin - (p.t0 - carried) : 0u;
-                const uint32_t running = t_end - last_begin + (n_done == 0u ? carried : 0u);
-                if (p.ep_return_sum) p.ep_return_sum[idx] = (float)ret;
-                if (p.ep_count) p.ep_count[idx] = n_done;
-                if (p.ep_len_io) p.ep_len_io[idx] = running;
-                if (p.out_planes) {
+            if (done_now) {
+                cnt[j] += 1u;
+                begin[j] = t_end;
+            }
+            if (p.out_planes) {
+                State a, b;
+                unpack_states(zz, a, b);
+                State mine = j ? b : a;
+                if (done_now) mine = start_state_folded(kr[j], fold16(4u * t_end));
+                const int64_t idx = base + j * 32 + lane;
+                if (idx < p.n) {
                     p.out_planes[idx] = mine.x;
                     p.out_planes[p.out_stride + idx] = mine.xd;
                     p.out_planes[2 * p.out_stride + idx] = mine.th;
                     p.out_planes[3 * p.out_stride + idx] = mine.thd;
                 }
-                tot_ret += ret;
-                tot_cnt += n_done;
             }
         };
 
@@ -129,6 +123,9 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
             constexpr bool TAIL = decltype(tail)::value;
             const bool live = act[j];
             if (live) t[j] += 1u;
+            // begin[j] is the time the running episode began (set by the restart pass; before t0 by
+            // the steps carried in): an episode that has lasted max_steps steps ends like a fall
+            if (LIMIT) done_now = done_now || (t[j] - begin[j]) >= p.max_steps;
             act[j] = live && !done_now;
             if (TAIL) {
                 if (live && t[j] == t_end) {
@@ -203,6 +200,22 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
             for (int k = 0; k < K; ++k) trip(std::true_type{});
             restart_pass(std::true_type{});
         }
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int64_t idx = base + j * 32 + lane;
+            if (idx >= p.n) continue;
+            // sum of the returns of the completed episodes = last termination time - time the first
+            // of them began (every step earns reward 1); begin[j] still holds its initial value if
+            // no episode ended in this launch
+            const uint32_t carried = p.ep_len_io ? p.ep_len_io[idx] : 0u;
+            const uint32_t ret = cnt[j] ? begin[j] - (p.t0 - carried) : 0u;
+            const uint32_t running = t_end - begin[j] + ((!LIMIT && cnt[j] == 0u) ? carried : 0u);
+            if (p.ep_return_sum) p.ep_return_sum[idx] = (float)ret;
+            if (p.ep_count) p.ep_count[idx] = cnt[j];
+            if (p.ep_len_io) p.ep_len_io[idx] = running;
+            tot_ret += ret;
+            tot_cnt += cnt[j];
+        }
     }
 
     if (p.totals) {
@@ -217,36 +230,43 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
     }
 }
 
-template <int POLICY, bool SHORT>
+template <int POLICY, bool SHORT, bool LIMIT>
 cudaError_t launch_k(RolloutParams &p, int k, cudaStream_t s) {
     p.n_tasks = (p.n + 63) / 64;
     int64_t grid = (p.n_tasks + 7) / 8;
     if (grid > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     switch (k) {
-        case 2: rollout_deferred_kernel<POLICY, 2, SHORT><<<(unsigned)grid, 256, 0, s>>>(p); break;
-        case 3: rollout_deferred_kernel<POLICY, 3, SHORT><<<(unsigned)grid, 256, 0, s>>>(p); break;
-        case 6: rollout_deferred_kernel<POLICY, 6, SHORT><<<(unsigned)grid, 256, 0, s>>>(p); break;
-        case 8: rollout_deferred_kernel<POLICY, 8, SHORT><<<(unsigned)grid, 256, 0, s>>>(p); break;
-        default: rollout_deferred_kernel<POLICY, 4, SHORT><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        case 2: rollout_deferred_kernel<POLICY, 2, SHORT, LIMIT><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        case 3: rollout_deferred_kernel<POLICY, 3, SHORT, LIMIT><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        case 6: rollout_deferred_kernel<POLICY, 6, SHORT, LIMIT><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        case 8: rollout_deferred_kernel<POLICY, 8, SHORT, LIMIT><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        default: rollout_deferred_kernel<POLICY, 4, SHORT, LIMIT><<<(unsigned)grid, 256, 0, s>>>(p); break;
     }
     count_launch();
     return cudaGetLastError();
 }
 
+template <int POLICY, bool SHORT>
+cudaError_t launch_limit(RolloutParams &p, int k, cudaStream_t s) {
+    return p.max_steps ? launch_k<POLICY, SHORT, true>(p, k, s) : launch_k<POLICY, SHORT, false>(p, k, s);
+}
+
 }  // namespace
 
 bool rollout_deferred_applies(const RolloutParams &p, int policy, bool streams) {
-    return !streams && p.max_steps == 0 && !p.action_bits_in && !p.start_in && (policy == 0 || policy == 1 || policy == 6);
+    return !streams && !p.action_bits_in && !p.start_in && (policy == 0 || policy == 1 || policy == 6);
 }
 
 cudaError_t launch_rollout_deferred(RolloutParams &p, int policy, cudaStream_t s) {
-    const int k = g_tuning.rollout_defer > 0 ? g_tuning.rollout_defer : 6;
+    // measured on 1,048,576 x 500: hashed actions (22-step episodes) 1.022 / 1.034 / 1.071 ms at
+    // K = 4 / 6 / 8, the linear policy (longer episodes) 0.952 / 0.934 / 1.008 ms
+    const int k = g_tuning.rollout_defer > 0 ? g_tuning.rollout_defer : (policy == 0 ? 4 : 6);
     // the action hash folds the time's upper half into the lower one: nothing to do below 2^16
     const bool short_times = (uint64_t)p.t0 + p.T <= 65536u;
     switch (policy) {
-        case 0: return short_times ? launch_k<0, true>(p, k, s) : launch_k<0, false>(p, k, s);
-        case 1: return launch_k<1, false>(p, k, s);
-        default: return launch_k<6, false>(p, k, s);
+        case 0: return short_times ? launch_limit<0, true>(p, k, s) : launch_limit<0, false>(p, k, s);
+        case 1: return launch_limit<1, false>(p, k, s);
+        default: return launch_limit<6, false>(p, k, s);
     }
 }
 

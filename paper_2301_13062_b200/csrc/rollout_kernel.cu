@@ -13,7 +13,7 @@ cudaError_t launch_rollout(RolloutParams &p, int policy, bool streams, bool cont
     // wherever it applies, any other forced shape keeps the general kernel
     const bool fills_chip = (p.n + 63) / 64 >= (int64_t)sm_count() * 16;
     const bool by_default = g_tuning.rollout_coop == 0 && g_tuning.rollout_ept == 0 && fills_chip &&
-                            (policy == 0 || policy == 1);
+                            (policy == 0 || policy == 1 || policy == 6);
     if ((by_default || g_tuning.rollout_coop == 5) && rollout_deferred_applies(p, policy, streams))
         return launch_rollout_deferred(p, policy, s);
     return launch_rollout_arith<false>(p, policy, streams, s);

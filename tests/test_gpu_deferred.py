@@ -1,0 +1,131 @@
+"""GPU tests of the deferred-restart rollout kernel (two environments per thread stepped by packed
+float32 instructions, a clock per environment, restarts every K trips): it must produce the bits
+of the general rollout kernel for every call it covers — any trip spacing, ragged sizes, horizons
+shorter than one block of trips, global times beyond 2^16, the episode step limit, steps carried
+in, caller-supplied states with angles outside the polynomial range — and the oracle's returns."""
+import numpy as np
+import pytest
+
+from paper_2301_13062_b200 import inputs
+from tests import gpu_helpers as H
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+GENERAL = (2, 1)   # two envs per thread, restarts by the whole warp after every step
+DEFERRED = (2, 5)
+
+
+@pytest.fixture(scope="module")
+def cp():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2301_13062_b200 import binding, build
+    build.build()
+    binding.lib()
+    torch.cuda.set_device(0)
+    return binding
+
+
+def outputs(n):
+    return {"ep_return_sum": torch.full((n,), -1.0, dtype=torch.float32, device="cuda"),
+            "ep_count": torch.full((n,), -1, dtype=torch.int32, device="cuda"),
+            "totals": torch.zeros(2, dtype=torch.int64, device="cuda"),
+            "final_state": torch.full((4, n), 9.0, dtype=torch.float32, device="cuda")}
+
+
+def fetch(out):
+    torch.cuda.synchronize()
+    return {k: v.cpu().numpy().view(np.uint32 if v.dtype != torch.int64 else np.uint64) for k, v in out.items()}
+
+
+def make_policy(cp, kind, n):
+    if kind == 0:
+        return None, None
+    if kind == 1:
+        w = inputs.policy_weights(1, 1)
+        return cp.policy(1, w), w
+    w = inputs.per_env_linear_weights(n, 11)
+    return cp.policy(cp.CP_POLICY_LINEAR_PER_ENV, torch.from_numpy(w).cuda()), w
+
+
+def run(cp, shape, k, **kw):
+    n = kw["n_envs"]
+    with H.rollout_shape(cp, *shape):
+        cp.cp_tune("rollout_defer", k)
+        try:
+            out = outputs(n)
+            cp.cp_rollout_ex(**kw, **out)
+            return fetch(out)
+        finally:
+            cp.cp_tune("rollout_defer", 0)
+
+
+@pytest.mark.parametrize("kind", [0, 1, 6])
+@pytest.mark.parametrize("n,T,t0,off,limit", [
+    (1, 1, 0, 0, 0), (63, 2, 0, 5, 0), (65, 5, 3, 0, 0), (4099, 61, 0, 77, 0), (4099, 61, 0, 77, 23),
+    (70001, 200, 0, 0, 0), (20000, 150, 70000, 1 << 20, 0), (20000, 150, 65500, 0, 40), (3000, 700, 11, 0, 500),
+])
+def test_same_bits_as_the_general_kernel(cp, kind, n, T, t0, off, limit):
+    pol, _ = make_policy(cp, kind, n)
+    kw = dict(n_envs=n, T=T, seed=3, t0=t0, env_offset=off, policy=pol, max_episode_steps=limit)
+    want = run(cp, GENERAL, 0, **kw)
+    assert want["ep_count"].max() > 0 or T < 8
+    for k in (2, 3, 4, 6, 8):
+        got = run(cp, DEFERRED, k, **kw)
+        for key in want:
+            assert np.array_equal(want[key], got[key]), (key, k)
+
+
+@pytest.mark.parametrize("kind", [0, 1])
+@pytest.mark.parametrize("limit", [0, 31])
+def test_chunks_from_a_callers_states(cp, kind, limit):
+    """States with angles far outside the polynomial range and running-episode lengths carried in
+    and out, advanced in chunks of 1, 2, 7 and 40 steps: general and deferred kernels stay
+    identical in the batch itself, the carried lengths and the per-chunk results."""
+    n, seed = 9001, 5
+    z = np.concatenate([inputs.random_states(n // 3, seed=4, spread="wide"),
+                        inputs.random_states(n // 3, seed=5, spread="live"),
+                        inputs.random_states(n - 2 * (n // 3), seed=6, spread="edge")], axis=1)
+    pol, _ = make_policy(cp, kind, n)
+    results = {}
+    for name, shape in (("general", GENERAL), ("deferred", DEFERRED)):
+        planes = torch.zeros(4, n + 3, dtype=torch.float32, device="cuda")
+        planes[:, :n] = torch.from_numpy(z).cuda()
+        st = cp.cp_wrap(planes, n, seed, 17, 64)  # plane stride n + 3: no alignment to lean on
+        ep_len = torch.from_numpy(np.arange(n, dtype=np.int32) % 29).cuda()
+        log = []
+        with H.rollout_shape(cp, *shape):
+            for T in (1, 2, 7, 40):
+                out = {"ep_return_sum": torch.zeros(n, device="cuda"),
+                       "ep_count": torch.zeros(n, dtype=torch.int32, device="cuda"),
+                       "totals": torch.zeros(2, dtype=torch.int64, device="cuda")}
+                cp.cp_rollout_ex(T=T, state=st, ep_len=ep_len, policy=pol, max_episode_steps=limit, **out)
+                torch.cuda.synchronize()
+                log.append({k: v.cpu().numpy().copy() for k, v in out.items()})
+                log.append({"planes": planes.cpu().numpy().copy(), "ep_len": ep_len.cpu().numpy().copy()})
+        assert st.info()["t"] == 17 + 50
+        results[name] = log
+    for a, b in zip(results["general"], results["deferred"]):
+        for key in a:
+            assert np.array_equal(a[key].view(np.uint32) if a[key].dtype == np.float32 else a[key],
+                                  b[key].view(np.uint32) if b[key].dtype == np.float32 else b[key]), key
+    assert sum(int(c["ep_count"].sum()) for c in results["deferred"][0::2]) > n // 4
+
+
+@pytest.mark.parametrize("kind", [0, 1, 6])
+def test_returns_against_the_oracle(cp, oracle, kind):
+    n, T, seed = 50001, 300, 2
+    pol, w = make_policy(cp, kind, n)
+    r = run(cp, DEFERRED, 0, n_envs=n, T=T, seed=seed, policy=pol)
+    o = oracle.rollout(n, T, seed, {0: 0, 1: 1, 6: inputs.POLICY_LINEAR_PER_ENV}[kind], w, final_state=True,
+                       min_gap=True, nthreads=8)
+    excuse = (o["min_gap"] < 1e-5) if kind else None
+    res = H.assert_returns_match(r["ep_return_sum"].view(np.float32), r["ep_count"], o["ep_return_sum"], o["ep_count"],
+                                 excuse)
+    assert int(r["totals"][0]) == int(r["ep_return_sum"].view(np.float32).astype(np.float64).sum())
+    assert int(r["totals"][1]) == int(r["ep_count"].astype(np.int64).sum())
+    same = (r["ep_return_sum"].view(np.float32) == o["ep_return_sum"]) & (r["ep_count"] == o["ep_count"])
+    err = np.abs(r["final_state"].view(np.float32)[:, same].astype(np.float64) - o["final_state"][:, same])
+    assert np.quantile(err.max(axis=0), 0.99) < 1e-3 and res["identical"] > 0.99
