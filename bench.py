@@ -36,20 +36,27 @@ SMS = 148
 # rollout_ept=1 rollout_coop=2): the instructions an environment needs, none counted for
 # lanes that idle or help a neighbour — the algorithmic figure. "slot" = 32 *
 # smsp__inst_executed.sum / (N*T) of the kernel the library launches by default at this size
-# (restarts by the whole warp): the issue slots it really occupies.
+# ("kernel"): the issue slots it really occupies; the deferred-restart kernel steps two
+# environments per packed float32 instruction, so its slots fall below the thread figure.
+# "fp32" = float32 multiply / add / fma lane operations of the method per env-step (40 in the
+# dynamics with the shortcuts of the kernels, 8 more for the linear policy).
+# COUNTED_AT = build.kernel_hash() of the sources these were captured from (a test compares it
+# with the current sources, so that the fractions cannot go stale unnoticed).
+COUNTED_AT = "unset"
 ROLLOUT_OPS = {
-    "random": {"thread": 68.6, "slot": 82.6},
-    "linear": {"thread": 73.8, "slot": 76.2},
-    # here the default kernel's own thread count (87.7) is below the per-lane formulation's (91.9:
-    # one running stream pointer per env instead of one per two envs), so it is the algorithmic one
-    "linear+streams": {"thread": 87.7, "slot": 87.8},
-    "mlp": {"thread": 440.3, "slot": 464.4},
-    "random+contracted": {"thread": 55.6, "slot": 68.6},
+    "random": {"thread": 68.6, "slot": 82.6, "fp32": 40.0, "kernel": "rollout_deferred_kernel"},
+    "linear": {"thread": 73.8, "slot": 76.2, "fp32": 48.0, "kernel": "rollout_deferred_kernel"},
+    # here the default kernel's own thread count is below the per-lane formulation's (one running
+    # stream pointer per two envs instead of one per env), so it is the algorithmic one
+    "linear+streams": {"thread": 87.7, "slot": 87.8, "fp32": 48.0, "kernel": "rollout_kernel"},
+    "mlp": {"thread": 440.3, "slot": 464.4, "kernel": "rollout_kernel"},
+    "random+contracted": {"thread": 55.6, "slot": 68.6, "kernel": "rollout_kernel"},
 }
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch in the same captures.
 ROLLOUT_DRAM_BYTES = {"random": 24.8e3, "linear": 24.6e3, "linear+streams": 381.1e6, "mlp": 21.8e3}
 STEP_DRAM_BYTES_16M = 568.2e6  # step_kernel at 16,777,216 envs, same kind of capture
 # Algorithmic HBM bytes per env-step of the step paths.
+LAST_TIMING: dict = {}  # median / best / worst of the per-iteration event times of the last timed() call
 STEP_BYTES = 37.0      # 16 in + 16 out + 4 reward + 1 done, hashed action
 LADDER_BYTES = 375.0   # sum over the 46 one-op kernels of their input and output planes
 
@@ -162,6 +169,29 @@ def run_reference(args) -> None:
 
 
 # ------------------------------------------------------------------------------ our arm
+def launch_plan(gpus: int, environ, argv: list[str], port: int | None = None):
+    """How `--gpus N` is honoured. Returns ("run", None): this process is a rank (or the only one);
+    ("spawn", cmd): no launcher started us and N > 1, so re-run this script as N local ranks, one
+    per GPU; ("error", text): the launcher's world size contradicts --gpus."""
+    if gpus < 1:
+        return "error", f"--gpus must be >= 1 (got {gpus})"
+    if "WORLD_SIZE" in environ:
+        world = int(environ["WORLD_SIZE"])
+        if world != gpus:
+            return "error", f"launched with WORLD_SIZE={world} but --gpus {gpus}: they must agree"
+        return "run", None
+    if gpus == 1:
+        return "run", None
+    if port is None:
+        import socket
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
+    return "spawn", cmd
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -172,12 +202,21 @@ def main() -> None:
     ap.add_argument("--no-paths", action="store_true", help="skip the ladder / fused-step / other-config lines")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--step-envs", type=int, default=1 << 24, help="batch of the HBM-bound fused-step measurement")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="weak: every GPU runs the whole workload on its own env-id range; strong: the "
+                         "workload's environments are split over the GPUs")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
         return
+    kind, detail = launch_plan(args.gpus, os.environ, sys.argv[1:])
+    if kind == "error":
+        print(f"bench.py: {detail}", file=sys.stderr)
+        sys.exit(2)
+    if kind == "spawn":  # --gpus N without a launcher: one rank per GPU under torch.distributed.run
+        sys.exit(subprocess.call(detail))
 
     import numpy as np
     import torch
@@ -189,6 +228,10 @@ def main() -> None:
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if torch.cuda.device_count() <= local_rank:
+        print(f"bench.py: rank {rank} needs GPU {local_rank}, this machine shows {torch.cuda.device_count()}",
+              file=sys.stderr)
+        sys.exit(2)
     torch.cuda.set_device(local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
@@ -224,7 +267,9 @@ def main() -> None:
             b.record()
         sync()
         launches = cp.cp_launch_count() - launches0
-        ms = sum(a.elapsed_time(b) for a, b in evs)
+        per = [a.elapsed_time(b) for a, b in evs]
+        ms = sum(per)
+        LAST_TIMING.update(median_ms=sorted(per)[len(per) // 2], best_ms=min(per), worst_ms=max(per))
         return (max_over_ranks(ms) if all_ranks else ms), launches
 
     # ---- headline: fused rollout ----
@@ -232,8 +277,12 @@ def main() -> None:
     pol_name = {0: "random", 1: "linear", 2: "mlp"}[w.policy]
     weights = inputs.policy_weights(w.policy, w.policy_seed) if w.policy else None
     pol = cp.policy(w.policy, weights) if w.policy else None
-    n, T = w.n_envs, w.T
-    env_offset = sharding.weak_env_offset(n, rank)  # weak scaling: a full batch per rank, own env range
+    T = w.T
+    if args.scaling == "strong":  # the workload's environments split over the ranks by global id
+        lo, hi = sharding.rank_env_range(w.n_envs, rank, world)
+        n, env_offset, job_envs = hi - lo, lo, w.n_envs
+    else:                          # weak: a full batch per rank on its own env-id range
+        n, env_offset, job_envs = w.n_envs, sharding.weak_env_offset(w.n_envs, rank), world * w.n_envs
     ret = torch.empty(n, dtype=torch.float32, device="cuda")
     cnt = torch.empty(n, dtype=torch.int32, device="cuda")
     tot = torch.zeros(2, dtype=torch.int64, device="cuda")
@@ -253,21 +302,29 @@ def main() -> None:
         rollout_step()
         torch.cuda.synchronize()
     ms, launches = timed(rollout_step, args.steps, args.warmup)
+    step_stats = dict(LAST_TIMING)  # this rank's own per-iteration times
     clocks = sampler.stop() if rank == 0 else {}
     ms_per_step = ms / args.steps
-    value = world * n * T / (ms_per_step * 1e-3)
-    ops = ROLLOUT_OPS[pol_name + ("+streams" if w.streams else "")]
+    value = job_envs * T / (ms_per_step * 1e-3)
+    variant = pol_name + ("+streams" if w.streams else "")
+    ops = ROLLOUT_OPS[variant]
     rate = n * T / (ms_per_step * 1e-3)  # per GPU
-    roofline = {"bound": "alu", "kernel": "rollout_kernel", "achieved": rate * ops["thread"] / 1e12,
+    roofline = {"bound": "alu", "kernel": ops["kernel"], "achieved": rate * ops["thread"] / 1e12,
                 "peak": peak_inst / 1e12, "unit": "Tinst/s", "frac": rate * ops["thread"] / peak_inst,
                 "issue_slot_frac": rate * ops["slot"] / peak_inst,
-                "traffic": ROLLOUT_DRAM_BYTES.get(pol_name + ("+streams" if w.streams else "")),
+                "fp32_pipe_frac": rate * ops["fp32"] / peak_inst if "fp32" in ops else None,
+                "traffic": ROLLOUT_DRAM_BYTES.get(variant),
                 "traffic_note": "ncu dram bytes of one launch at 1,048,576 envs x 100 steps; the 8 B/env of "
                                 "per-env results stay in L2, stream outputs scale with N*T",
                 "thread_inst_per_env_step": ops["thread"], "issue_slots_per_env_step": ops["slot"],
+                "fp32_lane_ops_per_env_step": ops.get("fp32"),
+                "counted_at": COUNTED_AT,
                 "peak_source": f"148 SMs x 4 schedulers x 32 lanes x {peaks['sm_max_mhz']:.0f} MHz ({peaks['source']} max clock)",
-                "note": "frac counts instructions executed by active lanes only; issue_slot_frac counts whole "
-                        "warp instructions x 32 (what the schedulers issue)"}
+                "note": "frac counts instructions executed by active lanes only in the per-lane formulation (what "
+                        "an environment needs); issue_slot_frac counts whole warp instructions x 32 of the kernel "
+                        "launched (a packed float32 instruction serves two environments in one slot); "
+                        "fp32_pipe_frac counts the float32 multiply/add/fma lane operations of the method "
+                        "against the same 128 lanes per SM and clock"}
     if w.streams:
         roofline["stream_write_gbs"] = n * T * 4.125 / (ms_per_step * 1e-3) / 1e9
         roofline["stream_write_frac_of_hbm"] = roofline["stream_write_gbs"] / peaks["hbm_gbs"]
@@ -282,7 +339,7 @@ def main() -> None:
 
     e2e_ms, _ = timed(e2e_step, max(3, args.steps // 2), 3)
     e2e_ms /= max(3, args.steps // 2)
-    e2e = {"value": world * n * T / (e2e_ms * 1e-3), "unit": UNIT,
+    e2e = {"value": job_envs * T / (e2e_ms * 1e-3), "unit": UNIT,
            "h2d_bytes_per_step": int(4 * inputs.N_WEIGHTS[w.policy]) + 24, "d2h_bytes_per_step": 8 * n + 16,
            "ms_per_step": e2e_ms,
            "note": "cp_rollout_host_shard: host scalars (n_envs, T, seed) and policy weights in; per-env returns and "
@@ -304,15 +361,28 @@ def main() -> None:
         o = oracle.rollout(sample, T, w.seed, w.policy, weights, nthreads=cores)
         dt = time.perf_counter() - t0
         same = float((o["ep_return_sum"] == ret[:sample].cpu().numpy()).mean()) if env_offset == 0 else None
+        one = min(n, 1 << 16)
+        t1 = time.perf_counter()
+        oracle.rollout(one, T, w.seed, w.policy, weights, nthreads=1)
+        dt1 = time.perf_counter() - t1
         cpu = {"value": sample * T / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": f"first {sample} envs x {T} steps of the workload, one pass, {dt:.2f} s",
-               "returns_identical_to_gpu": same}
+               "returns_identical_to_gpu": same,
+               "one_core": {"value": one * T / dt1, "unit": UNIT, "cores": 1,
+                            "sample": f"first {one} envs x {T} steps, one pass, {dt1:.2f} s"}}
 
     sharding.reduce_totals(tot)  # the only exchange the path has: 16 bytes, outside the timed region
+    # the other two rungs of the metric, inside the object the record keeps
+    for key, name in (("fused_step_hbm", "step_kernel"), ("ladder_hbm", "ladder")):
+        if key in paths:
+            e = paths[key]
+            roofline[name] = {"n_envs": e["n_envs"], "ms": e.get("ms_per_launch", e.get("ms_per_step")),
+                              "env_steps_per_sec": e["env_steps_per_sec"], **e["roofline"]}
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "ms_per_step_median": step_stats["median_ms"],
+            "ms_per_step_best": step_stats["best_ms"], "higher_is_better": True, "scaling": args.scaling,
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": workload_name(w),
                        "l2": "flushed between iterations (256 MiB fill outside the timed events)",
@@ -378,7 +448,8 @@ def measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args) -> dict:
     ms, _ = timed(fused_step, 20, 4)
     ms /= 20
     gbs = n * STEP_BYTES / (ms * 1e-3) / 1e9
-    out["fused_step_hbm"] = {"n_envs": n, "ms_per_launch": ms, "env_steps_per_sec": n / (ms * 1e-3),
+    out["fused_step_hbm"] = {"n_envs": n, "ms_per_launch": ms, "ms_median": LAST_TIMING["median_ms"],
+                             "ms_best": LAST_TIMING["best_ms"], "env_steps_per_sec": n / (ms * 1e-3),
                              "roofline": {"bound": "hbm", "kernel": "step_kernel", "achieved": gbs,
                                           "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs * 1e9 / hbm,
                                           "traffic": STEP_DRAM_BYTES_16M if n == 1 << 24 else None,
@@ -616,8 +687,6 @@ def measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args) -> dict:
         out[f"{name}_rollout"] = entry
         del outs
         torch.cuda.empty_cache()
-    if "fused_step_hbm" in out and args.workload == "c3":
-        pass
     return out
 
 

@@ -61,7 +61,12 @@
  *   start_j(seed,env,t)  = ((float)(H(K(stream 1), 4t+j)>>8) * 2^-24 - 0.5f) * 0.1f,
  *                          j=0..3 -> x, x_dot, theta, theta_dot of an episode that
  *                          begins at global time t (initial state: t of the reset;
- *                          after done at step t: t+1). Needs 4*(t+1) < 2^32.
+ *                          after done at step t: t+1). Steps exist for t < 2^30, so every
+ *                          start state an episode RUNS from has 4t+j < 2^32. The one start
+ *                          state of time 2^30 (handed over, never stepped from, when an episode
+ *                          ends on the very last permitted step) takes its counters mod 2^32,
+ *                          i.e. 0..3 — defined, shared with the reference implementation the
+ *                          tests use, and pinned by the end-of-time tests.
  */
 #ifndef CARTPOLE_H_
 #define CARTPOLE_H_
@@ -114,7 +119,9 @@ typedef struct cp_policy {
  * NULL (not produced). Per-step planes are time-major so that a warp writes one
  * contiguous 128-byte line per step. */
 typedef struct cp_returns {
-    float *ep_return_sum;  /* [n_envs] sum of the returns (= lengths) of episodes completed in the T steps */
+    float *ep_return_sum;  /* [n_envs] sum of the returns (= lengths) of episodes completed in the T steps;
+                              a whole number, exact in float32 up to 2^24 = 16,777,216 (any T below that;
+                              beyond it the value is rounded to float32 while `totals` stays exact) */
     uint32_t *ep_count;    /* [n_envs] number of completed episodes */
     uint64_t *totals;      /* [2] += {sum of ep_return_sum, sum of ep_count}; caller zeroes before the call */
     float *reward_stream;  /* [T][n_envs] reward of every step (1.0f) */
@@ -173,7 +180,10 @@ size_t cp_unfused_workspace_bytes(int64_t n_envs);
  *     (cp_last_error says so). The array (about 8.7 MiB) is resident on every GPU that loads
  *     this library until the process exits.
  *   - The first call on each device looks up the array's device address (with that device
- *     current) and keeps it; make that first call before starting any stream capture.
+ *     current) and keeps it. Where the CUDA runtime loads device code lazily, that first call
+ *     is also what brings the module holding the array onto the device, so only from then on
+ *     is the array resident and do calls leave the device's free memory untouched: make the
+ *     first call a warm-up, outside latency-critical code and before any stream capture.
  *   - All calls share the one array, which still holds the previous call's intermediates.
  *     Nothing in it needs to start at zero (each plane is fully rewritten before it is read),
  *     but two calls whose kernels overlap on the GPU (different streams, or different threads
@@ -196,11 +206,13 @@ void cp_free(cp_state *state);
 int cp_state_info(const cp_state *state, int64_t *n_envs, int64_t *plane_stride, uint32_t *seed,
                   uint32_t *t, uint32_t *env_offset, float **planes);
 
-/* Hashed actions of global step t for envs env_offset .. env_offset+n_envs-1 -> out DEVICE [n_envs]. */
+/* Sec. V-A (the random actions, drawn without a random-number kernel of their own): hashed actions
+ * of global step t for envs env_offset .. env_offset+n_envs-1 -> out DEVICE [n_envs]. */
 int cp_actions(int64_t n_envs, uint32_t seed, uint32_t t, uint32_t env_offset, uint8_t *out);
 
-/* cp_rollout for the env range [env_offset, env_offset + n_envs) of a larger job (one range
- * per GPU; no exchange is needed besides adding the ranks' `totals`). */
+/* Sec. V (N independent environments): cp_rollout for the env range [env_offset, env_offset +
+ * n_envs) of a larger job (one range per GPU; no exchange is needed besides adding the ranks'
+ * `totals`). The paper runs one GPU; the sharding itself has no counterpart there. */
 int cp_rollout_shard(uint32_t env_offset, int64_t n_envs, int64_t T, uint32_t seed,
                      const cp_policy *policy, const cp_returns *returns);
 
@@ -237,7 +249,11 @@ int cp_rollout_from(cp_state *state, int64_t T, uint32_t *ep_len, const cp_polic
  *     identical on more than 99.9 % of environments when the actions do not depend on the state
  *     (hashed or supplied actions: every restart re-synchronises the two arithmetics); under a
  *     state-feedback policy the per-step differences are amplified through the action choice and
- *     only the statistics (mean return, episode count) agree — use CP_ARITH_EXACT where
+ *     only the statistics (mean return, episode count) agree: measured on 40,000 environments,
+ *     identical returns on 96.3 % after 300 steps with a linear policy whose episodes last about
+ *     80 steps, on 100 % with a 4-16-2 network whose episodes last 9. What does hold under any
+ *     policy is the per-step contract: from the same state, the same action wherever the two
+ *     logits are 1e-5 apart, and then the tolerances above. Use CP_ARITH_EXACT where
  *     reproducibility against the per-op order matters.
  * struct_size must be sizeof(cp_rollout_args) (guards against a caller built for another layout).
  * state == NULL: start states of global time t0, env range [env_offset, env_offset + n_envs);
@@ -263,14 +279,16 @@ typedef struct cp_rollout_args {
 } cp_rollout_args;
 int cp_rollout_ex(const cp_rollout_args *args);
 
-/* cp_step with per-environment episode-length counters and the same optional step limit:
+/* Sec. V-C's step with CartPole-v1's episode limit (the paper names no limit; an option of this
+ * build): cp_step with per-environment episode-length counters and the same optional step limit:
  * ep_len DEVICE [n_envs] (16-byte aligned for the vector kernel) is incremented, compared with
  * max_episode_steps (0 = no limit; an env reaching it reports done = 1 and restarts) and reset to
  * 0 for finished environments. ep_len == NULL makes this cp_step (and then the limit must be 0). */
 int cp_step_ex(cp_state *state, const uint8_t *action, cp_state *out_state, float *reward, uint8_t *done,
                uint32_t *ep_len, uint32_t max_episode_steps);
 
-/* End-to-end forms with HOST buffers (pinned memory recommended): device staging buffers
+/* Plumbing, no counterpart in the paper (it times device-resident runs): end-to-end forms with
+ * HOST buffers (pinned memory recommended): device staging buffers
  * are owned by the library (grown on demand, released by cp_shutdown); the calls copy in,
  * launch, copy out and SYNCHRONISE the stream before returning.
  * cp_rollout_host: h_ep_return_sum [n_envs], h_ep_count [n_envs], h_totals [2] (overwritten).
@@ -302,7 +320,8 @@ void cp_set_stream(void *cuda_stream);
  * caller-provided, except the staging buffer of the HOST-buffer calls (always cudaMalloc). */
 int cp_set_allocator(void *(*alloc)(size_t), void (*release)(void *));
 
-/* Launch tuning, process-wide. key: "rollout_block" (threads per CTA, 32..256, multiple of 32;
+/* Launch tuning, process-wide (no counterpart in the paper; its analogue is XLA's flag for
+ * switching passes off, Sec. III). key: "rollout_block" (threads per CTA, 32..256, multiple of 32;
  * 0 = default: 128 for very small batches, else 256), "rollout_ept" (environments per thread: 1 or 2; 0 = default, 2 for large
  * batches except with the MLP policies), "rollout_coop" (how finished environments get their
  * start state: 1 = by the whole warp through shared memory, 2 = each lane its own when its env
@@ -311,8 +330,13 @@ int cp_set_allocator(void *(*alloc)(size_t), void (*release)(void *));
  * and start state ahead into shared memory (hashed or supplied actions and hashed start
  * states; otherwise as 2), 2, 3 and 4 only with one environment per
  * thread; 0 = default: helper warps for up to ten warps of environments per SM, per lane for
- * other batches too small to fill the GPU (ahead for the smaller ones), by the warp otherwise;
- * every choice gives the same bits), "rollout_ctas_per_sm" (0 = default: one 32*ept-environment task per warp and as many
+ * other batches too small to fill the GPU (ahead for the smaller ones), deferred (5) for batches
+ * that fill it where that form applies, by the warp otherwise;
+ * 5 = two environments per thread with a clock per environment and restarts deferred to every
+ * few loop trips (no per-step output streams; hashed actions or a linear policy; otherwise the
+ * default); every choice gives the same bits), "rollout_defer" (loop trips between the restart
+ * passes of that deferred form: 2, 3, 4, 6 or 8; 0 = default: 4 with hashed actions, else 6),
+ * "rollout_ctas_per_sm" (0 = default: one 32*ept-environment task per warp and as many
  * CTAs as that takes; k > 0 = persistent grid of k CTAs per SM looping over tasks), "step_block"
  * (32..256, default 64), "step_vec_min_envs" (batches smaller than this use the one-env-per-thread
  * step kernel even when the four-envs-per-thread vector form is possible; default 262144),
@@ -321,10 +345,13 @@ int cp_set_allocator(void *(*alloc)(size_t), void (*release)(void *));
  * Returns CP_EINVAL for an unknown key or value. */
 int cp_tune(const char *key, int value);
 
-/* Number of kernels this library has launched in this process (all threads). */
+/* Number of kernels this library has launched in this process (all threads). A measurement aid
+ * (the paper counts launches with a profiler, Sec. V-G); no counterpart as a call. */
 uint64_t cp_launch_count(void);
 
-/* Diagnostics: count float32 values v in [lo, hi] (bit patterns, both >= 0, lo <= hi, and their
+/* The cp_selftest_* calls below are diagnostics of this build's arithmetic shortcuts; the paper
+ * has no counterpart to any of them.
+ * Diagnostics: count float32 values v in [lo, hi] (bit patterns, both >= 0, lo <= hi, and their
  * negatives) for which the fused kernels' combined sine/cosine differs in any bit from the
  * ladder's separate sine and cosine kernels. mismatches DEVICE [1] uint64, caller zeroes. */
 int cp_selftest_sincos(uint32_t lo_bits, uint32_t hi_bits, uint64_t *mismatches);
@@ -341,7 +368,7 @@ int cp_selftest_sincos_accuracy(uint32_t lo_bits, uint32_t hi_bits, uint64_t *ou
  * negatives, largest value seen, in units of 1e-12. out DEVICE [2] uint64, caller zeroes. */
 int cp_selftest_tanh(uint32_t lo_bits, uint32_t hi_bits, uint64_t *out);
 
-/* Diagnostics: the kernels replace x / 1.1f by a three-operation exact sequence and the start-state
+/* Diagnostics: the kernels replace x / 1.1f by a two-operation exact sequence and the start-state
  * mapping by an equivalent two-operation one. This checks, over all 2^32 float bit patterns (2^24
  * for the mapping), that the replacements give the bits of the operations they stand for wherever
  * they are used. out DEVICE [4] uint64, caller zeroes; every count must come back 0. */

@@ -370,6 +370,9 @@ typedef struct {
     float *final_state;      /* [4][n] or NULL */
     float *trajectory;       /* [T][4][n] or NULL: state after step t (after any reset) */
     float *min_gap;          /* [n] or NULL: smallest |logit1-logit0| seen */
+    float *min_margin;       /* [n] or NULL: smallest distance of an updated |x| or |theta| from its
+                                termination threshold seen (a diagnostic for the comparison rules:
+                                "bit-exact wherever no state is within 1e-5 of a threshold") */
     uint32_t max_steps;      /* episode step limit (CartPole-v1 uses 500); 0 = none */
     const uint32_t *action_bits_in; /* [T][ceil(n/32)] supplied actions (bit i%32 of word i/32) or NULL */
     const float *start_states_in;   /* [T][4][n] supplied start states or NULL: an env that finishes at
@@ -397,6 +400,7 @@ static void co_rollout_range(co_rollout_job *J)
         uint32_t ep_len = J->ep_len_io ? J->ep_len_io[i] : 0u;
         uint32_t ret_sum = 0, ep_cnt = 0;
         float min_gap = INFINITY;
+        double min_margin = INFINITY;
         for (int64_t k = 0; k < T; ++k) {
             uint32_t t = J->t0 + (uint32_t)k;
             float gap;
@@ -416,6 +420,11 @@ static void co_rollout_range(co_rollout_job *J)
             }
             if (gap < min_gap) min_gap = gap;
             int d = co_dynamics_f32(z, a, zn);
+            if (J->min_margin) {
+                double mx = fabs(fabs((double)zn[0]) - (double)CO_XT), mt = fabs(fabs((double)zn[2]) - (double)CO_TT);
+                if (mx < min_margin) min_margin = mx;
+                if (mt < min_margin) min_margin = mt;
+            }
             ep_len += 1u; /* reward 1 per step, terminating step included */
             /* an episode that has lasted max_steps steps is cut off: it counts as finished
              * (done = 1, its return is its length) and the env restarts like after a fall */
@@ -445,6 +454,7 @@ static void co_rollout_range(co_rollout_job *J)
             for (int p = 0; p < 4; ++p)
                 J->final_state[p * n + i] = z[p];
         if (J->min_gap) J->min_gap[i] = min_gap;
+        if (J->min_margin) J->min_margin[i] = (float)min_margin;
         tot_ret += ret_sum;
         tot_cnt += ep_cnt;
     }
@@ -466,7 +476,7 @@ void co_rollout_ex(uint32_t env_offset, int64_t n, int64_t T, uint32_t seed, uin
                    float *ep_return_sum, uint32_t *ep_count, uint64_t *totals, float *reward_stream,
                    uint32_t *done_bits, uint32_t *action_bits, float *final_state, float *trajectory,
                    float *min_gap, int nthreads, uint32_t max_steps, const uint32_t *action_bits_in,
-                   const float *start_states_in)
+                   const float *start_states_in, float *min_margin)
 {
     if (nthreads < 1) nthreads = 1;
     if (nthreads > 256) nthreads = 256;
@@ -481,8 +491,8 @@ void co_rollout_ex(uint32_t env_offset, int64_t n, int64_t T, uint32_t seed, uin
         if (hi > n) hi = n;
         co_rollout_job J = {env_offset, n, T, seed, t0, kind, weights, init_state, ep_len_io,
                             ep_return_sum, ep_count, reward_stream, done_bits, action_bits,
-                            final_state, trajectory, min_gap, max_steps, action_bits_in, start_states_in,
-                            lo, hi, 0, 0};
+                            final_state, trajectory, min_gap, min_margin, max_steps, action_bits_in,
+                            start_states_in, lo, hi, 0, 0};
         jobs[used++] = J;
     }
     if (used == 1) {
@@ -509,7 +519,7 @@ void co_rollout(uint32_t env_offset, int64_t n, int64_t T, uint32_t seed, uint32
 {
     co_rollout_ex(env_offset, n, T, seed, t0, kind, weights, init_state, ep_len_io, ep_return_sum, ep_count,
                   totals, reward_stream, done_bits, action_bits, final_state, trajectory, min_gap, nthreads,
-                  0u, NULL, NULL);
+                  0u, NULL, NULL, NULL);
 }
 
 /* co_step with an episode step limit: ep_len [n] holds the steps already taken in each

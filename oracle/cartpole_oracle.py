@@ -83,7 +83,7 @@ def lib() -> C.CDLL:
         L.co_rollout.restype = None
         L.co_rollout.argtypes = [u32, i64, i64, u32, u32, i32, p, p, p, p, p, p, p, p, p, p, p, p, i32]
         L.co_rollout_ex.restype = None
-        L.co_rollout_ex.argtypes = [u32, i64, i64, u32, u32, i32, p, p, p, p, p, p, p, p, p, p, p, p, i32, u32, p, p]
+        L.co_rollout_ex.argtypes = [u32, i64, i64, u32, u32, i32, p, p, p, p, p, p, p, p, p, p, p, p, i32, u32, p, p, p]
         L.co_step_limited.restype = None
         L.co_step_limited.argtypes = [u32, i64, i64, i64, u32, u32, p, p, p, p, p, p, u32]
         _lib = L
@@ -220,14 +220,16 @@ def rollout(n: int, T: int, seed: int, policy_kind: int = POLICY_RANDOM, weights
             ep_len: np.ndarray | None = None, per_env: bool = True,
             reward_stream: bool = False, done_bits: bool = False,
             action_bits: bool = False, final_state: bool = False, trajectory: bool = False,
-            min_gap: bool = False, nthreads: int = 1, max_episode_steps: int = 0,
+            min_gap: bool = False, min_margin: bool = False, nthreads: int = 1, max_episode_steps: int = 0,
             action_bits_in: np.ndarray | None = None, start_states_in: np.ndarray | None = None) -> dict:
     """Rollout of n envs for T steps. Returns a dict of the requested outputs.
 
     max_episode_steps > 0 cuts episodes off at that length; action_bits_in ([T, ceil(n/32)]
     uint32, bit i%32 of word i//32) supplies the actions instead of the policy;
     start_states_in (float32 [T, 4, n]) supplies the start states: an env that finishes at the
-    k-th step of the call continues from row k instead of the hashed start state."""
+    k-th step of the call continues from row k instead of the hashed start state.
+    min_gap / min_margin report, per env, the smallest policy logit gap and the smallest distance
+    of an updated |x| or |theta| from its termination threshold seen during the rollout."""
     w = None
     if policy_kind != POLICY_RANDOM:
         w = np.ascontiguousarray(weights, np.float32).ravel()
@@ -244,6 +246,7 @@ def rollout(n: int, T: int, seed: int, policy_kind: int = POLICY_RANDOM, weights
         "final_state": np.empty((4, n), np.float32) if final_state else None,
         "trajectory": np.empty((T, 4, n), np.float32) if trajectory else None,
         "min_gap": np.empty(n, np.float32) if min_gap else None,
+        "min_margin": np.empty(n, np.float32) if min_margin else None,
     }
     if init_state is not None:
         init_state = np.ascontiguousarray(init_state, np.float32)
@@ -262,7 +265,8 @@ def rollout(n: int, T: int, seed: int, policy_kind: int = POLICY_RANDOM, weights
                         _ptr(res["ep_return_sum"]), _ptr(res["ep_count"]), _ptr(res["totals"]),
                         _ptr(res["reward_stream"]), _ptr(res["done_bits"]), _ptr(res["action_bits"]),
                         _ptr(res["final_state"]), _ptr(res["trajectory"]), _ptr(res["min_gap"]),
-                        int(nthreads), int(max_episode_steps), _ptr(action_bits_in), _ptr(start_states_in))
+                        int(nthreads), int(max_episode_steps), _ptr(action_bits_in), _ptr(start_states_in),
+                        _ptr(res["min_margin"]))
     return res
 
 

@@ -13,8 +13,7 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-# CARTPOLE_LIB selects another build of the same library (tuning experiments).
-LIB_PATH = os.environ.get("CARTPOLE_LIB") or os.path.join(_HERE, "libcartpole.so")
+LIB_PATH = os.path.join(_HERE, "libcartpole.so")
 
 CP_OK, CP_EINVAL, CP_ECUDA, CP_ENOMEM = 0, -1, -2, -3
 CP_POLICY_RANDOM, CP_POLICY_LINEAR, CP_POLICY_MLP, CP_POLICY_MLP32, CP_POLICY_MLP64 = 0, 1, 2, 4, 5

@@ -38,20 +38,31 @@ def _nvcc() -> str:
     return "nvcc"
 
 
-def source_hash(extra: list[str] | None = None) -> str:
+def source_hash() -> str:
     h = hashlib.sha256()
     for name in SOURCES + HEADERS:
         with open(os.path.normpath(os.path.join(CSRC, name)), "rb") as f:
             h.update(name.encode() + b"\0" + f.read() + b"\0")
-    h.update(" ".join(NVCC_FLAGS + (extra or [])).encode())
+    h.update(" ".join(NVCC_FLAGS).encode())
     return h.hexdigest()
 
 
-def _compile_and_link(out: str, extra: list[str], verbose: bool) -> None:
+def kernel_hash() -> str:
+    """Hash of the files and flags that determine the instruction streams of the rollout and step
+    kernels (bench.py records it beside the per-env-step instruction counts it was given)."""
+    h = hashlib.sha256()
+    for name in ("cartpole_device.cuh", "rollout_kernel.cuh", "rollout_deferred.cu", "step_kernel.cu"):
+        with open(os.path.join(CSRC, name), "rb") as f:
+            h.update(name.encode() + b"\0" + f.read() + b"\0")
+    h.update(" ".join(NVCC_FLAGS).encode())
+    return h.hexdigest()[:16]
+
+
+def _compile_and_link(out: str, verbose: bool) -> None:
     with tempfile.TemporaryDirectory() as tmp:
         def compile_one(src: str) -> str:
             o = os.path.join(tmp, src.replace(".cu", ".o"))
-            cmd = [_nvcc(), *NVCC_FLAGS, *extra, "-c", os.path.join(CSRC, src), "-o", o]
+            cmd = [_nvcc(), *NVCC_FLAGS, "-c", os.path.join(CSRC, src), "-o", o]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
                 print(" ".join(cmd), flush=True)
@@ -66,16 +77,12 @@ def _compile_and_link(out: str, extra: list[str], verbose: bool) -> None:
         os.replace(tmp_out, out)
 
 
-def build(force: bool = False, verbose: bool = False, extra: list[str] | None = None, out: str | None = None) -> str:
-    """Compile and link if needed. `extra` adds nvcc flags (e.g. -DCP_ROLLOUT_MIN_CTAS=5) and `out`
-    names another output file; both are for tuning experiments and always rebuild."""
-    if extra or out:
-        _compile_and_link(out or LIB, extra or [], verbose)
-        return out or LIB
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Compile and link if the library is missing or older than its sources (by hash)."""
     want = source_hash()
     have = open(STAMP).read().strip() if os.path.exists(STAMP) else ""
     if force or not os.path.exists(LIB) or have != want:
-        _compile_and_link(LIB, [], verbose)
+        _compile_and_link(LIB, verbose)
         with open(STAMP, "w") as f:
             f.write(want + "\n")
     return LIB

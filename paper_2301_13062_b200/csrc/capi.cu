@@ -143,6 +143,13 @@ int rollout_impl(uint32_t env_offset, int64_t n_envs, int64_t T, uint32_t seed, 
     if ((rc = check_policy(policy, &kind)) != CP_OK) return rc;
     if (!ret) return fail(CP_EINVAL, "returns is NULL");
     if (ret->totals && !is_aligned(ret->totals, 8)) return fail(CP_EINVAL, "totals must be 8-byte aligned");
+    // every other output is stored in 4-byte units: a misaligned pointer would fault on the device
+    const struct { const void *p; const char *name; } four_byte[] = {
+        {ret->ep_return_sum, "ep_return_sum"}, {ret->ep_count, "ep_count"}, {ret->reward_stream, "reward_stream"},
+        {ret->done_bits, "done_bits"}, {ret->action_bits, "action_bits"}, {ret->trajectory, "trajectory"},
+        {out_planes, "final_state"}, {init_planes, "state planes"}, {ep_len, "ep_len"}, {action_bits_in, "action_bits_in"}};
+    for (const auto &q : four_byte)
+        if (q.p && !is_aligned(q.p, 4)) return fail(CP_EINVAL, "%s is not 4-byte aligned", q.name);
     cp::RolloutParams p;
     memset(&p, 0, sizeof p);
     p.n = n_envs;

@@ -115,7 +115,11 @@ __global__ void __launch_bounds__(64 * PAIRS) rollout_assisted_kernel(const __gr
     const bool producer = warp >= (uint32_t)PAIRS;
     const uint32_t pair = producer ? warp - PAIRS : warp;
     const int64_t task = (int64_t)blockIdx.x * PAIRS + pair;
-    if (task >= p.n_tasks) return;  // both warps of the pair leave; no other pair uses their barrier
+    // Both warps of a pair leave here together, before their first barrier; no other pair uses
+    // their barrier. Nothing that differs between the two warps of a pair (or between lanes) may
+    // decide an exit or a barrier from here on: each warp must execute exactly 1 + n_chunks
+    // barriers, a count fixed by the launch parameters, or its partner waits for ever.
+    if (task >= p.n_tasks) return;
     PairBuffers<kChunk> &buf = s_buf[pair];
     const uint32_t n_chunks = (p.T + kChunk - 1) / kChunk;
 

@@ -47,13 +47,6 @@ __device__ __forceinline__ uint32_t policy_signbit(const RolloutParams &p, const
     }
 }
 
-#ifndef CP_ROLLOUT_MIN_CTAS
-#define CP_ROLLOUT_MIN_CTAS 1
-#endif
-#ifndef CP_CONTRACT_MIN_CTAS
-#define CP_CONTRACT_MIN_CTAS 1
-#endif
-
 constexpr int kMaxWarpsPerCta = 8;  // __launch_bounds__(256)
 
 // SHAPE: how a warp holds and restarts its environments.
@@ -74,17 +67,12 @@ constexpr int kMaxWarpsPerCta = 8;  // __launch_bounds__(256)
 // LIMIT: episodes are cut off after p.max_steps steps.
 // CONTRACT: the contracted arithmetic of euler_step_contracted instead of the canonical order.
 template <int POLICY, int SHAPE, int STREAMS, bool LIMIT, bool CONTRACT>
-__global__ void __launch_bounds__(256, CONTRACT ? CP_CONTRACT_MIN_CTAS : CP_ROLLOUT_MIN_CTAS)
-    rollout_kernel(const __grid_constant__ RolloutParams p) {
+__global__ void __launch_bounds__(256) rollout_kernel(const __grid_constant__ RolloutParams p) {
     constexpr int EPT = SHAPE == 2 ? 2 : 1;
     constexpr bool COOP = SHAPE == 1 || SHAPE == 2;
     constexpr bool AHEAD = SHAPE == 3;
     constexpr bool START_IN = SHAPE == 4;
-#ifdef CP_EXP_NOPAIR
-    constexpr bool PAIR = false;
-#else
     constexpr bool PAIR = SHAPE == 2 && !CONTRACT;  // packed two-env arithmetic
-#endif
     const uint32_t lane = threadIdx.x & 31u;
     // Per warp: key pairs of up to 8 finished envs, and their 8 x 4 start-state components.
     __shared__ uint2 s_keys[COOP ? kMaxWarpsPerCta : 1][8];

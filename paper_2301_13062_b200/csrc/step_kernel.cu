@@ -19,17 +19,13 @@ __device__ __forceinline__ uint32_t hashed_signbit(const StepParams &p, uint32_t
     return action_signbit(make_keys(p.salt_a, env), p.t);
 }
 
-#ifndef CP_STEP_MIN_CTAS
-#define CP_STEP_MIN_CTAS 1
-#endif
-
 // The kernel is written for programmatic dependent launch: everything that does not depend on
 // what the previous launch wrote (the action hashes, about a quarter of the instructions) comes
 // first; then the kernel waits for the previous launch's memory to be visible and immediately
 // lets the next launch begin its own preamble. Launched without that attribute the two
 // grid-dependency instructions do nothing.
 template <bool VEC>
-__global__ void __launch_bounds__(256, CP_STEP_MIN_CTAS) step_kernel(const __grid_constant__ StepParams p) {
+__global__ void __launch_bounds__(256) step_kernel(const __grid_constant__ StepParams p) {
     const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const bool has_action = p.action != nullptr;
     if (VEC) {

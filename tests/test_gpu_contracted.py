@@ -172,3 +172,45 @@ def test_unknown_arithmetic_is_rejected(cp):
     ret = torch.empty(8, device="cuda")
     with pytest.raises(cp.CartpoleError):
         cp.cp_rollout_ex(n_envs=8, T=1, arithmetic=2, ep_return_sum=ret)
+
+
+@pytest.mark.parametrize("kind,pseed", [(1, 1), (2, 2), (7, 7)])
+def test_contracted_steps_under_feedback_policies_follow_the_oracle_step_by_step(cp, oracle, kind, pseed):
+    """Where the per-step contract CAN hold under a state-feedback policy: teacher-forced. Along a
+    200-step trajectory of the oracle, every step is launched (T = 1) from the oracle's own
+    states; the action must be the oracle's wherever its logits are 1e-5 apart, and with the same
+    action the new state must be within 2e-6 relative, the done flag equal outside the 1e-5
+    threshold band and the start state of a finished env bit-exact. (Free-running, the same
+    differences feed back through the action choice; see the statistical test above.)"""
+    n, T, seed, off = 2000, 200, 5, 40
+    wts = inputs.policy_weights(kind, pseed)
+    pol = cp.policy(kind, wts)
+    words = (n + 31) // 32
+    z = oracle.initial_state(n, seed, 0, off)
+    planes = torch.zeros(4, n, dtype=torch.float32, device="cuda")
+    ties = flips = 0
+    for t in range(T):
+        o1 = oracle.rollout(n, 1, seed, kind, wts, env_offset=off, t0=t, init_state=z, action_bits=True,
+                            min_gap=True, final_state=True)
+        o_act = H.unpack_bits(o1["action_bits"], n)[0]
+        want = oracle.step(z, seed, t, action_u8=o_act, env_offset=off, want_pre_reset=True)
+        assert np.array_equal(want["state"].view(np.uint32), o1["final_state"].view(np.uint32))
+        planes.copy_(dev(z))
+        st = cp.cp_wrap(planes, n, seed, t, off)
+        out = {"reward_stream": torch.zeros(1, n, device="cuda"),
+               "done_bits": torch.zeros(1, words, dtype=torch.int32, device="cuda"),
+               "action_bits": torch.zeros(1, words, dtype=torch.int32, device="cuda")}
+        cp.cp_rollout_ex(state=st, T=1, policy=pol, arithmetic=cp.CP_ARITH_CONTRACTED, **out)
+        torch.cuda.synchronize()
+        g_act = H.unpack_bits(host(out["action_bits"]), n)[0]
+        g_done = H.unpack_bits(host(out["done_bits"]), n)[0]
+        differ = g_act != o_act
+        assert not np.any(differ & (o1["min_gap"] >= 1e-5)), "action differs although the logits are 1e-5 apart"
+        ties += int((o1["min_gap"] < 1e-5).sum())
+        flips += int(differ.sum())
+        keep = ~differ
+        sub = {k: (v[:, keep] if v.ndim == 2 else v[keep]) for k, v in want.items()}
+        H.assert_step_matches(sub, z[:, keep], host(planes)[:, keep], host(out["reward_stream"])[0][keep],
+                              g_done[keep], g_act[keep])
+        z = want["state"]
+    assert flips <= ties

@@ -90,7 +90,8 @@ def test_random_combination_against_oracle(cp, oracle, case):
     torch.cuda.synchronize()
     r = {k: v.cpu().numpy() for k, v in out.items()}
     o = oracle.rollout(n, T, seed, kind, weights, env_offset=off, t0=t0, max_episode_steps=limit,
-                       done_bits=True, action_bits=True, final_state=True, min_gap=True, **ora_kw)
+                       done_bits=True, action_bits=True, final_state=True, min_gap=True, min_margin=True,
+                       **ora_kw)
 
     ret, cnt = r["ep_return_sum"], r["ep_count"].view(np.uint32)
     same = (ret == o["ep_return_sum"]) & (cnt == o["ep_count"])
@@ -99,14 +100,19 @@ def test_random_combination_against_oracle(cp, oracle, case):
         # statistics only (per-step differences feed back through the action choice)
         assert same.mean() >= 0.9 or n < 100
     else:
-        excused = same | (o["min_gap"] < 1e-5)
-        # a last-bit sine/cosine difference may flip a done flag inside the 1e-5 band: rare
-        assert excused.sum() >= n - max(1, n // 500), (n, int((~excused).sum()))
+        # excused: an env that came within 1e-5 of a logit tie or of a termination threshold (a
+        # last-bit sine/cosine difference may then take the other branch); of the rest 99.9 % must
+        # have identical returns
+        excused = same | (o["min_gap"] < 1e-5) | (o["min_margin"] < 1e-5)
+        # (the contracted arithmetic differs from the oracle by a few 1e-7 per step, which an
+        # episode can grow past the 1e-5 band: one env is always tolerated there)
+        allowed = max(1, n // 1000) if contracted else n // 1000
+        assert excused.sum() >= n - allowed, (n, int((~excused).sum()))
     assert int(r["totals"][0]) == int(ret.astype(np.int64).sum())
     assert int(r["totals"][1]) == int(cnt.astype(np.int64).sum())
     # An env that came within 1e-5 of a threshold or of a logit tie may have taken the other branch
     # once and still show the same returns: per-step bits and states are compared on the others.
-    sure = same & (o["min_gap"] >= 1e-5)
+    sure = same & (o["min_gap"] >= 1e-5) & (o["min_margin"] >= 1e-5)
     if "done_bits" in r:
         gd, od = H.unpack_bits(r["done_bits"], n), H.unpack_bits(o["done_bits"], n)
         assert np.array_equal(gd.sum(axis=0), cnt)

@@ -361,44 +361,54 @@ def test_policy_rollouts_against_oracle(cp, oracle, kind, pseed, n, T):
     assert np.array_equal(gd.sum(axis=0), r["ep_count"])
 
 
-def test_full_size_policy_configs_on_sampled_envs(cp, oracle):
+@pytest.mark.parametrize("name", ["c4", "c5"])
+def test_full_size_policy_configs_against_oracle(cp, oracle, name):
     """Configs 4 (4,194,304 x 1,000, linear policy, reward plane + done bitmask) and 5
-    (16,777,216 x 200, MLP policy) exactly as bench.py launches them; the oracle recomputes
-    sampled env ranges one by one (results of an env do not depend on its neighbours)."""
-    for name in ("c4", "c5"):
-        w = inputs.WORKLOADS[name]
-        wts = inputs.policy_weights(w.policy, w.policy_seed)
-        n, T = w.n_envs, w.T
-        words = (n + 31) // 32
-        outs = {"ep_return_sum": torch.empty(n, dtype=torch.float32, device="cuda"),
-                "ep_count": torch.empty(n, dtype=torch.int32, device="cuda"),
-                "totals": torch.zeros(2, dtype=torch.int64, device="cuda")}
+    (16,777,216 x 200, MLP policy) exactly as bench.py launches them. The oracle recomputes the
+    first 1,048,576 environments for all T steps, a range in the middle and the last 4,992 (results of
+    an env do not depend on its neighbours): returns identical on >= 99.9 % of the envs that stayed
+    1e-5 clear of every logit tie and termination threshold, and so is the whole done bit stream."""
+    import os
+    w = inputs.WORKLOADS[name]
+    wts = inputs.policy_weights(w.policy, w.policy_seed)
+    n, T = w.n_envs, w.T
+    words = (n + 31) // 32
+    outs = {"ep_return_sum": torch.empty(n, dtype=torch.float32, device="cuda"),
+            "ep_count": torch.empty(n, dtype=torch.int32, device="cuda"),
+            "totals": torch.zeros(2, dtype=torch.int64, device="cuda")}
+    if w.streams:
+        outs["reward_stream"] = torch.empty(T, n, dtype=torch.float32, device="cuda")
+        outs["done_bits"] = torch.empty(T, words, dtype=torch.int32, device="cuda")
+    cp.cp_rollout(n, T, w.seed, cp.policy(w.policy, wts), **outs)
+    torch.cuda.synchronize()
+    ret, cnt = host(outs["ep_return_sum"]), host(outs["ep_count"]).view(np.uint32)
+    cores = os.cpu_count() or 1
+    for lo, m in ((0, 1 << 20), (n // 2 - 1024, 2048), (n - 4992, 4992)):
+        o = oracle.rollout(m, T, w.seed, w.policy, wts, env_offset=lo, min_gap=True, min_margin=True,
+                           done_bits=w.streams, nthreads=cores)
+        excuse = (o["min_gap"] < 1e-5) | (o["min_margin"] < 1e-5)
+        H.assert_returns_match(ret[lo:lo + m], cnt[lo:lo + m], o["ep_return_sum"], o["ep_count"], excuse,
+                               min_identical=0.999)
         if w.streams:
-            outs["reward_stream"] = torch.empty(T, n, dtype=torch.float32, device="cuda")
-            outs["done_bits"] = torch.empty(T, words, dtype=torch.int32, device="cuda")
-        cp.cp_rollout(n, T, w.seed, cp.policy(w.policy, wts), **outs)
-        torch.cuda.synchronize()
-        ret, cnt = host(outs["ep_return_sum"]), host(outs["ep_count"]).view(np.uint32)
-        m = 2048
-        for lo in (0, n // 2 - 1024, n - m):
-            o = oracle.rollout(m, T, w.seed, w.policy, wts, env_offset=lo, min_gap=True, done_bits=w.streams)
-            excuse = o["min_gap"] < 1e-5
-            H.assert_returns_match(ret[lo:lo + m], cnt[lo:lo + m], o["ep_return_sum"], o["ep_count"], excuse,
-                                   min_identical=0.998)
-            if w.streams:
-                gd = H.unpack_bits(host(outs["done_bits"][:, lo // 32:(lo + m) // 32]), m)
-                od = H.unpack_bits(o["done_bits"], m)
-                same_env = (ret[lo:lo + m] == o["ep_return_sum"]) & (cnt[lo:lo + m] == o["ep_count"])
-                assert np.array_equal(gd[:, same_env], od[:, same_env])
-                assert np.array_equal(gd.sum(axis=0), cnt[lo:lo + m])
-                assert bool((outs["reward_stream"][:, lo:lo + m] == 1.0).all())
-        tot = host(outs["totals"]).view(np.uint64)
-        assert int(tot[1]) == int(cnt.astype(np.int64).sum())
-        assert int(tot[0]) == int(ret.astype(np.float64).sum())
-        if w.streams:  # every row of the reward plane was written, every done bit is accounted for
-            assert float(outs["reward_stream"].min()) == 1.0 and float(outs["reward_stream"].max()) == 1.0
-        del outs
-        torch.cuda.empty_cache()
+            gd = host(outs["done_bits"][:, lo // 32:(lo + m) // 32]).view(np.uint32)
+            # the whole done bit stream, step by step: identical on >= 99.9 % of the envs that stayed
+            # clear of the bands (under a feedback policy a last-bit sine difference can grow past
+            # 1e-5 within an 80-step episode; measured: 132 of 1,048,576 such envs differ somewhere)
+            diff = np.bitwise_or.reduce(gd ^ o["done_bits"], axis=0)
+            differs = np.unpackbits(diff.view(np.uint8), bitorder="little").astype(bool)
+            assert int((differs & ~excuse).sum()) <= m // 1000
+            pop = np.zeros(m, np.int64)
+            for k in range(32):                                       # done bits per env == its episode count
+                pop[k::32] = ((gd >> np.uint32(k)) & np.uint32(1)).sum(axis=0)
+            assert np.array_equal(pop, cnt[lo:lo + m])
+            assert bool((outs["reward_stream"][:, lo:lo + min(m, 65536)] == 1.0).all())
+    tot = host(outs["totals"]).view(np.uint64)
+    assert int(tot[1]) == int(cnt.astype(np.int64).sum())
+    assert int(tot[0]) == int(ret.astype(np.float64).sum())
+    if w.streams:  # every row of the reward plane was written
+        assert float(outs["reward_stream"].min()) == 1.0 and float(outs["reward_stream"].max()) == 1.0
+    del outs
+    torch.cuda.empty_cache()
 
 
 def test_config2_step_path_at_full_size(cp, oracle):

@@ -102,6 +102,29 @@ def test_binding_structs_have_the_layout_the_header_declares(cp, tmp_path):
         assert len(members) == len(cls._fields_), (name, members)
 
 
+def test_misaligned_rollout_outputs_are_refused_before_any_launch(cp):
+    """Every cp_returns member is stored in 4-byte units (totals in 8-byte units): an odd pointer
+    must come back as CP_EINVAL from the host-side checks, never reach a kernel (no GPU is needed
+    for this test, and none must be touched)."""
+    L = cp.lib()
+    before = L.cp_launch_count()
+    base = 0x7000_0000_0000
+    for field in ("ep_return_sum", "ep_count", "reward_stream", "done_bits", "action_bits", "final_state",
+                  "trajectory", "totals"):
+        for odd in (1, 2, 3) if field != "totals" else (4,):
+            r = cp.cp_returns()
+            setattr(r, field, base + odd)
+            assert L.cp_rollout(64, 10, 0, None, C.byref(r)) == cp.CP_EINVAL, field
+            assert field.encode() in L.cp_last_error() or b"aligned" in L.cp_last_error()
+    a = cp.cp_rollout_args()
+    a.struct_size = C.sizeof(cp.cp_rollout_args)
+    r = cp.cp_returns()
+    a.n_envs, a.T, a.returns = 64, 10, C.pointer(r)
+    a.ep_len = base + 2
+    assert L.cp_rollout_ex(C.byref(a)) == cp.CP_EINVAL
+    assert L.cp_launch_count() == before
+
+
 def test_general_rollout_rejects_bad_arguments_on_the_host(cp):
     L = cp.lib()
     r = cp.cp_returns()

@@ -184,3 +184,21 @@ def test_policy_rollout_uses_pre_step_observation_and_tie_rule(oracle):
     wm = inputs.policy_weights(inputs.POLICY_MLP, 2)
     rm = oracle.rollout(16, 20, 0, inputs.POLICY_MLP, wm, min_gap=True)
     assert np.all(np.isfinite(rm["min_gap"])) and rm["totals"][1] > 0
+
+
+def test_threshold_margin_diagnostic_matches_a_walk(oracle):
+    """min_margin (used by the GPU comparison rules to excuse envs that came within 1e-5 of a
+    termination threshold) against a per-env walk composed from the scalar calls."""
+    n, T, seed = 40, 120, 6
+    r = oracle.rollout(n, T, seed, min_margin=True, done_bits=True)
+    xt, tt = float(np.float32(2.4)), float(np.float32(12 * 2 * np.pi / 360))
+    for i in range(n):
+        z = oracle.reset_state(seed, i, 0)
+        best = np.inf
+        for t in range(T):
+            zn, d = oracle.dynamics_f32(z, oracle.action(seed, i, t))
+            best = min(best, abs(abs(float(zn[0])) - xt), abs(abs(float(zn[2])) - tt))
+            z = oracle.reset_state(seed, i, t + 1) if d else zn
+        assert r["min_margin"][i] == np.float32(best)
+    # an env that terminates has passed a threshold by less than one step's travel
+    assert (r["min_margin"] < 0.05).all() and (r["min_margin"] >= 0).all()

@@ -76,5 +76,29 @@ def test_noalloc_step_rejects_oversized_batches(cp):
         cp.cp_step_unfused_noalloc(s_in, None, s_out, reward, done)
     assert e.value.code == cp.CP_EINVAL and "CP_NOALLOC_MAX_ENVS" in str(e.value)
     assert cp.cp_launch_count() == before and s_out.info()["t"] == 0
-    with pytest.raises(cp.CartpoleError):
+
+
+def test_noalloc_step_refuses_in_place_use_and_takes_no_device_memory(cp):
+    n = 4096
+    z = inputs.random_states(n, seed=1, spread="live")
+    pin, pout = _planes(n, z), _planes(n)
+    s_in, s_out = cp.cp_wrap(pin, n, 0), cp.cp_wrap(pout, n, 0)
+    reward = torch.empty(n, dtype=torch.float32, device="cuda")
+    done = torch.empty(n, dtype=torch.uint8, device="cuda")
+    # in place (a size the call accepts otherwise): refused on the host, nothing launched
+    before = cp.cp_launch_count()
+    with pytest.raises(cp.CartpoleError) as e:
         cp.cp_step_unfused_noalloc(s_in, None, s_in, reward, done)
+    assert e.value.code == cp.CP_EINVAL and "in place" in str(e.value)
+    assert cp.cp_launch_count() == before and s_in.info()["t"] == 0
+    # a call after the first one on this device (which may have loaded the module that holds the
+    # array) leaves the device's free memory exactly as it found it
+    cp.cp_step_unfused_noalloc(s_in, None, s_out, reward, done)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    cp.cp_set_time(s_in, 0)
+    cp.cp_step_unfused_noalloc(s_in, None, s_out, reward, done)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    assert cp.cp_launch_count() - before == 2 * 46
