@@ -23,9 +23,10 @@
 // the price is idle slots (about 7 % at K = 4 with the random policy's 22-step episodes) and a
 // ragged end.
 //
-// Scope: no per-step output streams (they are rows of global time); hashed actions, the shared
-// linear policy or one linear policy per environment; canonical arithmetic; with or without the
-// episode step limit. Everything else takes the general kernel.
+// Scope: hashed actions, the shared linear policy or one linear policy per environment; canonical
+// arithmetic; with or without the episode step limit; per-step outputs either none or exactly the
+// reward plane + done bitmask (the action bitmask and the trajectory are rows of global time that
+// half the lanes would have to touch every step). Everything else takes the general kernel.
 //
 // No warp waits for another one and nothing spins: the loop's trip count is bounded by the
 // launch parameters (every trip block advances every unfinished slot by at least one step).
@@ -49,7 +50,8 @@ __device__ __forceinline__ uint32_t deferred_action(const RolloutParams &p, cons
 
 // POLICY: 0 hashed actions, 1 shared linear policy, 6 one linear policy per environment.
 // K: trips between restart passes. LIMIT: episodes are cut off after p.max_steps steps.
-template <int POLICY, int K, bool SHORT, bool LIMIT>
+// RD: the reward plane and the done bitmask are written (see the comment at reward_row).
+template <int POLICY, int K, bool SHORT, bool LIMIT, bool RD>
 __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_constant__ RolloutParams p) {
     const uint32_t lane = threadIdx.x & 31u;
     const int64_t task = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -91,6 +93,35 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
         }
         StatePair zz = pack_states(z0[0], z0[1]);
 
+        // Per-step outputs although the environments run on clocks of their own (RD):
+        //  * every step of every environment earns reward 1, so row r of the reward plane does not
+        //    depend on any clock: the warp writes it for its 64 environments in trip r, as full lines;
+        //  * a done bit is rare. The warp first clears its two words of every row, then an
+        //    environment whose episode ended at step t sets its bit in row t - t0 with one atomic
+        //    OR — in the restart pass, where its stopped clock still tells that time.
+        const int64_t words = (p.n + 31) >> 5;
+        const int64_t word0 = task * 2;
+        float *rew_row = RD ? p.reward_stream + base + lane : nullptr;
+        if (RD) {
+            for (uint32_t r = lane; r < p.T; r += 32u) {
+                if (word0 < words) p.done_bits[(int64_t)r * words + word0] = 0u;
+                if (word0 + 1 < words) p.done_bits[(int64_t)r * words + word0 + 1] = 0u;
+            }
+            __syncwarp();  // orders the clearing stores before any lane's later atomic on the same word
+        }
+        auto reward_row = [&](uint32_t row) {
+            if (RD && row < p.T) {
+                if (base + lane < p.n) rew_row[0] = 1.0f;
+                if (base + 32 + lane < p.n) rew_row[32] = 1.0f;
+                rew_row += p.n;
+            }
+        };
+        // the done bit of slot j's episode that ended with the step of time t_done
+        auto set_done_bit = [&](int j, uint32_t t_done) {
+            if (RD && base + j * 32 + lane < p.n)
+                atomicOr(p.done_bits + (int64_t)(t_done - p.t0) * words + word0 + j, 1u << lane);
+        };
+
         // Slot j has done its last step (its clock reached t_end) and retires. cnt / begin are
         // brought up to date by the restart pass, so an episode that ended on this very step
         // (done_now) is added here; it also hands over the start state of t_end. The final state is
@@ -101,6 +132,7 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
             if (done_now) {
                 cnt[j] += 1u;
                 begin[j] = t_end;
+                set_done_bit(j, t_end - 1u);
             }
             if (p.out_planes) {
                 State a, b;
@@ -148,6 +180,7 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
                 if (!act[j] && (!TAIL || t[j] != t_end)) {
                     cnt[j] += 1u;
                     begin[j] = t[j];
+                    set_done_bit(j, t[j] - 1u);
                     State a, b;
                     unpack_states(zz, a, b);
                     (j ? b : a) = start_state_folded(kr[j], fold16(4u * t[j]));
@@ -157,7 +190,9 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
             }
         };
 
+        uint32_t row = 0;  // trips made so far = the row of the reward plane the next trip writes
         auto trip = [&](auto tail) {
+            if (RD) reward_row(row++);
             State a, b;
             unpack_states(zz, a, b);
             const uint32_t sb0 = deferred_action<POLICY, SHORT>(p, ka[0], own[0], t[0], a);
@@ -173,6 +208,7 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
             // A caller's states may hold any angle: the first trip uses the general scalar step.
             // From then on every stepping slot is a survivor (|theta| <= 0.2095) or a fresh
             // start state (|theta| <= 0.05), which is the packed step's domain.
+            if (RD) reward_row(row++);
             State a, b;
             unpack_states(zz, a, b);
             const uint32_t sb0 = deferred_action<POLICY, SHORT>(p, ka[0], own[0], t[0], a);
@@ -230,17 +266,17 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
     }
 }
 
-template <int POLICY, bool SHORT, bool LIMIT>
+template <int POLICY, bool SHORT, bool LIMIT, bool RD>
 cudaError_t launch_k(RolloutParams &p, int k, cudaStream_t s) {
     p.n_tasks = (p.n + 63) / 64;
     int64_t grid = (p.n_tasks + 7) / 8;
     if (grid > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     switch (k) {
-        case 2: rollout_deferred_kernel<POLICY, 2, SHORT, LIMIT><<<(unsigned)grid, 256, 0, s>>>(p); break;
-        case 3: rollout_deferred_kernel<POLICY, 3, SHORT, LIMIT><<<(unsigned)grid, 256, 0, s>>>(p); break;
-        case 6: rollout_deferred_kernel<POLICY, 6, SHORT, LIMIT><<<(unsigned)grid, 256, 0, s>>>(p); break;
-        case 8: rollout_deferred_kernel<POLICY, 8, SHORT, LIMIT><<<(unsigned)grid, 256, 0, s>>>(p); break;
-        default: rollout_deferred_kernel<POLICY, 4, SHORT, LIMIT><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        case 2: rollout_deferred_kernel<POLICY, 2, SHORT, LIMIT, RD><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        case 3: rollout_deferred_kernel<POLICY, 3, SHORT, LIMIT, RD><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        case 6: rollout_deferred_kernel<POLICY, 6, SHORT, LIMIT, RD><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        case 8: rollout_deferred_kernel<POLICY, 8, SHORT, LIMIT, RD><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        default: rollout_deferred_kernel<POLICY, 4, SHORT, LIMIT, RD><<<(unsigned)grid, 256, 0, s>>>(p); break;
     }
     count_launch();
     return cudaGetLastError();
@@ -248,13 +284,17 @@ cudaError_t launch_k(RolloutParams &p, int k, cudaStream_t s) {
 
 template <int POLICY, bool SHORT>
 cudaError_t launch_limit(RolloutParams &p, int k, cudaStream_t s) {
-    return p.max_steps ? launch_k<POLICY, SHORT, true>(p, k, s) : launch_k<POLICY, SHORT, false>(p, k, s);
+    const bool rd = p.reward_stream != nullptr;  // rollout_deferred_applies: then done_bits too, nothing else
+    if (p.max_steps) return rd ? launch_k<POLICY, SHORT, true, true>(p, k, s) : launch_k<POLICY, SHORT, true, false>(p, k, s);
+    return rd ? launch_k<POLICY, SHORT, false, true>(p, k, s) : launch_k<POLICY, SHORT, false, false>(p, k, s);
 }
 
 }  // namespace
 
 bool rollout_deferred_applies(const RolloutParams &p, int policy, bool streams) {
-    return !streams && !p.action_bits_in && !p.start_in && (policy == 0 || policy == 1 || policy == 6);
+    // per-step outputs: none, or exactly the reward plane + done bitmask
+    const bool outputs_ok = !streams || (p.reward_stream && p.done_bits && !p.action_bits && !p.trajectory);
+    return outputs_ok && !p.action_bits_in && !p.start_in && (policy == 0 || policy == 1 || policy == 6);
 }
 
 cudaError_t launch_rollout_deferred(RolloutParams &p, int policy, cudaStream_t s) {

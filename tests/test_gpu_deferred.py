@@ -129,3 +129,34 @@ def test_returns_against_the_oracle(cp, oracle, kind):
     same = (r["ep_return_sum"].view(np.float32) == o["ep_return_sum"]) & (r["ep_count"] == o["ep_count"])
     err = np.abs(r["final_state"].view(np.float32)[:, same].astype(np.float64) - o["final_state"][:, same])
     assert np.quantile(err.max(axis=0), 0.99) < 1e-3 and res["identical"] > 0.99
+
+
+@pytest.mark.parametrize("kind", [0, 1, 6])
+@pytest.mark.parametrize("n,T,t0,limit", [(1, 3, 0, 0), (33, 40, 7, 0), (4099, 61, 0, 19), (70001, 120, 0, 0),
+                                          (20000, 90, 65530, 0)])
+def test_reward_plane_and_done_bits_with_clocks_per_environment(cp, kind, n, T, t0, limit):
+    """The deferred kernel writes the reward plane row by row and sets done bits by atomic OR from
+    the restart pass: every word must equal the general kernel's, padding bits included."""
+    pol, _ = make_policy(cp, kind, n)
+    words = (n + 31) // 32
+    res = {}
+    for name, shape, k in (("general", GENERAL, 0), ("deferred4", DEFERRED, 4), ("deferred3", DEFERRED, 3)):
+        out = outputs(n)
+        out["reward_stream"] = torch.full((T, n), -7.0, dtype=torch.float32, device="cuda")
+        out["done_bits"] = torch.full((T, words), -1, dtype=torch.int32, device="cuda")  # stale bits everywhere
+        with H.rollout_shape(cp, *shape):
+            cp.cp_tune("rollout_defer", k)
+            try:
+                cp.cp_rollout_ex(n_envs=n, T=T, seed=6, t0=t0, env_offset=9, policy=pol, max_episode_steps=limit, **out)
+            finally:
+                cp.cp_tune("rollout_defer", 0)
+        res[name] = fetch(out)
+    for name in ("deferred4", "deferred3"):
+        for key in res["general"]:
+            assert np.array_equal(res["general"][key], res[name][key]), (key, name)
+    r = res["deferred4"]
+    assert (r["reward_stream"].view(np.float32) == 1.0).all()
+    done = H.unpack_bits(r["done_bits"], n)
+    assert np.array_equal(done.sum(axis=0), r["ep_count"])
+    if n % 32:
+        assert not np.any(r["done_bits"][:, -1] >> (n % 32))
