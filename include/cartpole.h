@@ -335,7 +335,7 @@ int cp_set_allocator(void *(*alloc)(size_t), void (*release)(void *));
  * 5 = two environments per thread with a clock per environment and restarts deferred to every
  * few loop trips (no per-step output streams; hashed actions or a linear policy; otherwise the
  * default); every choice gives the same bits), "rollout_defer" (loop trips between the restart
- * passes of that deferred form: 2, 3, 4, 6 or 8; 0 = default: 4 with hashed actions, else 6),
+ * passes of that deferred form: 2, 3, 4, 6 or 8; 0 = default: 6),
  * "rollout_ctas_per_sm" (0 = default: one 32*ept-environment task per warp and as many
  * CTAs as that takes; k > 0 = persistent grid of k CTAs per SM looping over tasks), "step_block"
  * (32..256, default 64), "step_vec_min_envs" (batches smaller than this use the one-env-per-thread

@@ -51,8 +51,14 @@ __device__ __forceinline__ uint32_t deferred_action(const RolloutParams &p, cons
 // POLICY: 0 hashed actions, 1 shared linear policy, 6 one linear policy per environment.
 // K: trips between restart passes. LIMIT: episodes are cut off after p.max_steps steps.
 // RD: the reward plane and the done bitmask are written (see the comment at reward_row).
+// One CTA per SM is all the launch bounds ask for, which lets the assembler take the registers it
+// wants (77-96 instead of the 58-64 it settles for when left to aim at occupancy): the kernel is
+// bound by the float32 pipe, not by latency, and the extra registers hold the packed constants
+// that are otherwise re-materialised every trip (1,048,576 x 500: 1.032 -> 0.988 ms; with the
+// reward plane and done bits, 4,194,304 x 100: 0.936 -> 0.828 ms; forcing 3 or 4 CTAs per SM
+// measured 1.04 / 1.01 and 0.87 / 0.93 ms).
 template <int POLICY, int K, bool SHORT, bool LIMIT, bool RD>
-__global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_constant__ RolloutParams p) {
+__global__ void __launch_bounds__(256, 1) rollout_deferred_kernel(const __grid_constant__ RolloutParams p) {
     const uint32_t lane = threadIdx.x & 31u;
     const int64_t task = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     unsigned long long tot_ret = 0, tot_cnt = 0;
@@ -109,10 +115,12 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
             }
             __syncwarp();  // orders the clearing stores before any lane's later atomic on the same word
         }
-        auto reward_row = [&](uint32_t row) {
-            if (RD && row < p.T) {
-                if (base + lane < p.n) rew_row[0] = 1.0f;
-                if (base + 32 + lane < p.n) rew_row[32] = 1.0f;
+        const bool has0 = base + lane < p.n, has1 = base + 32 + lane < p.n;
+        // CHECK: the row may lie beyond the last one (only the tail's trips can)
+        auto reward_row = [&](auto check, uint32_t row) {
+            if (RD && (!decltype(check)::value || row < p.T)) {
+                if (has0) rew_row[0] = 1.0f;
+                if (has1) rew_row[32] = 1.0f;
                 rew_row += p.n;
             }
         };
@@ -192,7 +200,7 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
 
         uint32_t row = 0;  // trips made so far = the row of the reward plane the next trip writes
         auto trip = [&](auto tail) {
-            if (RD) reward_row(row++);
+            if (RD) reward_row(tail, row++);
             State a, b;
             unpack_states(zz, a, b);
             const uint32_t sb0 = deferred_action<POLICY, SHORT>(p, ka[0], own[0], t[0], a);
@@ -208,7 +216,7 @@ __global__ void __launch_bounds__(256) rollout_deferred_kernel(const __grid_cons
             // A caller's states may hold any angle: the first trip uses the general scalar step.
             // From then on every stepping slot is a survivor (|theta| <= 0.2095) or a fresh
             // start state (|theta| <= 0.05), which is the packed step's domain.
-            if (RD) reward_row(row++);
+            if (RD) reward_row(std::false_type{}, row++);
             State a, b;
             unpack_states(zz, a, b);
             const uint32_t sb0 = deferred_action<POLICY, SHORT>(p, ka[0], own[0], t[0], a);
@@ -298,9 +306,9 @@ bool rollout_deferred_applies(const RolloutParams &p, int policy, bool streams) 
 }
 
 cudaError_t launch_rollout_deferred(RolloutParams &p, int policy, cudaStream_t s) {
-    // measured on 1,048,576 x 500: hashed actions (22-step episodes) 1.022 / 1.034 / 1.071 ms at
-    // K = 4 / 6 / 8, the linear policy (longer episodes) 0.952 / 0.934 / 1.008 ms
-    const int k = g_tuning.rollout_defer > 0 ? g_tuning.rollout_defer : (policy == 0 ? 4 : 6);
+    // measured on 1,048,576 x 500 at K = 3 / 4 / 6 / 8: hashed actions (22-step episodes) 0.996 /
+    // 0.987 / 0.965 / 0.987 ms, the linear policy (80-step episodes) 0.945 / 0.924 / 0.907 / 0.908 ms
+    const int k = g_tuning.rollout_defer > 0 ? g_tuning.rollout_defer : 6;
     // the action hash folds the time's upper half into the lower one: nothing to do below 2^16
     const bool short_times = (uint64_t)p.t0 + p.T <= 65536u;
     switch (policy) {

@@ -67,7 +67,7 @@ constexpr int kMaxWarpsPerCta = 8;  // __launch_bounds__(256)
 // LIMIT: episodes are cut off after p.max_steps steps.
 // CONTRACT: the contracted arithmetic of euler_step_contracted instead of the canonical order.
 template <int POLICY, int SHAPE, int STREAMS, bool LIMIT, bool CONTRACT>
-__global__ void __launch_bounds__(256) rollout_kernel(const __grid_constant__ RolloutParams p) {
+__global__ void __launch_bounds__(256, 1) rollout_kernel(const __grid_constant__ RolloutParams p) {
     constexpr int EPT = SHAPE == 2 ? 2 : 1;
     constexpr bool COOP = SHAPE == 1 || SHAPE == 2;
     constexpr bool AHEAD = SHAPE == 3;

@@ -25,7 +25,7 @@ __device__ __forceinline__ uint32_t hashed_signbit(const StepParams &p, uint32_t
 // lets the next launch begin its own preamble. Launched without that attribute the two
 // grid-dependency instructions do nothing.
 template <bool VEC>
-__global__ void __launch_bounds__(256) step_kernel(const __grid_constant__ StepParams p) {
+__global__ void __launch_bounds__(256, 1) step_kernel(const __grid_constant__ StepParams p) {
     const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const bool has_action = p.action != nullptr;
     if (VEC) {
