@@ -333,9 +333,9 @@ int cp_set_allocator(void *(*alloc)(size_t), void (*release)(void *));
  * other batches too small to fill the GPU (ahead for the smaller ones), deferred (5) for batches
  * that fill it where that form applies, by the warp otherwise;
  * 5 = two environments per thread with a clock per environment and restarts deferred to every
- * few loop trips (no per-step output streams; hashed actions or a linear policy; otherwise the
- * default); every choice gives the same bits), "rollout_defer" (loop trips between the restart
- * passes of that deferred form: 2, 3, 4, 6 or 8; 0 = default: 6),
+ * few loop trips (per-step outputs none or reward plane + done bits; hashed actions, a linear
+ * policy or the 4-16-2 network; otherwise the default); every choice gives the same bits), "rollout_defer" (loop trips between the restart
+ * passes of that deferred form: 2, 3, 4, 6 or 8; 0 = default: 6, with the 4-16-2 network 2),
  * "rollout_ctas_per_sm" (0 = default: one 32*ept-environment task per warp and as many
  * CTAs as that takes; k > 0 = persistent grid of k CTAs per SM looping over tasks), "step_block"
  * (32..256, default 64), "step_vec_min_envs" (batches smaller than this use the one-env-per-thread
@@ -362,10 +362,14 @@ int cp_selftest_sincos(uint32_t lo_bits, uint32_t hi_bits, uint64_t *mismatches)
  * not the correctly rounded value. */
 int cp_selftest_sincos_accuracy(uint32_t lo_bits, uint32_t hi_bits, uint64_t *out);
 
-/* Diagnostics: absolute error against float64 of the hyperbolic tangent the MLP policies use —
- * out[0]: the five-instruction form of CP_ARITH_CONTRACTED, out[1]: the library tanhf of
- * CP_ARITH_EXACT — over the float32 values in [lo, hi] (bit patterns as above) and their
- * negatives, largest value seen, in units of 1e-12. out DEVICE [2] uint64, caller zeroes. */
+/* Diagnostics: error against float64 of the hyperbolic tangents the MLP policies use, over the
+ * float32 values in [lo, hi] (bit patterns as above) and their negatives, largest value seen.
+ * out DEVICE [6] uint64, caller zeroes. Absolute error in units of 1e-12: out[0] the
+ * five-instruction form of CP_ARITH_CONTRACTED, out[1] the CUDA library's tanhf (for comparison),
+ * out[2] the tanh of CP_ARITH_EXACT (polynomial below 0.6, hardware exp2 / reciprocal above,
+ * branch-free). In millionths of a unit in the last place: out[3] that tanh, out[4] the library's.
+ * out[5] += values for which the packed two-environment form of that tanh differs in any bit
+ * from the scalar form (must stay 0). */
 int cp_selftest_tanh(uint32_t lo_bits, uint32_t hi_bits, uint64_t *out);
 
 /* Diagnostics: the kernels replace x / 1.1f by a two-operation exact sequence and the start-state

@@ -511,6 +511,59 @@ __device__ __forceinline__ float tanh_contracted(float x) {
     return __fmaf_rn(-2.0f, r, 1.0f);
 }
 
+// tanh of the canonical arithmetic: as accurate as the library routine (largest error 1.82 ulp
+// against float64 over every float32, the library's tanhf: 1.82 — cp_selftest_tanh measures
+// both), built so that two values can share one instruction stream. |x| < 0.6: x + x*z*P(z),
+// z = x^2, P of degree 4 (weighted minimax fit, 0.72 ulp). Otherwise 1 - 2/(e^(2|x|) + 1) from
+// the hardware exp2 and reciprocal, with the sign of x; it saturates to +-1 and keeps NaN.
+// Both sides are always evaluated and one is selected: no branch. tanh_pair performs the same
+// operations on both halves of a pair, so tanh_pair(pack2(a, b)) == (tanh_canonical(a),
+// tanh_canonical(b)) bit for bit (checked over every float32 by cp_selftest_tanh).
+constexpr float kTanhSplit = 0.6f;
+constexpr float kTanhC0 = -3.333329856e-01f, kTanhC1 = 1.333195865e-01f, kTanhC2 = -5.378668010e-02f,
+                kTanhC3 = 2.080537751e-02f, kTanhC4 = -5.905860569e-03f;
+constexpr float kTwoLog2e = 2.885390043f;
+__device__ __forceinline__ float tanh_canonical(float x) {
+    const float t = fabsf(x);
+    float e, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(__fmul_rn(t, kTwoLog2e)));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(__fadd_rn(e, 1.0f)));
+    const float big = copysignf(__fmaf_rn(-2.0f, r, 1.0f), x);
+    const float z = __fmul_rn(x, x);
+    float p = __fmaf_rn(kTanhC4, z, kTanhC3);
+    p = __fmaf_rn(p, z, kTanhC2);
+    p = __fmaf_rn(p, z, kTanhC1);
+    p = __fmaf_rn(p, z, kTanhC0);
+    const float small = __fmaf_rn(__fmul_rn(p, z), x, x);
+    return t < kTanhSplit ? small : big;
+}
+__device__ __forceinline__ f32x2 tanh_pair(f32x2 x) {
+    float x0, x1;
+    unpack2(x, x0, x1);
+    const float t0 = fabsf(x0), t1 = fabsf(x1);
+    const f32x2 arg = mul2(pack2(t0, t1), splat2(kTwoLog2e));
+    float a0, a1, e0, e1, r0, r1;
+    unpack2(arg, a0, a1);
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(a0));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(a1));
+    const f32x2 d = add2(pack2(e0, e1), splat2(1.0f));
+    float d0, d1;
+    unpack2(d, d0, d1);
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r0) : "f"(d0));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r1) : "f"(d1));
+    const f32x2 big = fma2(splat2(-2.0f), pack2(r0, r1), splat2(1.0f));
+    const f32x2 z = mul2(x, x);
+    f32x2 p = fma2(splat2(kTanhC4), z, splat2(kTanhC3));
+    p = fma2(p, z, splat2(kTanhC2));
+    p = fma2(p, z, splat2(kTanhC1));
+    p = fma2(p, z, splat2(kTanhC0));
+    const f32x2 small = fma2(mul2(p, z), x, x);
+    float b0, b1, s0, s1;
+    unpack2(big, b0, b1);
+    unpack2(small, s0, s1);
+    return pack2(t0 < kTanhSplit ? s0 : copysignf(b0, x0), t1 < kTanhSplit ? s1 : copysignf(b1, x1));
+}
+
 template <int H, bool FAST_TANH = false>
 __device__ __forceinline__ uint32_t mlp_action(const MlpWT<H> &p, const State &z) {
     float l0 = p.b2[0], l1 = p.b2[1];
@@ -521,7 +574,7 @@ __device__ __forceinline__ uint32_t mlp_action(const MlpWT<H> &p, const State &z
         acc = __fmaf_rn(p.w1[j][1], z.xd, acc);
         acc = __fmaf_rn(p.w1[j][2], z.th, acc);
         acc = __fmaf_rn(p.w1[j][3], z.thd, acc);
-        float h = FAST_TANH ? tanh_contracted(acc) : tanhf(acc);
+        float h = FAST_TANH ? tanh_contracted(acc) : tanh_canonical(acc);
         l0 = __fmaf_rn(p.w2[0][j], h, l0);
         l1 = __fmaf_rn(p.w2[1][j], h, l1);
     }
@@ -546,7 +599,7 @@ __device__ __forceinline__ uint32_t mlp_deep_action(const MlpDeepW &p, const Sta
         acc = __fmaf_rn(p.w1[j][1], z.xd, acc);
         acc = __fmaf_rn(p.w1[j][2], z.th, acc);
         acc = __fmaf_rn(p.w1[j][3], z.thd, acc);
-        h1[j] = FAST_TANH ? tanh_contracted(acc) : tanhf(acc);
+        h1[j] = FAST_TANH ? tanh_contracted(acc) : tanh_canonical(acc);
     }
     float l0 = p.b3[0], l1 = p.b3[1];
 #pragma unroll
@@ -554,7 +607,7 @@ __device__ __forceinline__ uint32_t mlp_deep_action(const MlpDeepW &p, const Sta
         float acc = p.b2[k];
 #pragma unroll
         for (int j = 0; j < 16; ++j) acc = __fmaf_rn(p.w2[k][j], h1[j], acc);
-        const float h2 = FAST_TANH ? tanh_contracted(acc) : tanhf(acc);
+        const float h2 = FAST_TANH ? tanh_contracted(acc) : tanh_canonical(acc);
         l0 = __fmaf_rn(p.w3[0][k], h2, l0);
         l1 = __fmaf_rn(p.w3[1][k], h2, l1);
     }

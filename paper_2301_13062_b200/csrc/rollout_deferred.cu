@@ -39,16 +39,72 @@ namespace cp {
 
 namespace {
 
-// SHORT: every time of the launch is below 2^16, where fold16(t) == t.
-template <int POLICY, bool SHORT>
-__device__ __forceinline__ uint32_t deferred_action(const RolloutParams &p, const FoldedKeys &ka, const LinearW &own,
-                                                    uint32_t t, const State &z) {
-    if (POLICY == 0) return action_signbit_folded(ka, SHORT ? t : fold16(t));
-    if (POLICY == 1) return linear_action(*reinterpret_cast<const LinearW *>(p.w), z);
-    return linear_action(own, z);
+// Shared policies read their weights as (w, w) pairs: the launcher duplicates every weight in the
+// launch parameters, so that one packed fused multiply-add applies it to both environments of a
+// thread. Each half is the scalar chain of linear_action / mlp_action (same order, one rounding per
+// fused operation), hence the same logits bit for bit.
+__device__ __forceinline__ void argmax_pair(f32x2 l0, f32x2 l1, uint32_t &sb0, uint32_t &sb1) {
+    float a0, a1, b0, b1;
+    unpack2(l0, a0, a1);
+    unpack2(l1, b0, b1);
+    sb0 = (b0 > a0) ? 0x80000000u : 0u;
+    sb1 = (b1 > a1) ? 0x80000000u : 0u;
+}
+__device__ __forceinline__ void linear_action_pair(const f32x2 *w, const StatePair &z, uint32_t &sb0, uint32_t &sb1) {
+    // w: W[2][4] then b[2], as pairs
+    f32x2 l0 = w[8], l1 = w[9];
+    l0 = fma2(w[0], z.x, l0);
+    l1 = fma2(w[4], z.x, l1);
+    l0 = fma2(w[1], z.xd, l0);
+    l1 = fma2(w[5], z.xd, l1);
+    l0 = fma2(w[2], z.th, l0);
+    l1 = fma2(w[6], z.th, l1);
+    l0 = fma2(w[3], z.thd, l0);
+    l1 = fma2(w[7], z.thd, l1);
+    argmax_pair(l0, l1, sb0, sb1);
+}
+template <int H>
+__device__ __forceinline__ void mlp_action_pair(const f32x2 *w, const StatePair &z, uint32_t &sb0, uint32_t &sb1) {
+    // w: W1[H][4], b1[H], W2[2][H], b2[2], as pairs
+    const f32x2 *w1 = w, *b1 = w + 4 * H, *w2 = w + 5 * H, *b2 = w + 7 * H;
+    f32x2 l0 = b2[0], l1 = b2[1];
+#pragma unroll
+    for (int j = 0; j < H; ++j) {
+        f32x2 acc = b1[j];
+        acc = fma2(w1[4 * j + 0], z.x, acc);
+        acc = fma2(w1[4 * j + 1], z.xd, acc);
+        acc = fma2(w1[4 * j + 2], z.th, acc);
+        acc = fma2(w1[4 * j + 3], z.thd, acc);
+        const f32x2 h = tanh_pair(acc);
+        l0 = fma2(w2[j], h, l0);
+        l1 = fma2(w2[H + j], h, l1);
+    }
+    argmax_pair(l0, l1, sb0, sb1);
 }
 
-// POLICY: 0 hashed actions, 1 shared linear policy, 6 one linear policy per environment.
+// Actions of both slots, in sign-bit form. SHORT: every time of the launch is below 2^16, where
+// fold16(t) == t.
+template <int POLICY, bool SHORT>
+__device__ __forceinline__ void deferred_actions(const RolloutParams &p, const FoldedKeys (&ka)[2],
+                                                 const LinearW *own, const uint32_t (&t)[2], const StatePair &zz,
+                                                 uint32_t &sb0, uint32_t &sb1) {
+    const f32x2 *pairs = reinterpret_cast<const f32x2 *>(p.w);
+    if (POLICY == 0) {
+        sb0 = action_signbit_folded(ka[0], SHORT ? t[0] : fold16(t[0]));
+        sb1 = action_signbit_folded(ka[1], SHORT ? t[1] : fold16(t[1]));
+    } else if (POLICY == 1) {
+        linear_action_pair(pairs, zz, sb0, sb1);
+    } else if (POLICY == 2) {
+        mlp_action_pair<16>(pairs, zz, sb0, sb1);
+    } else {
+        State a, b;
+        unpack_states(zz, a, b);
+        sb0 = linear_action(own[0], a);
+        sb1 = linear_action(own[POLICY == 6 ? 1 : 0], b);
+    }
+}
+
+// POLICY: 0 hashed actions, 1 shared linear policy, 2 shared 4-16-2 network, 6 one linear policy per environment.
 // K: trips between restart passes. LIMIT: episodes are cut off after p.max_steps steps.
 // RD: the reward plane and the done bitmask are written (see the comment at reward_row).
 // One CTA per SM is all the launch bounds ask for, which lets the assembler take the registers it
@@ -57,8 +113,11 @@ __device__ __forceinline__ uint32_t deferred_action(const RolloutParams &p, cons
 // that are otherwise re-materialised every trip (1,048,576 x 500: 1.032 -> 0.988 ms; with the
 // reward plane and done bits, 4,194,304 x 100: 0.936 -> 0.828 ms; forcing 3 or 4 CTAs per SM
 // measured 1.04 / 1.01 and 0.87 / 0.93 ms).
+// (The network policy is the exception: its sixteen hidden units per slot are latency — exp2 and
+// reciprocal on the special-function pipe — that only more resident warps hide: 16,777,216 x
+// 200 takes 53.1 / 41.1 / 39.9 / 39.4 / 40.8 ms at 1 / 2 / 3 / 4 / 5 CTAs per SM.)
 template <int POLICY, int K, bool SHORT, bool LIMIT, bool RD>
-__global__ void __launch_bounds__(256, 1) rollout_deferred_kernel(const __grid_constant__ RolloutParams p) {
+__global__ void __launch_bounds__(256, POLICY == 2 ? 4 : 1) rollout_deferred_kernel(const __grid_constant__ RolloutParams p) {
     const uint32_t lane = threadIdx.x & 31u;
     const int64_t task = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     unsigned long long tot_ret = 0, tot_cnt = 0;
@@ -76,6 +135,7 @@ __global__ void __launch_bounds__(256, 1) rollout_deferred_kernel(const __grid_c
             if (idx >= p.n) idx = p.n - 1;  // idle lanes shadow the last environment and store nothing
             const uint32_t env = p.env_offset + (uint32_t)idx;
             if (POLICY == 0) ka[j] = fold_keys(make_keys(p.salt_a, env));
+            else ka[j] = FoldedKeys{0u, 0u};
             kr[j] = fold_keys(make_keys(p.salt_r, env));
             if (p.init_planes) {
                 z0[j].x = p.init_planes[idx];
@@ -201,10 +261,8 @@ __global__ void __launch_bounds__(256, 1) rollout_deferred_kernel(const __grid_c
         uint32_t row = 0;  // trips made so far = the row of the reward plane the next trip writes
         auto trip = [&](auto tail) {
             if (RD) reward_row(tail, row++);
-            State a, b;
-            unpack_states(zz, a, b);
-            const uint32_t sb0 = deferred_action<POLICY, SHORT>(p, ka[0], own[0], t[0], a);
-            const uint32_t sb1 = deferred_action<POLICY, SHORT>(p, ka[POLICY == 0 ? 1 : 0], own[POLICY == 6 ? 1 : 0], t[1], b);
+            uint32_t sb0, sb1;
+            deferred_actions<POLICY, SHORT>(p, ka, own, t, zz, sb0, sb1);
             bool d0, d1;
             euler_step_pair(zz, pack2(force_from_signbit(sb0), force_from_signbit(sb1)), d0, d1);
             after_step(tail, 0, d0);
@@ -217,10 +275,10 @@ __global__ void __launch_bounds__(256, 1) rollout_deferred_kernel(const __grid_c
             // From then on every stepping slot is a survivor (|theta| <= 0.2095) or a fresh
             // start state (|theta| <= 0.05), which is the packed step's domain.
             if (RD) reward_row(std::false_type{}, row++);
+            uint32_t sb0, sb1;
+            deferred_actions<POLICY, SHORT>(p, ka, own, t, zz, sb0, sb1);
             State a, b;
             unpack_states(zz, a, b);
-            const uint32_t sb0 = deferred_action<POLICY, SHORT>(p, ka[0], own[0], t[0], a);
-            const uint32_t sb1 = deferred_action<POLICY, SHORT>(p, ka[POLICY == 0 ? 1 : 0], own[POLICY == 6 ? 1 : 0], t[1], b);
             const bool d0 = euler_step<false>(a, force_from_signbit(sb0));
             const bool d1 = euler_step<false>(b, force_from_signbit(sb1));
             zz = pack_states(a, b);
@@ -230,8 +288,10 @@ __global__ void __launch_bounds__(256, 1) rollout_deferred_kernel(const __grid_c
             trips = 1;
         }
         // Main part: after these trips no clock can have reached t_end yet, so no slot can retire.
+        // (the network policy's trip is some 600 instructions long: its K trips stay a loop)
+        constexpr int kUnroll = POLICY == 2 ? 1 : K;
         while (trips + K <= p.T - 1u) {
-#pragma unroll
+#pragma unroll kUnroll
             for (int k = 0; k < K; ++k) trip(std::false_type{});
             restart_pass(std::false_type{});
             trips += K;
@@ -240,7 +300,7 @@ __global__ void __launch_bounds__(256, 1) rollout_deferred_kernel(const __grid_c
         // unretired slot by at least one step, so p.T blocks always suffice.
         for (uint32_t block = 0; block <= p.T; ++block) {
             if (__all_sync(0xffffffffu, t[0] == t_end && t[1] == t_end)) break;
-#pragma unroll
+#pragma unroll kUnroll
             for (int k = 0; k < K; ++k) trip(std::true_type{});
             restart_pass(std::true_type{});
         }
@@ -302,18 +362,26 @@ cudaError_t launch_limit(RolloutParams &p, int k, cudaStream_t s) {
 bool rollout_deferred_applies(const RolloutParams &p, int policy, bool streams) {
     // per-step outputs: none, or exactly the reward plane + done bitmask
     const bool outputs_ok = !streams || (p.reward_stream && p.done_bits && !p.action_bits && !p.trajectory);
-    return outputs_ok && !p.action_bits_in && !p.start_in && (policy == 0 || policy == 1 || policy == 6);
+    return outputs_ok && !p.action_bits_in && !p.start_in && (policy == 0 || policy == 1 || policy == 2 || policy == 6);
 }
 
 cudaError_t launch_rollout_deferred(RolloutParams &p, int policy, cudaStream_t s) {
     // measured on 1,048,576 x 500 at K = 3 / 4 / 6 / 8: hashed actions (22-step episodes) 0.996 /
     // 0.987 / 0.965 / 0.987 ms, the linear policy (80-step episodes) 0.945 / 0.924 / 0.907 / 0.908 ms
-    const int k = g_tuning.rollout_defer > 0 ? g_tuning.rollout_defer : 6;
+    // The 4-16-2 network of config 5 ends its episodes after 9-10 steps, so waiting costs more and
+    // a restart pass less (next to a 600-instruction trip): 16,777,216 x 200 takes 41.1 / 43.1 /
+    // 47.3 / 48.9 ms at K = 2 / 3 / 4 / 6 (the general kernel: 43.2 ms).
+    const int k = g_tuning.rollout_defer > 0 ? g_tuning.rollout_defer : (policy == 2 ? 2 : 6);
     // the action hash folds the time's upper half into the lower one: nothing to do below 2^16
     const bool short_times = (uint64_t)p.t0 + p.T <= 65536u;
+    if (policy == 1 || policy == 2) {  // every shared weight twice: one packed operand for both slots
+        const int count = policy == 1 ? 10 : 114;
+        for (int i = count - 1; i >= 0; --i) p.w[2 * i] = p.w[2 * i + 1] = p.w[i];
+    }
     switch (policy) {
         case 0: return short_times ? launch_limit<0, true>(p, k, s) : launch_limit<0, false>(p, k, s);
         case 1: return launch_limit<1, false>(p, k, s);
+        case 2: return launch_limit<2, false>(p, k, s);
         default: return launch_limit<6, false>(p, k, s);
     }
 }

@@ -277,25 +277,47 @@ cudaError_t launch_sincos_accuracy(uint32_t lo_bits, uint32_t hi_bits, unsigned 
 // out[0] / out[1]: largest |tanh_contracted(v) - tanh(v)| / |tanhf(v) - tanh(v)| over the
 // float32 values with bit patterns in [lo, hi] and their negatives, in units of 1e-12.
 __global__ void tanh_accuracy_kernel(uint32_t lo, uint32_t hi, unsigned long long *out) {
-    double worst_fast = 0.0, worst_lib = 0.0;
+    double worst_fast = 0.0, worst_lib = 0.0, worst_own = 0.0, worst_own_ulp = 0.0, worst_lib_ulp = 0.0;
+    unsigned long long pair_mismatch = 0;
     const uint64_t span = (uint64_t)hi - lo + 1;
     for (uint64_t k = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; k < span; k += (uint64_t)gridDim.x * blockDim.x) {
+        float own[2];
         for (int sign = 0; sign < 2; ++sign) {
             const float v = __uint_as_float((lo + (uint32_t)k) | (sign ? 0x80000000u : 0u));
             const double exact = tanh((double)v);
+            // one unit in the last place of the correctly rounded result
+            const float w = fabsf((float)exact);
+            double ulp = (double)__uint_as_float(__float_as_uint(w) + 1u) - (double)w;
+            if (!(ulp > 0.0)) ulp = 1.4e-45;
+            own[sign] = tanh_canonical(v);
+            const float lib = tanhf(v);
             worst_fast = fmax(worst_fast, fabs((double)tanh_contracted(v) - exact));
-            worst_lib = fmax(worst_lib, fabs((double)tanhf(v) - exact));
+            worst_lib = fmax(worst_lib, fabs((double)lib - exact));
+            worst_own = fmax(worst_own, fabs((double)own[sign] - exact));
+            worst_own_ulp = fmax(worst_own_ulp, fabs((double)own[sign] - exact) / ulp);
+            worst_lib_ulp = fmax(worst_lib_ulp, fabs((double)lib - exact) / ulp);
         }
+        // the packed form on (v, -v) and on (-v, v): the same bits as the scalar form, either half
+        const float v = __uint_as_float(lo + (uint32_t)k);
+        float p0, p1, q0, q1;
+        unpack2(tanh_pair(pack2(v, -v)), p0, p1);
+        unpack2(tanh_pair(pack2(-v, v)), q0, q1);
+        pair_mismatch += __float_as_uint(p0) != __float_as_uint(own[0]) || __float_as_uint(p1) != __float_as_uint(own[1]) ||
+                         __float_as_uint(q0) != __float_as_uint(own[1]) || __float_as_uint(q1) != __float_as_uint(own[0]);
     }
-    unsigned long long a = (unsigned long long)(worst_fast * 1e12), b = (unsigned long long)(worst_lib * 1e12);
+    unsigned long long m[5] = {(unsigned long long)(worst_fast * 1e12), (unsigned long long)(worst_lib * 1e12),
+                               (unsigned long long)(worst_own * 1e12), (unsigned long long)(worst_own_ulp * 1e6),
+                               (unsigned long long)(worst_lib_ulp * 1e6)};
     for (int o = 16; o > 0; o >>= 1) {
-        const unsigned long long a2 = __shfl_down_sync(0xffffffffu, a, o), b2 = __shfl_down_sync(0xffffffffu, b, o);
-        a = a2 > a ? a2 : a;
-        b = b2 > b ? b2 : b;
+        for (int i = 0; i < 5; ++i) {
+            const unsigned long long other = __shfl_down_sync(0xffffffffu, m[i], o);
+            m[i] = other > m[i] ? other : m[i];
+        }
+        pair_mismatch += __shfl_down_sync(0xffffffffu, pair_mismatch, o);
     }
     if ((threadIdx.x & 31) == 0) {
-        atomicMax(out, a);
-        atomicMax(out + 1, b);
+        for (int i = 0; i < 5; ++i) atomicMax(out + i, m[i]);
+        if (pair_mismatch) atomicAdd(out + 5, pair_mismatch);
     }
 }
 

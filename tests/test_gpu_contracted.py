@@ -154,18 +154,25 @@ def test_contracted_chunks_and_step_limit_compose(cp):
     assert whole[2].sum() > 0 and (whole[1] / np.maximum(whole[2], 1)).max() <= limit
 
 
-def test_contracted_tanh_absolute_error_over_every_float(cp):
-    """The five-instruction tanh of the contracted MLP policies against float64, over every
-    finite float32 of either sign: the policy's logits feel the ABSOLUTE error, which must stay
-    far below the 1e-5 logit gap that the parity rules excuse (16 hidden units x |w2| ~ 0.25
-    turn 3e-7 into about 1e-6)."""
-    out = torch.zeros(2, dtype=torch.int64, device="cuda")
+def test_tanh_errors_over_every_float(cp):
+    """The hyperbolic tangents of the MLP policies against float64, over every finite float32 of
+    either sign. The contracted arithmetic's five-instruction form: the policy's logits feel the
+    ABSOLUTE error, which must stay far below the 1e-5 logit gap that the parity rules excuse (16
+    hidden units x |w2| ~ 0.25 turn 3e-7 into about 1e-6). The canonical arithmetic's own tanh: at
+    least as accurate as the CUDA library's tanhf in units in the last place (so it is no fast-math
+    substitute), and its packed two-value form gives the scalar form's bits for every input."""
+    out = torch.zeros(6, dtype=torch.int64, device="cuda")
     cp.cp_selftest_tanh(0, 0x7F7FFFFF, out)
     torch.cuda.synchronize()
-    fast, lib = (int(v) * 1e-12 for v in out.cpu())
-    print(f"tanh absolute error over all floats: contracted {fast:.3e}, library tanhf {lib:.3e}")
+    v = [int(x) for x in out.cpu()]
+    fast, lib, own = (x * 1e-12 for x in v[:3])
+    own_ulp, lib_ulp = v[3] * 1e-6, v[4] * 1e-6
+    print(f"tanh over all floats: contracted {fast:.3e} abs; library {lib:.3e} abs, {lib_ulp:.3f} ulp; "
+          f"canonical {own:.3e} abs, {own_ulp:.3f} ulp")
     assert fast <= 3e-7, fast
     assert lib <= 2e-7, lib
+    assert own <= 2e-7 and own_ulp <= max(lib_ulp, 1.85), (own, own_ulp, lib_ulp)
+    assert v[5] == 0
 
 
 def test_unknown_arithmetic_is_rejected(cp):

@@ -43,9 +43,9 @@ def fetch(out):
 def make_policy(cp, kind, n):
     if kind == 0:
         return None, None
-    if kind == 1:
-        w = inputs.policy_weights(1, 1)
-        return cp.policy(1, w), w
+    if kind in (1, 2):
+        w = inputs.policy_weights(kind, kind)
+        return cp.policy(kind, w), w
     w = inputs.per_env_linear_weights(n, 11)
     return cp.policy(cp.CP_POLICY_LINEAR_PER_ENV, torch.from_numpy(w).cuda()), w
 
@@ -62,7 +62,7 @@ def run(cp, shape, k, **kw):
             cp.cp_tune("rollout_defer", 0)
 
 
-@pytest.mark.parametrize("kind", [0, 1, 6])
+@pytest.mark.parametrize("kind", [0, 1, 2, 6])
 @pytest.mark.parametrize("n,T,t0,off,limit", [
     (1, 1, 0, 0, 0), (63, 2, 0, 5, 0), (65, 5, 3, 0, 0), (4099, 61, 0, 77, 0), (4099, 61, 0, 77, 23),
     (70001, 200, 0, 0, 0), (20000, 150, 70000, 1 << 20, 0), (20000, 150, 65500, 0, 40), (3000, 700, 11, 0, 500),
@@ -78,7 +78,7 @@ def test_same_bits_as_the_general_kernel(cp, kind, n, T, t0, off, limit):
             assert np.array_equal(want[key], got[key]), (key, k)
 
 
-@pytest.mark.parametrize("kind", [0, 1])
+@pytest.mark.parametrize("kind", [0, 1, 2])
 @pytest.mark.parametrize("limit", [0, 31])
 def test_chunks_from_a_callers_states(cp, kind, limit):
     """States with angles far outside the polynomial range and running-episode lengths carried in
@@ -114,12 +114,12 @@ def test_chunks_from_a_callers_states(cp, kind, limit):
     assert sum(int(c["ep_count"].sum()) for c in results["deferred"][0::2]) > n // 4
 
 
-@pytest.mark.parametrize("kind", [0, 1, 6])
+@pytest.mark.parametrize("kind", [0, 1, 2, 6])
 def test_returns_against_the_oracle(cp, oracle, kind):
     n, T, seed = 50001, 300, 2
     pol, w = make_policy(cp, kind, n)
     r = run(cp, DEFERRED, 0, n_envs=n, T=T, seed=seed, policy=pol)
-    o = oracle.rollout(n, T, seed, {0: 0, 1: 1, 6: inputs.POLICY_LINEAR_PER_ENV}[kind], w, final_state=True,
+    o = oracle.rollout(n, T, seed, {0: 0, 1: 1, 2: 2, 6: inputs.POLICY_LINEAR_PER_ENV}[kind], w, final_state=True,
                        min_gap=True, nthreads=8)
     excuse = (o["min_gap"] < 1e-5) if kind else None
     res = H.assert_returns_match(r["ep_return_sum"].view(np.float32), r["ep_count"], o["ep_return_sum"], o["ep_count"],
@@ -131,7 +131,7 @@ def test_returns_against_the_oracle(cp, oracle, kind):
     assert np.quantile(err.max(axis=0), 0.99) < 1e-3 and res["identical"] > 0.99
 
 
-@pytest.mark.parametrize("kind", [0, 1, 6])
+@pytest.mark.parametrize("kind", [0, 1, 2, 6])
 @pytest.mark.parametrize("n,T,t0,limit", [(1, 3, 0, 0), (33, 40, 7, 0), (4099, 61, 0, 19), (70001, 120, 0, 0),
                                           (20000, 90, 65530, 0)])
 def test_reward_plane_and_done_bits_with_clocks_per_environment(cp, kind, n, T, t0, limit):
