@@ -393,8 +393,9 @@ int cp_selftest_tame_div(uint32_t den_step, uint64_t *out);
  * kernels step both with sm_100a's packed float32 instructions (one instruction, two
  * independent roundings). This steps `count` pseudo-random pairs of states (|theta| <= 0.22, the
  * other components across and beyond the live range; drawn from `seed`) both ways and compares
- * all eight new components and both termination flags bit for bit. out DEVICE [2] uint64, caller
- * zeroes: out[0] += pairs that differ (must stay 0), out[1] += pairs tested. */
+ * all eight new components and both termination flags bit for bit. out DEVICE [3] uint64, caller
+ * zeroes: out[0] += pairs that differ (must stay 0), out[1] += pairs tested, out[2] += pairs for
+ * which the packed and scalar steps of CP_ARITH_CONTRACTED differ (must stay 0). */
 int cp_selftest_pair(uint64_t count, uint32_t seed, uint64_t *out);
 
 /* Calibration of the roofline denominators (a measurement aid; the paper has no counterpart):

@@ -469,6 +469,43 @@ __device__ __forceinline__ bool euler_step_contracted(State &z, float force) {
     return (fabsf(nx) > kXT) | (fabsf(nth) > kTT);
 }
 
+// euler_step_contracted<true> for two environments at once: the same fused operations on each
+// half, hence the bits of the scalar form. temp is carried with its sign flipped (the constant
+// it is multiplied by is negated, which is exact), so that -c*temp and xacc need no negation;
+// -xacc then meets -tau in the velocity update.
+__device__ __forceinline__ void euler_step_contracted_pair(StatePair &z, f32x2 force, bool &done0, bool &done1) {
+    const f32x2 zz = mul2(z.th, z.th);
+    const f32x2 sp = fma2(splat2(8.319973014e-03f), zz, splat2(-1.666664630e-01f));
+    const f32x2 s = fma2(mul2(sp, zz), z.th, z.th);
+    f32x2 cq = fma2(splat2(-1.387019176e-03f), zz, splat2(4.166663438e-02f));
+    cq = fma2(cq, zz, splat2(-0.5f));
+    const f32x2 c = fma2(cq, zz, splat2(1.0f));
+    const f32x2 t1 = mul2(mul2(z.thd, z.thd), splat2(kPML));
+    const f32x2 ntemp = mul2(fma2(t1, s, force), splat2(-kRcpMTot));
+    const f32x2 num = fma2(c, ntemp, mul2(splat2(kG), s));
+    const f32x2 den = fma2(mul2(c, c), splat2(kDenK), splat2(kDenC));
+    float d0, d1, r0, r1;
+    unpack2(den, d0, d1);
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r0) : "f"(d0));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r1) : "f"(d1));
+    const f32x2 thacc = mul2(num, pack2(r0, r1));
+    const f32x2 nxacc = fma2(mul2(thacc, c), splat2(-kXaccK), ntemp);
+    const f32x2 tau = splat2(kTau);
+    const f32x2 nx = fma2(tau, z.xd, z.x);
+    const f32x2 nxd = fma2(splat2(-kTau), nxacc, z.xd);
+    const f32x2 nth = fma2(tau, z.thd, z.th);
+    const f32x2 nthd = fma2(tau, thacc, z.thd);
+    z.x = nx;
+    z.xd = nxd;
+    z.th = nth;
+    z.thd = nthd;
+    float x0, x1, a0, a1;
+    unpack2(nx, x0, x1);
+    unpack2(nth, a0, a1);
+    done0 = (fabsf(x0) > kXT) | (fabsf(a0) > kTT);
+    done1 = (fabsf(x1) > kXT) | (fabsf(a1) > kTT);
+}
+
 // ---- policies (observation = state before the step) ----
 struct LinearW {
     float w[2][4];
@@ -562,6 +599,21 @@ __device__ __forceinline__ f32x2 tanh_pair(f32x2 x) {
     unpack2(big, b0, b1);
     unpack2(small, s0, s1);
     return pack2(t0 < kTanhSplit ? s0 : copysignf(b0, x0), t1 < kTanhSplit ? s1 : copysignf(b1, x1));
+}
+
+// tanh_contracted on both halves of a pair (same operations, same bits).
+__device__ __forceinline__ f32x2 tanh_contracted_pair(f32x2 x) {
+    const f32x2 arg = mul2(x, splat2(kTwoLog2e));
+    float a0, a1, t0, t1, r0, r1;
+    unpack2(arg, a0, a1);
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(t0) : "f"(a0));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(t1) : "f"(a1));
+    const f32x2 d = add2(pack2(t0, t1), splat2(1.0f));
+    float d0, d1;
+    unpack2(d, d0, d1);
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r0) : "f"(d0));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r1) : "f"(d1));
+    return fma2(splat2(-2.0f), pack2(r0, r1), splat2(1.0f));
 }
 
 template <int H, bool FAST_TANH = false>

@@ -83,7 +83,7 @@ bool rollout_assisted_applies(const RolloutParams &p, int policy, bool streams);
 cudaError_t launch_rollout_assisted(RolloutParams &p, bool contracted, cudaStream_t s);
 // the deferred-restart kernel (large batches, no per-step streams), and whether a call is one it covers
 bool rollout_deferred_applies(const RolloutParams &p, int policy, bool streams);
-cudaError_t launch_rollout_deferred(RolloutParams &p, int policy, cudaStream_t s);
+cudaError_t launch_rollout_deferred(RolloutParams &p, int policy, bool contracted, cudaStream_t s);
 // the MLP policies (kinds 2, 4, 5, 7), canonical and contracted arithmetic; mode and shape as
 // chosen by launch_rollout_arith
 cudaError_t launch_rollout_networks(RolloutParams &p, int policy, int mode, int shape, cudaStream_t s);

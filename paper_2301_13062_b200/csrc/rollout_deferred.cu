@@ -23,8 +23,8 @@
 // the price is idle slots (about 7 % at K = 4 with the random policy's 22-step episodes) and a
 // ragged end.
 //
-// Scope: hashed actions, the shared linear policy or one linear policy per environment; canonical
-// arithmetic; with or without the episode step limit; per-step outputs either none or exactly the
+// Scope: hashed actions, the shared linear policy, the shared 4-16-2 network or one linear policy per
+// environment; either arithmetic; with or without the episode step limit; per-step outputs either none or exactly the
 // reward plane + done bitmask (the action bitmask and the trajectory are rows of global time that
 // half the lanes would have to touch every step). Everything else takes the general kernel.
 //
@@ -63,7 +63,7 @@ __device__ __forceinline__ void linear_action_pair(const f32x2 *w, const StatePa
     l1 = fma2(w[7], z.thd, l1);
     argmax_pair(l0, l1, sb0, sb1);
 }
-template <int H>
+template <int H, bool CONTRACT>
 __device__ __forceinline__ void mlp_action_pair(const f32x2 *w, const StatePair &z, uint32_t &sb0, uint32_t &sb1) {
     // w: W1[H][4], b1[H], W2[2][H], b2[2], as pairs
     const f32x2 *w1 = w, *b1 = w + 4 * H, *w2 = w + 5 * H, *b2 = w + 7 * H;
@@ -75,7 +75,7 @@ __device__ __forceinline__ void mlp_action_pair(const f32x2 *w, const StatePair 
         acc = fma2(w1[4 * j + 1], z.xd, acc);
         acc = fma2(w1[4 * j + 2], z.th, acc);
         acc = fma2(w1[4 * j + 3], z.thd, acc);
-        const f32x2 h = tanh_pair(acc);
+        const f32x2 h = CONTRACT ? tanh_contracted_pair(acc) : tanh_pair(acc);
         l0 = fma2(w2[j], h, l0);
         l1 = fma2(w2[H + j], h, l1);
     }
@@ -84,7 +84,7 @@ __device__ __forceinline__ void mlp_action_pair(const f32x2 *w, const StatePair 
 
 // Actions of both slots, in sign-bit form. SHORT: every time of the launch is below 2^16, where
 // fold16(t) == t.
-template <int POLICY, bool SHORT>
+template <int POLICY, bool SHORT, bool CONTRACT>
 __device__ __forceinline__ void deferred_actions(const RolloutParams &p, const FoldedKeys (&ka)[2],
                                                  const LinearW *own, const uint32_t (&t)[2], const StatePair &zz,
                                                  uint32_t &sb0, uint32_t &sb1) {
@@ -95,7 +95,7 @@ __device__ __forceinline__ void deferred_actions(const RolloutParams &p, const F
     } else if (POLICY == 1) {
         linear_action_pair(pairs, zz, sb0, sb1);
     } else if (POLICY == 2) {
-        mlp_action_pair<16>(pairs, zz, sb0, sb1);
+        mlp_action_pair<16, CONTRACT>(pairs, zz, sb0, sb1);
     } else {
         State a, b;
         unpack_states(zz, a, b);
@@ -107,6 +107,7 @@ __device__ __forceinline__ void deferred_actions(const RolloutParams &p, const F
 // POLICY: 0 hashed actions, 1 shared linear policy, 2 shared 4-16-2 network, 6 one linear policy per environment.
 // K: trips between restart passes. LIMIT: episodes are cut off after p.max_steps steps.
 // RD: the reward plane and the done bitmask are written (see the comment at reward_row).
+// CONTRACT: the contracted arithmetic (euler_step_contracted_pair, tanh_contracted_pair).
 // One CTA per SM is all the launch bounds ask for, which lets the assembler take the registers it
 // wants (77-96 instead of the 58-64 it settles for when left to aim at occupancy): the kernel is
 // bound by the float32 pipe, not by latency, and the extra registers hold the packed constants
@@ -116,7 +117,7 @@ __device__ __forceinline__ void deferred_actions(const RolloutParams &p, const F
 // (The network policy is the exception: its sixteen hidden units per slot are latency — exp2 and
 // reciprocal on the special-function pipe — that only more resident warps hide: 16,777,216 x
 // 200 takes 53.1 / 41.1 / 39.9 / 39.4 / 40.8 ms at 1 / 2 / 3 / 4 / 5 CTAs per SM.)
-template <int POLICY, int K, bool SHORT, bool LIMIT, bool RD>
+template <int POLICY, int K, bool SHORT, bool LIMIT, bool RD, bool CONTRACT>
 __global__ void __launch_bounds__(256, POLICY == 2 ? 4 : 1) rollout_deferred_kernel(const __grid_constant__ RolloutParams p) {
     const uint32_t lane = threadIdx.x & 31u;
     const int64_t task = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -262,9 +263,11 @@ __global__ void __launch_bounds__(256, POLICY == 2 ? 4 : 1) rollout_deferred_ker
         auto trip = [&](auto tail) {
             if (RD) reward_row(tail, row++);
             uint32_t sb0, sb1;
-            deferred_actions<POLICY, SHORT>(p, ka, own, t, zz, sb0, sb1);
+            deferred_actions<POLICY, SHORT, CONTRACT>(p, ka, own, t, zz, sb0, sb1);
             bool d0, d1;
-            euler_step_pair(zz, pack2(force_from_signbit(sb0), force_from_signbit(sb1)), d0, d1);
+            const f32x2 force = pack2(force_from_signbit(sb0), force_from_signbit(sb1));
+            if (CONTRACT) euler_step_contracted_pair(zz, force, d0, d1);
+            else euler_step_pair(zz, force, d0, d1);
             after_step(tail, 0, d0);
             after_step(tail, 1, d1);
         };
@@ -276,11 +279,13 @@ __global__ void __launch_bounds__(256, POLICY == 2 ? 4 : 1) rollout_deferred_ker
             // start state (|theta| <= 0.05), which is the packed step's domain.
             if (RD) reward_row(std::false_type{}, row++);
             uint32_t sb0, sb1;
-            deferred_actions<POLICY, SHORT>(p, ka, own, t, zz, sb0, sb1);
+            deferred_actions<POLICY, SHORT, CONTRACT>(p, ka, own, t, zz, sb0, sb1);
             State a, b;
             unpack_states(zz, a, b);
-            const bool d0 = euler_step<false>(a, force_from_signbit(sb0));
-            const bool d1 = euler_step<false>(b, force_from_signbit(sb1));
+            const bool d0 = CONTRACT ? euler_step_contracted<false>(a, force_from_signbit(sb0))
+                                     : euler_step<false>(a, force_from_signbit(sb0));
+            const bool d1 = CONTRACT ? euler_step_contracted<false>(b, force_from_signbit(sb1))
+                                     : euler_step<false>(b, force_from_signbit(sb1));
             zz = pack_states(a, b);
             after_step(std::true_type{}, 0, d0);
             after_step(std::true_type{}, 1, d1);
@@ -335,26 +340,34 @@ __global__ void __launch_bounds__(256, POLICY == 2 ? 4 : 1) rollout_deferred_ker
 }
 
 template <int POLICY, bool SHORT, bool LIMIT, bool RD>
-cudaError_t launch_k(RolloutParams &p, int k, cudaStream_t s) {
+cudaError_t launch_k(RolloutParams &p, int k, bool contracted, cudaStream_t s) {
     p.n_tasks = (p.n + 63) / 64;
     int64_t grid = (p.n_tasks + 7) / 8;
     if (grid > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    switch (k) {
-        case 2: rollout_deferred_kernel<POLICY, 2, SHORT, LIMIT, RD><<<(unsigned)grid, 256, 0, s>>>(p); break;
-        case 3: rollout_deferred_kernel<POLICY, 3, SHORT, LIMIT, RD><<<(unsigned)grid, 256, 0, s>>>(p); break;
-        case 6: rollout_deferred_kernel<POLICY, 6, SHORT, LIMIT, RD><<<(unsigned)grid, 256, 0, s>>>(p); break;
-        case 8: rollout_deferred_kernel<POLICY, 8, SHORT, LIMIT, RD><<<(unsigned)grid, 256, 0, s>>>(p); break;
-        default: rollout_deferred_kernel<POLICY, 4, SHORT, LIMIT, RD><<<(unsigned)grid, 256, 0, s>>>(p); break;
+    if (contracted) {  // the optional arithmetic comes at the default trip spacing only
+        if (POLICY == 2) rollout_deferred_kernel<POLICY, 2, SHORT, LIMIT, RD, true><<<(unsigned)grid, 256, 0, s>>>(p);
+        else rollout_deferred_kernel<POLICY, 6, SHORT, LIMIT, RD, true><<<(unsigned)grid, 256, 0, s>>>(p);
+    } else {
+        switch (k) {
+            case 2: rollout_deferred_kernel<POLICY, 2, SHORT, LIMIT, RD, false><<<(unsigned)grid, 256, 0, s>>>(p); break;
+            case 3: rollout_deferred_kernel<POLICY, 3, SHORT, LIMIT, RD, false><<<(unsigned)grid, 256, 0, s>>>(p); break;
+            case 6: rollout_deferred_kernel<POLICY, 6, SHORT, LIMIT, RD, false><<<(unsigned)grid, 256, 0, s>>>(p); break;
+            case 8: rollout_deferred_kernel<POLICY, 8, SHORT, LIMIT, RD, false><<<(unsigned)grid, 256, 0, s>>>(p); break;
+            default: rollout_deferred_kernel<POLICY, 4, SHORT, LIMIT, RD, false><<<(unsigned)grid, 256, 0, s>>>(p); break;
+        }
     }
     count_launch();
     return cudaGetLastError();
 }
 
 template <int POLICY, bool SHORT>
-cudaError_t launch_limit(RolloutParams &p, int k, cudaStream_t s) {
+cudaError_t launch_limit(RolloutParams &p, int k, bool contracted, cudaStream_t s) {
     const bool rd = p.reward_stream != nullptr;  // rollout_deferred_applies: then done_bits too, nothing else
-    if (p.max_steps) return rd ? launch_k<POLICY, SHORT, true, true>(p, k, s) : launch_k<POLICY, SHORT, true, false>(p, k, s);
-    return rd ? launch_k<POLICY, SHORT, false, true>(p, k, s) : launch_k<POLICY, SHORT, false, false>(p, k, s);
+    if (p.max_steps)
+        return rd ? launch_k<POLICY, SHORT, true, true>(p, k, contracted, s)
+                  : launch_k<POLICY, SHORT, true, false>(p, k, contracted, s);
+    return rd ? launch_k<POLICY, SHORT, false, true>(p, k, contracted, s)
+              : launch_k<POLICY, SHORT, false, false>(p, k, contracted, s);
 }
 
 }  // namespace
@@ -365,7 +378,7 @@ bool rollout_deferred_applies(const RolloutParams &p, int policy, bool streams) 
     return outputs_ok && !p.action_bits_in && !p.start_in && (policy == 0 || policy == 1 || policy == 2 || policy == 6);
 }
 
-cudaError_t launch_rollout_deferred(RolloutParams &p, int policy, cudaStream_t s) {
+cudaError_t launch_rollout_deferred(RolloutParams &p, int policy, bool contracted, cudaStream_t s) {
     // measured on 1,048,576 x 500 at K = 3 / 4 / 6 / 8: hashed actions (22-step episodes) 0.996 /
     // 0.987 / 0.965 / 0.987 ms, the linear policy (80-step episodes) 0.945 / 0.924 / 0.907 / 0.908 ms
     // The 4-16-2 network of config 5 ends its episodes after 9-10 steps, so waiting costs more and
@@ -379,10 +392,10 @@ cudaError_t launch_rollout_deferred(RolloutParams &p, int policy, cudaStream_t s
         for (int i = count - 1; i >= 0; --i) p.w[2 * i] = p.w[2 * i + 1] = p.w[i];
     }
     switch (policy) {
-        case 0: return short_times ? launch_limit<0, true>(p, k, s) : launch_limit<0, false>(p, k, s);
-        case 1: return launch_limit<1, false>(p, k, s);
-        case 2: return launch_limit<2, false>(p, k, s);
-        default: return launch_limit<6, false>(p, k, s);
+        case 0: return short_times ? launch_limit<0, true>(p, k, contracted, s) : launch_limit<0, false>(p, k, contracted, s);
+        case 1: return launch_limit<1, false>(p, k, contracted, s);
+        case 2: return launch_limit<2, false>(p, k, contracted, s);
+        default: return launch_limit<6, false>(p, k, contracted, s);
     }
 }
 

@@ -466,9 +466,10 @@ cudaError_t launch_pipe_rate(int kind, const float *seed, float *sink, int iters
 // count pseudo-random pairs of states from the domain the packed step is used on (|theta| <= 0.22)
 // and a little beyond what an episode visits in the other components; every pair is stepped by
 // euler_step_pair and, half by half, by euler_step<true>. out[0] += pairs whose eight new state
-// components or two termination flags differ in any bit, out[1] += pairs tested.
+// components or two termination flags differ in any bit, out[1] += pairs tested, out[2] += pairs
+// for which the contracted arithmetic's packed and scalar steps differ.
 __global__ void pair_selftest_kernel(unsigned long long count, uint32_t seed, unsigned long long *out) {
-    unsigned long long bad = 0, seen = 0;
+    unsigned long long bad = 0, bad_c = 0, seen = 0;
     const uint32_t s0 = salt(seed, 7u);
     for (unsigned long long k = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; k < count;
          k += (unsigned long long)gridDim.x * blockDim.x) {
@@ -502,14 +503,29 @@ __global__ void pair_selftest_kernel(unsigned long long count, uint32_t seed, un
                           pd0 == d0 && pd1 == d1;
         bad += !same;
         seen += 1;
+        // the same for the contracted arithmetic (a and b now hold the stepped states: step them again)
+        State ca = a, cb = b;
+        StatePair cz = pack_states(a, b);
+        bool qd0, qd1;
+        euler_step_contracted_pair(cz, pack2(fa, fb), qd0, qd1);
+        State qa, qb;
+        unpack_states(cz, qa, qb);
+        const bool e0 = euler_step_contracted<true>(ca, fa), e1 = euler_step_contracted<true>(cb, fb);
+        bad_c += !(__float_as_uint(qa.x) == __float_as_uint(ca.x) && __float_as_uint(qa.xd) == __float_as_uint(ca.xd) &&
+                   __float_as_uint(qa.th) == __float_as_uint(ca.th) && __float_as_uint(qa.thd) == __float_as_uint(ca.thd) &&
+                   __float_as_uint(qb.x) == __float_as_uint(cb.x) && __float_as_uint(qb.xd) == __float_as_uint(cb.xd) &&
+                   __float_as_uint(qb.th) == __float_as_uint(cb.th) && __float_as_uint(qb.thd) == __float_as_uint(cb.thd) &&
+                   qd0 == e0 && qd1 == e1);
     }
     for (int o = 16; o > 0; o >>= 1) {
         bad += __shfl_down_sync(0xffffffffu, bad, o);
+        bad_c += __shfl_down_sync(0xffffffffu, bad_c, o);
         seen += __shfl_down_sync(0xffffffffu, seen, o);
     }
     if ((threadIdx.x & 31) == 0) {
         if (bad) atomicAdd(out, bad);
         atomicAdd(out + 1, seen);
+        if (bad_c) atomicAdd(out + 2, bad_c);
     }
 }
 

@@ -76,6 +76,12 @@ def test_same_bits_as_the_general_kernel(cp, kind, n, T, t0, off, limit):
         got = run(cp, DEFERRED, k, **kw)
         for key in want:
             assert np.array_equal(want[key], got[key]), (key, k)
+    # the contracted arithmetic: its deferred form gives the bits of its general form
+    kw["arithmetic"] = cp.CP_ARITH_CONTRACTED
+    want_c, got_c = run(cp, GENERAL, 0, **kw), run(cp, DEFERRED, 0, **kw)
+    for key in want_c:
+        assert np.array_equal(want_c[key], got_c[key]), (key, "contracted")
+    assert n < 4000 or not np.array_equal(want_c["final_state"], want["final_state"])
 
 
 @pytest.mark.parametrize("kind", [0, 1, 2])

@@ -657,13 +657,13 @@ def test_packed_two_env_step_has_the_bits_of_the_scalar_step(cp):
     """2^30 pseudo-random state pairs through the packed float32 instructions and through the scalar
     step (which the ladder tests tie to the one-op kernels): no bit may differ. Guards against an
     assembler that contracts a packed multiply and add (CUDA 12.9 does where it can)."""
-    out = torch.zeros(2, dtype=torch.int64, device="cuda")
+    out = torch.zeros(3, dtype=torch.int64, device="cuda")
     for seed in (0, 1):
         cp.cp_selftest_pair(1 << 29, seed, out)
     torch.cuda.synchronize()
-    bad, pairs = (int(v) for v in out.cpu())
+    bad, pairs, bad_contracted = (int(v) for v in out.cpu())
     assert pairs == 1 << 30
-    assert bad == 0
+    assert bad == 0 and bad_contracted == 0
 
 
 def test_tame_state_division_equals_ieee_division_on_its_whole_domain(cp):
