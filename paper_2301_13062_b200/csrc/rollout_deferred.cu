@@ -384,7 +384,12 @@ cudaError_t launch_rollout_deferred(RolloutParams &p, int policy, bool contracte
     // The 4-16-2 network of config 5 ends its episodes after 9-10 steps, so waiting costs more and
     // a restart pass less (next to a 600-instruction trip): 16,777,216 x 200 takes 41.1 / 43.1 /
     // 47.3 / 48.9 ms at K = 2 / 3 / 4 / 6 (the general kernel: 43.2 ms).
-    const int k = g_tuning.rollout_defer > 0 ? g_tuning.rollout_defer : (policy == 2 ? 2 : 6);
+    // Short launches (chunked rollouts of a batch in place) pay the ragged end on every call, so
+    // the passes come closer together (us per step of 1,048,576 envs at K = 2 / 4 / 6, hashed
+    // actions: T = 16: 3.39 / 3.65 / 4.03, T = 64: 2.41 / 2.38 / 2.45, T = 256: 2.17 / 2.02 / 2.00;
+    // below 12 steps the general kernel is as fast or faster and keeps the call).
+    const int by_length = p.T < 48u ? 2 : p.T < 192u ? 4 : 6;
+    const int k = g_tuning.rollout_defer > 0 ? g_tuning.rollout_defer : (policy == 2 ? 2 : by_length);
     // the action hash folds the time's upper half into the lower one: nothing to do below 2^16
     const bool short_times = (uint64_t)p.t0 + p.T <= 65536u;
     if (policy == 1 || policy == 2) {  // every shared weight twice: one packed operand for both slots
