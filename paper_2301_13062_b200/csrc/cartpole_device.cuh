@@ -540,7 +540,7 @@ __device__ __forceinline__ uint32_t linear_action(const LinearW &p, const State 
 // reciprocal approximations (five instructions instead of the library routine's ~18). Small
 // arguments lose RELATIVE accuracy to the cancellation in 1 - (...), which a policy does not
 // feel: its logits depend on the absolute error, measured <= 2.4e-7 over every float32
-// (cp_selftest_tanh; the library tanhf: 1.2e-7). Saturates to +-1, NaN stays NaN.
+// (cp_selftest_tanh; tanh_canonical: 1.1e-7). Saturates to +-1, NaN stays NaN.
 __device__ __forceinline__ float tanh_contracted(float x) {
     float t, r;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(__fmul_rn(x, 2.885390043f)));  // 2 * log2(e)

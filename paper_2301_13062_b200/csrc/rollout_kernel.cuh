@@ -15,6 +15,13 @@
 // only synchronisation is __syncwarp() around a warp's own 192 bytes of shared memory in the
 // cooperative restart.
 //
+// Where a thread owns two environments (SHAPE 2) and the arithmetic is the canonical one, both
+// are stepped by the packed float32 instructions of sm_100a (euler_step_pair). Batches that fill
+// the chip mostly go to the deferred-restart kernel of rollout_deferred.cu instead; this
+// kernel keeps every call that one does not cover (action bit stream or trajectory written,
+// supplied actions or start states, the wider and deeper networks, very short launches, batches
+// too small to fill the chip) and is the form the others are compared with bit for bit.
+//
 // This header holds the kernel template and its dispatch; rollout_kernel.cu and
 // rollout_networks.cu instantiate it for the canonical (one rounding per op) arithmetic,
 // rollout_contracted.cu and rollout_networks_contracted.cu for the contracted arithmetic (the

@@ -273,9 +273,11 @@ cudaError_t launch_sincos_accuracy(uint32_t lo_bits, uint32_t hi_bits, unsigned 
     return cudaGetLastError();
 }
 
-// ---- self-test: absolute error of the two hyperbolic tangents against float64 ----
-// out[0] / out[1]: largest |tanh_contracted(v) - tanh(v)| / |tanhf(v) - tanh(v)| over the
-// float32 values with bit patterns in [lo, hi] and their negatives, in units of 1e-12.
+// ---- self-test: error of the hyperbolic tangents against float64 ----
+// Over the float32 values with bit patterns in [lo, hi] and their negatives. Largest absolute
+// error in units of 1e-12: out[0] tanh_contracted, out[1] the library's tanhf, out[2]
+// tanh_canonical; largest error in millionths of an ulp: out[3] tanh_canonical, out[4] the
+// library's; out[5] += values for which tanh_pair differs from tanh_canonical in any bit.
 __global__ void tanh_accuracy_kernel(uint32_t lo, uint32_t hi, unsigned long long *out) {
     double worst_fast = 0.0, worst_lib = 0.0, worst_own = 0.0, worst_own_ulp = 0.0, worst_lib_ulp = 0.0;
     unsigned long long pair_mismatch = 0;
@@ -331,7 +333,7 @@ cudaError_t launch_tanh_accuracy(uint32_t lo_bits, uint32_t hi_bits, unsigned lo
 // out[0]: bit patterns x (all 2^32) where div_mtot(x) != __fdiv_rn(x, 1.1f)
 // out[1]: patterns inside div_mtot_not_tiny's domain (+0, NaN, Inf, |x| >= 2^-100) where it differs
 // out[2]: patterns inside div_mtot_normal's domain (+0, NaN, 2^-100 <= |x| <= FLT_MAX) where it differs
-// out[3]: 24-bit inputs where start_from_bits differs from the three-operation definition
+// out[3]: 24-bit inputs where start_from_bits differs from the definition's three operations
 __global__ void arith_selftest_kernel(unsigned long long *out) {
     unsigned long long b0 = 0, b1 = 0, b2 = 0, b3 = 0;
     for (uint64_t k = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; k < (1ull << 32);
