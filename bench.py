@@ -30,31 +30,35 @@ sys.path.insert(0, ROOT)
 METRIC = "env_steps_per_sec"
 UNIT = "env-steps/s"
 SMS = 148
-# Work per env-step of each rollout variant, counted by ncu on 1,048,576 envs x 100 steps
-# (summaries under profiles/). "thread" = smsp__thread_inst_executed.sum / (N*T) of the
-# per-lane formulation (one env per thread, each lane restarts its own env; tuning
+# Work per env-step of each rollout variant, counted by ncu (summaries under profiles/).
+# "thread" = smsp__thread_inst_executed.sum / (N*T) of the per-lane formulation on 1,048,576 x 100 (one env per thread, each lane restarts its own env; tuning
 # rollout_ept=1 rollout_coop=2): the instructions an environment needs, none counted for
 # lanes that idle or help a neighbour — the algorithmic figure. "slot" = 32 *
 # smsp__inst_executed.sum / (N*T) of the kernel the library launches by default at this size
 # ("kernel"): the issue slots it really occupies; the deferred-restart kernel steps two
 # environments per packed float32 instruction, so its slots fall below the thread figure.
-# "fp32" = float32 multiply / add / fma lane operations of the method per env-step (40 in the
-# dynamics with the shortcuts of the kernels, 8 more for the linear policy).
+# "fp32" = float32 multiply / add / fma lane operations of the method per env-step (37 in the
+# dynamics with the shortcuts of the kernels, 22 in the contracted arithmetic, 0.2 for the start
+# states of the 4.5 % of env-steps that restart, 8 more for the linear policy).
 # COUNTED_AT = build.kernel_hash() of the sources these were captured from (a test compares it
 # with the current sources, so that the fractions cannot go stale unnoticed).
-COUNTED_AT = "unset"
+COUNTED_AT = "588158ac8a71c93e"
 ROLLOUT_OPS = {
-    "random": {"thread": 68.6, "slot": 82.6, "fp32": 40.0, "kernel": "rollout_deferred_kernel"},
-    "linear": {"thread": 73.8, "slot": 76.2, "fp32": 48.0, "kernel": "rollout_deferred_kernel"},
-    # here the default kernel's own thread count is below the per-lane formulation's (one running
-    # stream pointer per two envs instead of one per env), so it is the algorithmic one
-    "linear+streams": {"thread": 87.7, "slot": 87.8, "fp32": 48.0, "kernel": "rollout_kernel"},
-    "mlp": {"thread": 440.3, "slot": 464.4, "kernel": "rollout_kernel"},
-    "random+contracted": {"thread": 55.6, "slot": 68.6, "kernel": "rollout_kernel"},
+    # slots: 1,048,576 x 500 (the deferred kernel's ragged end makes them depend a little on T)
+    "random": {"thread": 65.6, "slot": 48.8, "fp32": 37.2, "kernel": "rollout_deferred_kernel"},
+    "linear": {"thread": 70.8, "slot": 41.3, "fp32": 45.2, "kernel": "rollout_deferred_kernel"},
+    # slots: 1,048,576 x 1,000 with the reward plane and the done bitmask
+    "linear+streams": {"thread": 88.9, "slot": 47.1, "fp32": 45.2, "kernel": "rollout_deferred_kernel"},
+    # slots: 2,097,152 x 200; both sides of the branch-free tanh are evaluated for every value
+    "mlp": {"thread": 210.7, "slot": 328.0, "kernel": "rollout_deferred_kernel"},
+    "random+contracted": {"thread": 55.6, "slot": 40.0, "fp32": 22.2, "kernel": "rollout_deferred_kernel"},
 }
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch in the same captures.
-ROLLOUT_DRAM_BYTES = {"random": 24.8e3, "linear": 24.6e3, "linear+streams": 381.1e6, "mlp": 21.8e3}
-STEP_DRAM_BYTES_16M = 568.2e6  # step_kernel at 16,777,216 envs, same kind of capture
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch in the same captures (the per-env
+# results stay in L2); with the per-step streams: bytes per env-step (4,517.6 MB for 1,048,576 x
+# 1,000; the algorithmic figure is 4.125), which scale with N*T.
+ROLLOUT_DRAM_BYTES = {"random": 55.8e3, "linear": 54.5e3, "mlp": 57.6e3, "random+contracted": 54.8e3}
+STREAM_DRAM_BYTES_PER_ENV_STEP = 4.3083
+STEP_DRAM_BYTES_16M = 567.3e6  # step_kernel at 16,777,216 envs, same kind of capture
 # Algorithmic HBM bytes per env-step of the step paths.
 LAST_TIMING: dict = {}  # median / best / worst of the per-iteration event times of the last timed() call
 STEP_BYTES = 37.0      # 16 in + 16 out + 4 reward + 1 done, hashed action
@@ -313,9 +317,9 @@ def main() -> None:
                 "peak": peak_inst / 1e12, "unit": "Tinst/s", "frac": rate * ops["thread"] / peak_inst,
                 "issue_slot_frac": rate * ops["slot"] / peak_inst,
                 "fp32_pipe_frac": rate * ops["fp32"] / peak_inst if "fp32" in ops else None,
-                "traffic": ROLLOUT_DRAM_BYTES.get(variant),
-                "traffic_note": "ncu dram bytes of one launch at 1,048,576 envs x 100 steps; the 8 B/env of "
-                                "per-env results stay in L2, stream outputs scale with N*T",
+                "traffic": (n * T * STREAM_DRAM_BYTES_PER_ENV_STEP if w.streams else ROLLOUT_DRAM_BYTES.get(variant)),
+                "traffic_note": "ncu dram bytes of one launch at 1,048,576 envs (the 8 B/env of per-env results stay "
+                                "in L2); with per-step streams the capture's bytes per env-step x N x T",
                 "thread_inst_per_env_step": ops["thread"], "issue_slots_per_env_step": ops["slot"],
                 "fp32_lane_ops_per_env_step": ops.get("fp32"),
                 "counted_at": COUNTED_AT,
