@@ -337,7 +337,7 @@ int cp_set_allocator(void *(*alloc)(size_t), void (*release)(void *));
  * few loop trips (per-step outputs none or reward plane + done bits; hashed actions, a linear
  * policy or the 4-16-2 network; otherwise the default); every choice gives the same bits), "rollout_defer" (loop trips between the restart
  * passes of that deferred form: 2, 3, 4, 6 or 8; 0 = default: 2, 4 or 6 by the number of steps,
- * 2 with the 4-16-2 network),
+ * 3 with the 4-16-2 network),
  * "rollout_ctas_per_sm" (0 = default: one 32*ept-environment task per warp and as many
  * CTAs as that takes; k > 0 = persistent grid of k CTAs per SM looping over tasks), "step_block"
  * (32..256, default 64), "step_vec_min_envs" (batches smaller than this use the one-env-per-thread
