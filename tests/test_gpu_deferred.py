@@ -85,8 +85,8 @@ def test_same_bits_as_the_general_kernel(cp, kind, n, T, t0, off, limit):
 
 
 @pytest.mark.parametrize("kind", [0, 1, 2])
-@pytest.mark.parametrize("limit", [0, 31])
-def test_chunks_from_a_callers_states(cp, kind, limit):
+@pytest.mark.parametrize("limit,streams", [(0, False), (31, False), (0, True), (13, True)])
+def test_chunks_from_a_callers_states(cp, kind, limit, streams):
     """States with angles far outside the polynomial range and running-episode lengths carried in
     and out, advanced in chunks of 1, 2, 7 and 40 steps: general and deferred kernels stay
     identical in the batch itself, the carried lengths and the per-chunk results."""
@@ -107,6 +107,9 @@ def test_chunks_from_a_callers_states(cp, kind, limit):
                 out = {"ep_return_sum": torch.zeros(n, device="cuda"),
                        "ep_count": torch.zeros(n, dtype=torch.int32, device="cuda"),
                        "totals": torch.zeros(2, dtype=torch.int64, device="cuda")}
+                if streams:  # the reward plane and the done bits of a chunk that starts from given states
+                    out["reward_stream"] = torch.full((T, n), -2.0, device="cuda")
+                    out["done_bits"] = torch.full((T, (n + 31) // 32), -1, dtype=torch.int32, device="cuda")
                 cp.cp_rollout_ex(T=T, state=st, ep_len=ep_len, policy=pol, max_episode_steps=limit, **out)
                 torch.cuda.synchronize()
                 log.append({k: v.cpu().numpy().copy() for k, v in out.items()})
