@@ -331,8 +331,9 @@ int cp_set_allocator(void *(*alloc)(size_t), void (*release)(void *));
  * and start state ahead into shared memory (hashed or supplied actions and hashed start
  * states; otherwise as 2), 2, 3 and 4 only with one environment per
  * thread; 0 = default: helper warps for up to ten warps of environments per SM, per lane for
- * other batches too small to fill the GPU (ahead for the smaller ones), deferred (5) for batches
- * that fill it where that form applies, by the warp otherwise;
+ * other batches too small to fill the GPU (ahead for the smaller ones), deferred (5) from one
+ * 64-environment warp per scheduler on (37,888 environments on 148 SMs) where that form applies,
+ * by the warp otherwise;
  * 5 = two environments per thread with a clock per environment and restarts deferred to every
  * few loop trips (per-step outputs none or reward plane + done bits; hashed actions, a linear
  * policy or the 4-16-2 network; otherwise the default); every choice gives the same bits), "rollout_defer" (loop trips between the restart
