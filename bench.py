@@ -414,7 +414,10 @@ def measure_paths(cp, inputs, torch, timed, peaks, peak_inst, args) -> dict:
     sink = torch.empty(cp.CP_CALIBRATE_THREADS_PER_SM * torch.cuda.get_device_properties(0).multi_processor_count,
                        device="cuda")
     calib = {"issue_peak_tinst_per_s": peak_inst / 1e12}
-    for name, kind, iters in (("ffma", 0, 20000), ("imad", 1, 20000), ("mufu_rcp", 2, 5000)):
+    # (kinds 3-7: the packed FFMA2 alone and half-and-half mixes, which show what shares a pipe with it)
+    for name, kind, iters in (("ffma", 0, 20000), ("imad", 1, 20000), ("mufu_rcp", 2, 5000), ("ffma2", 3, 20000),
+                              ("ffma2+ffma", 4, 20000), ("ffma2+imad", 5, 20000), ("ffma2+alu_x2", 6, 20000),
+                              ("ffma+imad", 7, 20000)):
         count = {"n": 0}
 
         def fn():
