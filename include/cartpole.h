@@ -343,8 +343,9 @@ int cp_set_allocator(void *(*alloc)(size_t), void (*release)(void *));
  * CTAs as that takes; k > 0 = persistent grid of k CTAs per SM looping over tasks), "step_block"
  * (32..256, default 64), "step_vec_min_envs" (batches smaller than this use the one-env-per-thread
  * step kernel even when the four-envs-per-thread vector form is possible; default 262144),
- * "step_pdl" (1 = default: step kernels are launched with programmatic stream serialization, so
- * that the action hashing of one step overlaps the tail of the step before it; 0 = plain launches).
+ * "step_pdl" (1 = default: the step kernels and the ladder's one-op kernels are launched with
+ * programmatic stream serialization, so that a launch is set up — and, in the fused step, the
+ * actions hashed — while the launch before it still runs; 0 = plain launches).
  * Returns CP_EINVAL for an unknown key or value. */
 int cp_tune(const char *key, int value);
 

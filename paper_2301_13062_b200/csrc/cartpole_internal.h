@@ -64,6 +64,8 @@ struct LaunchTuning {
     // 1: launch the step kernel with programmatic stream serialization, so that a launch's
     // memory-independent preamble overlaps the tail of the launch before it (same stream).
     // Measured per launch, 65,536 envs: 4.10 -> 2.38 us issued eagerly, 2.01 -> 1.46 us from a graph.
+    // The ladder's 46 one-op kernels are launched the same way (each waits for its predecessor
+    // before its first access): 16,777,216 envs 1.209 -> 1.106 ms per step, 4,194,304 envs 0.386 -> 0.295 ms.
     int step_pdl = 1;
 };
 extern LaunchTuning g_tuning;

@@ -53,7 +53,13 @@ __device__ __forceinline__ void store4(T *p, int64_t i, int cnt, bool vec, const
     }
 }
 
+// Every kernel may be launched with programmatic stream serialization (Launcher::go): it waits
+// for the launch before it — whose plane it reads — ahead of its first memory access, and lets the
+// launch after it be set up at once; that one waits the same way. (Without the launch attribute
+// both calls return immediately.)
 #define CP_EW_PROLOGUE                                                          \
+    cudaGridDependencySynchronize();                                            \
+    cudaTriggerProgrammaticLaunchCompletion();                                  \
     const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;     \
     if (i >= n) return;                                                         \
     const int cnt = (n - i) < 4 ? (int)(n - i) : 4;
@@ -184,29 +190,46 @@ struct Launcher {
     int64_t n;
     cudaStream_t s;
     unsigned grid() const { return (unsigned)(((n + 3) / 4 + 255) / 256); }
+    // One launch of the ladder. With g_tuning.step_pdl the launch may be set up while the one
+    // before it in the stream still runs (the kernels wait for it themselves): what an eager
+    // executor that issues one kernel per operation can do about launch latency without fusing.
+    template <typename... P, typename... A>
+    void go(void (*kernel)(P...), A... args) const {
+        if (!g_tuning.step_pdl) {
+            kernel<<<grid(), 256, 0, s>>>(args...);
+        } else {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(grid());
+            cfg.blockDim = dim3(256);
+            cfg.stream = s;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            cudaLaunchKernelEx(&cfg, kernel, P(args)...);
+        }
+        count_launch();
+    }
     template <class Op, typename TO>
     void gen(TO *out, Op op) const {
-        ew0<<<grid(), 256, 0, s>>>(n, aligned(out, 4 * sizeof(TO)), out, op);
-        count_launch();
+        go(ew0<Op, TO>, n, aligned(out, 4 * sizeof(TO)), out, op);
     }
     template <class Op, typename TO, typename TA>
     void un(TO *out, const TA *a, Op op) const {
         const bool v = aligned(out, 4 * sizeof(TO)) && aligned(a, 4 * sizeof(TA));
-        ew1<<<grid(), 256, 0, s>>>(n, v, out, a, op);
-        count_launch();
+        go(ew1<Op, TO, TA>, n, v, out, a, op);
     }
     template <class Op, typename TO, typename TA, typename TB>
     void bin(TO *out, const TA *a, const TB *b, Op op) const {
         const bool v = aligned(out, 4 * sizeof(TO)) && aligned(a, 4 * sizeof(TA)) && aligned(b, 4 * sizeof(TB));
-        ew2<<<grid(), 256, 0, s>>>(n, v, out, a, b, op);
-        count_launch();
+        go(ew2<Op, TO, TA, TB>, n, v, out, a, b, op);
     }
     template <class Op, typename TO, typename TA, typename TB, typename TC>
     void tri(TO *out, const TA *a, const TB *b, const TC *c, Op op) const {
         const bool v = aligned(out, 4 * sizeof(TO)) && aligned(a, 4 * sizeof(TA)) && aligned(b, 4 * sizeof(TB)) &&
                        aligned(c, 4 * sizeof(TC));
-        ew3<<<grid(), 256, 0, s>>>(n, v, out, a, b, c, op);
-        count_launch();
+        go(ew3<Op, TO, TA, TB, TC>, n, v, out, a, b, c, op);
     }
 };
 

@@ -204,6 +204,40 @@ def test_ladder_equals_fused_step_bitwise(cp, n):
     assert cp.cp_launch_count() - before == 3 * (46 + 45 + 2)
 
 
+@pytest.mark.parametrize("n", [1, 4099, 2_000_003])
+def test_ladder_chain_with_and_without_dependent_launches(cp, n):
+    """Twelve ladder steps back to back (46 launches each, every kernel reading the plane the
+    launch before it wrote, the two batches swapping roles after every step) give the bits of
+    twelve fused steps — with plain launches and with programmatic dependent launches, where a
+    kernel is set up while its predecessor still runs and waits for it itself."""
+    T, seed = 12, 4
+    a, b = alloc_planes(n), alloc_planes(n)
+    reward = torch.empty(n, dtype=torch.float32, device="cuda")
+    done = torch.empty(n, dtype=torch.uint8, device="cuda")
+    ws = torch.empty(cp.cp_unfused_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    ref = alloc_planes(n)
+    st = cp.cp_wrap(ref, n, seed)
+    cp.cp_fill_start(st)
+    cp.cp_step_repeat(st, T, reward, done)
+    torch.cuda.synchronize()
+    want, want_done = host(ref[:, :n]), host(done)
+    try:
+        for pdl in (0, 1):
+            cp.cp_tune("step_pdl", pdl)
+            sa, sb = cp.cp_wrap(a, n, seed), cp.cp_wrap(b, n, seed)
+            cp.cp_fill_start(sa)
+            done.fill_(7)
+            for _ in range(T // 2):
+                cp.cp_step_unfused(sa, None, sb, reward, done, ws)
+                cp.cp_step_unfused(sb, None, sa, reward, done, ws)
+            torch.cuda.synchronize()
+            assert sa.info()["t"] == T
+            assert np.array_equal(host(a[:, :n]).view(np.uint32), want.view(np.uint32)), pdl
+            assert np.array_equal(host(done), want_done), pdl
+    finally:
+        cp.cp_tune("step_pdl", 1)
+
+
 def test_ladder_argument_checks(cp):
     n = 100
     pin, pout = alloc_planes(n), alloc_planes(n)
