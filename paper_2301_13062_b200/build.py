@@ -22,8 +22,8 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcartpole.so")
 STAMP = os.path.join(HERE, "libcartpole.so.stamp")
 SOURCES = ["rollout_networks.cu", "rollout_networks_contracted.cu", "rollout_kernel.cu", "rollout_contracted.cu",
-           "rollout_assisted.cu", "rollout_deferred.cu", "capi.cu", "step_kernel.cu", "ladder_kernels.cu", "ladder_noalloc.cu"]
-HEADERS = ["cartpole_device.cuh", "cartpole_internal.h", "rollout_kernel.cuh", os.path.join("..", "..", "include", "cartpole.h")]
+           "rollout_assisted.cu", "rollout_deferred.cu", "rollout_deferred_networks.cu", "rollout_deferred_mlp64.cu", "capi.cu", "step_kernel.cu", "ladder_kernels.cu", "ladder_noalloc.cu"]
+HEADERS = ["cartpole_device.cuh", "cartpole_internal.h", "rollout_kernel.cuh", "rollout_deferred.cuh", os.path.join("..", "..", "include", "cartpole.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "--fmad=false",
@@ -51,7 +51,7 @@ def kernel_hash() -> str:
     """Hash of the files and flags that determine the instruction streams of the rollout and step
     kernels (bench.py records it beside the per-env-step instruction counts it was given)."""
     h = hashlib.sha256()
-    for name in ("cartpole_device.cuh", "rollout_kernel.cuh", "rollout_deferred.cu", "step_kernel.cu"):
+    for name in ("cartpole_device.cuh", "rollout_kernel.cuh", "rollout_deferred.cuh", "rollout_deferred.cu", "step_kernel.cu"):
         with open(os.path.join(CSRC, name), "rb") as f:
             h.update(name.encode() + b"\0" + f.read() + b"\0")
     h.update(" ".join(NVCC_FLAGS).encode())

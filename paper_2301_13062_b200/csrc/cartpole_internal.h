@@ -45,7 +45,9 @@ struct RolloutParams {
     const uint32_t *action_bits_in;  // [T][words] supplied actions or nullptr
     const float *start_in;           // [T][4][n] supplied start states or nullptr
     const float *env_weights;        // [10][n] one linear policy per env (policy kind 6) or nullptr
-    float w[450];  // largest policy: MLP with 64 hidden units, 7*64 + 2 floats
+    // largest policy: the network with 64 hidden units, 7*64 + 2 floats; twice the room, because the
+    // deferred-restart kernel reads every shared weight as a (w, w) pair
+    float w[900];
 };
 
 struct LaunchTuning {
@@ -55,7 +57,7 @@ struct LaunchTuning {
                                   // 3 per lane, computed ahead; 4 handed over by a producer warp;
                                   // 5 deferred (two envs per thread, own clock per env, restarts every few trips)
     int rollout_ctas_per_sm = 0;  // 0: one task per warp (non-persistent grid)
-    int rollout_defer = 0;        // deferred-restart kernel: trips between restart passes (0: 4; 2, 4 or 8)
+    int rollout_defer = 0;        // deferred-restart kernel: trips between restart passes (0: by horizon and policy)
     int step_block = 64;
     // Below this many envs the one-env-per-thread kernel is used: a small batch is latency-bound,
     // and four envs in sequence per thread take longer than four times as many threads
@@ -86,6 +88,7 @@ cudaError_t launch_rollout_assisted(RolloutParams &p, bool contracted, cudaStrea
 // the deferred-restart kernel (large batches, no per-step streams), and whether a call is one it covers
 bool rollout_deferred_applies(const RolloutParams &p, int policy, bool streams);
 cudaError_t launch_rollout_deferred(RolloutParams &p, int policy, bool contracted, cudaStream_t s);
+cudaError_t launch_rollout_deferred_wide(RolloutParams &p, int policy, bool contracted, cudaStream_t s);  // policies 4, 5, 7
 // the MLP policies (kinds 2, 4, 5, 7), canonical and contracted arithmetic; mode and shape as
 // chosen by launch_rollout_arith
 cudaError_t launch_rollout_networks(RolloutParams &p, int policy, int mode, int shape, cudaStream_t s);

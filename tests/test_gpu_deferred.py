@@ -1,6 +1,6 @@
 """GPU tests of the deferred-restart rollout kernel (two environments per thread stepped by packed
 float32 instructions, a clock per environment, restarts every K trips): it must produce the bits
-of the general rollout kernel for every call it covers — any trip spacing, ragged sizes, horizons
+of the general rollout kernel for every call it covers — every policy, any trip spacing, ragged sizes, horizons
 shorter than one block of trips, global times beyond 2^16, the episode step limit, steps carried
 in, caller-supplied states with angles outside the polynomial range — and the oracle's returns."""
 import numpy as np
@@ -13,6 +13,7 @@ pytestmark = pytest.mark.gpu
 
 torch = pytest.importorskip("torch")
 
+WIDE = (inputs.POLICY_MLP32, inputs.POLICY_MLP64, inputs.POLICY_MLP_DEEP)  # 4-32-2, 4-64-2, 4-16-16-2
 GENERAL = (2, 1)   # two envs per thread, restarts by the whole warp after every step
 DEFERRED = (2, 5)
 
@@ -45,6 +46,9 @@ def make_policy(cp, kind, n):
         return None, None
     if kind in (1, 2):
         w = inputs.policy_weights(kind, kind)
+        return cp.policy(kind, w), w
+    if kind in WIDE:  # weight draws for which the network uses both actions
+        w = inputs.policy_weights(kind, 7 if kind == inputs.POLICY_MLP_DEEP else 3)
         return cp.policy(kind, w), w
     w = inputs.per_env_linear_weights(n, 11)
     return cp.policy(cp.CP_POLICY_LINEAR_PER_ENV, torch.from_numpy(w).cuda()), w
@@ -82,6 +86,26 @@ def test_same_bits_as_the_general_kernel(cp, kind, n, T, t0, off, limit):
     for key in want_c:
         assert np.array_equal(want_c[key], got_c[key]), (key, "contracted")
     assert n < 4000 or not np.array_equal(want_c["final_state"], want["final_state"])
+
+
+@pytest.mark.parametrize("kind", WIDE)
+@pytest.mark.parametrize("n,T,t0,off", [(1, 1, 0, 0), (63, 2, 0, 5), (4099, 61, 3, 77), (70001, 120, 0, 0),
+                                        (20000, 90, 70000, 1 << 20)])
+def test_wider_and_deeper_networks_same_bits_as_the_general_kernel(cp, kind, n, T, t0, off):
+    """The deferred kernel covers these networks for the plain call (no step limit, no per-step
+    outputs), in both arithmetics; with a limit the call must still come out right (it takes the
+    general kernel)."""
+    pol, _ = make_policy(cp, kind, n)
+    for arith in (cp.CP_ARITH_EXACT, cp.CP_ARITH_CONTRACTED):
+        for limit in (0, 17):
+            kw = dict(n_envs=n, T=T, seed=8, t0=t0, env_offset=off, policy=pol, max_episode_steps=limit, arithmetic=arith)
+            want = run(cp, GENERAL, 0, **kw)
+            before = cp.cp_launch_count()
+            got = run(cp, DEFERRED, 0, **kw)
+            assert cp.cp_launch_count() - before == 1
+            for key in want:
+                assert np.array_equal(want[key], got[key]), (key, arith, limit)
+        assert want["ep_count"].max() > 0 or T < 8
 
 
 @pytest.mark.parametrize("kind", [0, 1, 2])
@@ -123,12 +147,12 @@ def test_chunks_from_a_callers_states(cp, kind, limit, streams):
     assert sum(int(c["ep_count"].sum()) for c in results["deferred"][0::2]) > n // 4
 
 
-@pytest.mark.parametrize("kind", [0, 1, 2, 6])
+@pytest.mark.parametrize("kind", [0, 1, 2, 6, *WIDE])
 def test_returns_against_the_oracle(cp, oracle, kind):
     n, T, seed = 50001, 300, 2
     pol, w = make_policy(cp, kind, n)
     r = run(cp, DEFERRED, 0, n_envs=n, T=T, seed=seed, policy=pol)
-    o = oracle.rollout(n, T, seed, {0: 0, 1: 1, 2: 2, 6: inputs.POLICY_LINEAR_PER_ENV}[kind], w, final_state=True,
+    o = oracle.rollout(n, T, seed, inputs.POLICY_LINEAR_PER_ENV if kind == 6 else kind, w, final_state=True,
                        min_gap=True, nthreads=8)
     excuse = (o["min_gap"] < 1e-5) if kind else None
     res = H.assert_returns_match(r["ep_return_sum"].view(np.float32), r["ep_count"], o["ep_return_sum"], o["ep_count"],
