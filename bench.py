@@ -42,7 +42,7 @@ SMS = 148
 # states of the 4.5 % of env-steps that restart, 8 more for the linear policy).
 # COUNTED_AT = build.kernel_hash() of the sources these were captured from (a test compares it
 # with the current sources, so that the fractions cannot go stale unnoticed).
-COUNTED_AT = "a9fef3c57faa7e14"
+COUNTED_AT = "03022f096a091510"
 ROLLOUT_OPS = {
     # slots: 1,048,576 x 500 (the deferred kernel's ragged end makes them depend a little on T)
     "random": {"thread": 65.6, "slot": 48.8, "fp32": 37.2, "kernel": "rollout_deferred_kernel"},
@@ -54,11 +54,11 @@ ROLLOUT_OPS = {
     "random+contracted": {"thread": 55.6, "slot": 40.0, "fp32": 22.2, "kernel": "rollout_deferred_kernel"},
 }
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch in the same captures (the per-env
-# results stay in L2); with the per-step streams: bytes per env-step (4,518.8 MB for 1,048,576 x
+# results stay in L2); with the per-step streams: bytes per env-step (4,518.5 MB for 1,048,576 x
 # 1,000; the algorithmic figure is 4.125), which scale with N*T.
-ROLLOUT_DRAM_BYTES = {"random": 56.1e3, "linear": 54.5e3, "mlp": 58.6e3, "random+contracted": 54.8e3}
-STREAM_DRAM_BYTES_PER_ENV_STEP = 4.3095
-STEP_DRAM_BYTES_16M = 567.6e6  # step_kernel at 16,777,216 envs, same kind of capture
+ROLLOUT_DRAM_BYTES = {"random": 55.6e3, "linear": 54.8e3, "mlp": 58.6e3, "random+contracted": 54.8e3}
+STREAM_DRAM_BYTES_PER_ENV_STEP = 4.3091
+STEP_DRAM_BYTES_16M = 566.8e6  # step_kernel at 16,777,216 envs, same kind of capture
 # Algorithmic HBM bytes per env-step of the step paths.
 LAST_TIMING: dict = {}  # median / best / worst of the per-iteration event times of the last timed() call
 STEP_BYTES = 37.0      # 16 in + 16 out + 4 reward + 1 done, hashed action
