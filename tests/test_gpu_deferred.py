@@ -109,12 +109,13 @@ def test_wider_and_deeper_networks_same_bits_as_the_general_kernel(cp, kind, n, 
 
 
 @pytest.mark.parametrize("kind", [0, 1, 2])
-@pytest.mark.parametrize("limit,streams", [(0, False), (31, False), (0, True), (13, True)])
-def test_chunks_from_a_callers_states(cp, kind, limit, streams):
+@pytest.mark.parametrize("limit,streams,n", [(0, False, 9001), (31, False, 9001), (0, True, 9001), (13, True, 9001),
+                                             (0, True, 9028), (13, True, 9028)])
+def test_chunks_from_a_callers_states(cp, kind, limit, streams, n):
     """States with angles far outside the polynomial range and running-episode lengths carried in
     and out, advanced in chunks of 1, 2, 7 and 40 steps: general and deferred kernels stay
     identical in the batch itself, the carried lengths and the per-chunk results."""
-    n, seed = 9001, 5
+    seed = 5
     z = np.concatenate([inputs.random_states(n // 3, seed=4, spread="wide"),
                         inputs.random_states(n // 3, seed=5, spread="live"),
                         inputs.random_states(n - 2 * (n // 3), seed=6, spread="edge")], axis=1)
@@ -166,7 +167,8 @@ def test_returns_against_the_oracle(cp, oracle, kind):
 
 @pytest.mark.parametrize("kind", [0, 1, 2, 6])
 @pytest.mark.parametrize("n,T,t0,limit", [(1, 3, 0, 0), (33, 40, 7, 0), (4099, 61, 0, 19), (70001, 120, 0, 0),
-                                          (20000, 90, 65530, 0)])
+                                          (20000, 90, 65530, 0), (4164, 1, 0, 0), (4164, 2, 5, 0), (8192, 37, 0, 7),
+                                          (66564, 250, 0, 0)])
 def test_reward_plane_and_done_bits_with_clocks_per_environment(cp, kind, n, T, t0, limit):
     """The deferred kernel writes the reward plane row by row and sets done bits by atomic OR from
     the restart pass: every word must equal the general kernel's, padding bits included."""

@@ -53,7 +53,7 @@ def check_plane_tails(g, n, name, allowed=None):
     g.check(name)
 
 
-SIZES = [1, 31, 33, 1025, 70001]
+SIZES = [1, 31, 33, 1025, 4164, 70001]
 
 
 @pytest.mark.parametrize("n", SIZES)
