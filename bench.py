@@ -43,15 +43,17 @@ SMS = 148
 # COUNTED_AT = build.kernel_hash() of the sources these were captured from (a test compares it
 # with the current sources, so that the fractions cannot go stale unnoticed).
 COUNTED_AT = "03022f096a091510"
+# pipe_busy: sm__pipe_fmaheavy_cycles_active (share of the launch's cycles) in the same captures — the
+# resource that bounds these kernels; it counts idle slots' arithmetic and the integer multiply-adds too.
 ROLLOUT_OPS = {
     # slots: 1,048,576 x 500 (the deferred kernel's ragged end makes them depend a little on T)
-    "random": {"thread": 65.6, "slot": 48.8, "fp32": 37.2, "kernel": "rollout_deferred_kernel"},
-    "linear": {"thread": 70.8, "slot": 41.3, "fp32": 45.2, "kernel": "rollout_deferred_kernel"},
+    "random": {"thread": 65.6, "slot": 48.8, "fp32": 37.2, "pipe_busy": 0.837, "kernel": "rollout_deferred_kernel"},
+    "linear": {"thread": 70.8, "slot": 41.3, "fp32": 45.2, "pipe_busy": 0.824, "kernel": "rollout_deferred_kernel"},
     # slots: 1,048,576 x 1,000 with the reward plane and the done bitmask
-    "linear+streams": {"thread": 88.9, "slot": 47.1, "fp32": 45.2, "kernel": "rollout_deferred_kernel"},
+    "linear+streams": {"thread": 88.9, "slot": 47.1, "fp32": 45.2, "pipe_busy": 0.776, "kernel": "rollout_deferred_kernel"},
     # slots: 2,097,152 x 200; both sides of the branch-free tanh are evaluated for every value
-    "mlp": {"thread": 210.7, "slot": 311.6, "kernel": "rollout_deferred_kernel"},
-    "random+contracted": {"thread": 55.6, "slot": 40.0, "fp32": 22.2, "kernel": "rollout_deferred_kernel"},
+    "mlp": {"thread": 210.7, "slot": 311.6, "pipe_busy": 0.742, "kernel": "rollout_deferred_kernel"},
+    "random+contracted": {"thread": 55.6, "slot": 40.0, "fp32": 22.2, "pipe_busy": 0.812, "kernel": "rollout_deferred_kernel"},
 }
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch in the same captures (the per-env
 # results stay in L2); with the per-step streams: bytes per env-step (4,518.5 MB for 1,048,576 x
@@ -322,13 +324,15 @@ def main() -> None:
                                 "in L2); with per-step streams the capture's bytes per env-step x N x T",
                 "thread_inst_per_env_step": ops["thread"], "issue_slots_per_env_step": ops["slot"],
                 "fp32_lane_ops_per_env_step": ops.get("fp32"),
+                "fp32_pipe_busy_ncu": ops.get("pipe_busy"),
                 "counted_at": COUNTED_AT,
                 "peak_source": f"148 SMs x 4 schedulers x 32 lanes x {peaks['sm_max_mhz']:.0f} MHz ({peaks['source']} max clock)",
                 "note": "frac counts instructions executed by active lanes only in the per-lane formulation (what "
                         "an environment needs); issue_slot_frac counts whole warp instructions x 32 of the kernel "
                         "launched (a packed float32 instruction serves two environments in one slot); "
                         "fp32_pipe_frac counts the float32 multiply/add/fma lane operations of the method "
-                        "against the same 128 lanes per SM and clock"}
+                        "against the same 128 lanes per SM and clock; fp32_pipe_busy_ncu is the share of cycles the "
+                        "profiler saw that pipe busy in the capture the counts come from (the kernel's bound)"}
     if w.streams:
         roofline["stream_write_gbs"] = n * T * 4.125 / (ms_per_step * 1e-3) / 1e9
         roofline["stream_write_frac_of_hbm"] = roofline["stream_write_gbs"] / peaks["hbm_gbs"]
