@@ -339,7 +339,7 @@ int cp_set_allocator(void *(*alloc)(size_t), void (*release)(void *));
  * policy or the 4-16-2 network; the wider and deeper networks without step limit and per-step
  * outputs; otherwise the default); every choice gives the same bits), "rollout_defer" (loop
  * trips between the restart passes of that deferred form: 2, 3, 4, 6 or 8; 0 = default: 2, 4 or
- * 6 by the number of steps, 3 with a network policy; the wider and deeper networks always use 3),
+ * 6 by the number of steps (8 for the shared linear policy from 384 steps on), 3 with a network policy; the wider and deeper networks always use 3),
  * "rollout_ctas_per_sm" (0 = default: one 32*ept-environment task per warp and as many
  * CTAs as that takes; k > 0 = persistent grid of k CTAs per SM looping over tasks), "step_block"
  * (32..256, default 64), "step_vec_min_envs" (batches smaller than this use the one-env-per-thread

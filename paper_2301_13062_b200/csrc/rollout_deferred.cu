@@ -24,7 +24,12 @@ cudaError_t launch_rollout_deferred(RolloutParams &p, int policy, bool contracte
     // the passes come closer together (us per step of 1,048,576 envs at K = 2 / 4 / 6, hashed
     // actions: T = 16: 3.39 / 3.65 / 4.03, T = 64: 2.41 / 2.38 / 2.45, T = 256: 2.17 / 2.02 / 2.00;
     // below 12 steps the general kernel is as fast or faster and keeps the call).
-    const int by_length = p.T < 48u ? 2 : p.T < 192u ? 4 : 6;
+    // The shared linear policy's 80-step episodes leave a pass little to do, so long launches
+    // space them further (with the reward plane and done bits, K = 4 / 6 / 8: 1,048,576 x 500
+    // 1.076 / 1.041 / 1.027 ms, 4,194,304 x 1,000 8.45 / 8.12 / 7.97 ms; without them 4,194,304 x
+    // 1,000 7.05 / 7.01 ms at K = 6 / 8; at 200 steps K = 6 is ahead, and so it is at every length
+    // with hashed actions: 4,194,304 x 1,000 with streams 9.11 / 8.57 / 8.90 ms).
+    const int by_length = p.T < 48u ? 2 : p.T < 192u ? 4 : (policy == 1 && p.T >= 384u) ? 8 : 6;
     const int k = g_tuning.rollout_defer > 0 ? g_tuning.rollout_defer : (is_network(policy) ? 3 : by_length);
     // the action hash folds the time's upper half into the lower one: nothing to do below 2^16
     const bool short_times = (uint64_t)p.t0 + p.T <= 65536u;
