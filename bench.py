@@ -42,25 +42,25 @@ SMS = 148
 # states of the 4.5 % of env-steps that restart, 8 more for the linear policy).
 # COUNTED_AT = build.kernel_hash() of the sources these were captured from (a test compares it
 # with the current sources, so that the fractions cannot go stale unnoticed).
-COUNTED_AT = "e8edd23c335814d8"
+COUNTED_AT = "24d7494f85ce7c00"
 # pipe_busy: sm__pipe_fmaheavy_cycles_active (share of the launch's cycles) in the same captures — the
 # resource that bounds these kernels; it counts idle slots' arithmetic and the integer multiply-adds too.
 ROLLOUT_OPS = {
     # slots: 1,048,576 x 500 (the deferred kernel's ragged end makes them depend a little on T)
-    "random": {"thread": 65.6, "slot": 48.8, "fp32": 37.2, "pipe_busy": 0.836, "kernel": "rollout_deferred_kernel"},
+    "random": {"thread": 65.6, "slot": 48.8, "fp32": 37.2, "pipe_busy": 0.837, "kernel": "rollout_deferred_kernel"},
     "linear": {"thread": 70.8, "slot": 40.8, "fp32": 45.2, "pipe_busy": 0.813, "kernel": "rollout_deferred_kernel"},
     # slots: 1,048,576 x 1,000 with the reward plane and the done bitmask
-    "linear+streams": {"thread": 88.9, "slot": 46.2, "fp32": 45.2, "pipe_busy": 0.805, "kernel": "rollout_deferred_kernel"},
+    "linear+streams": {"thread": 88.9, "slot": 46.2, "fp32": 45.2, "pipe_busy": 0.800, "kernel": "rollout_deferred_kernel"},
     # slots: 2,097,152 x 200; both sides of the branch-free tanh are evaluated for every value
-    "mlp": {"thread": 210.7, "slot": 311.6, "pipe_busy": 0.742, "kernel": "rollout_deferred_kernel"},
-    "random+contracted": {"thread": 55.6, "slot": 40.0, "fp32": 22.2, "pipe_busy": 0.810, "kernel": "rollout_deferred_kernel"},
+    "mlp": {"thread": 210.7, "slot": 311.6, "pipe_busy": 0.740, "kernel": "rollout_deferred_kernel"},
+    "random+contracted": {"thread": 55.6, "slot": 40.0, "fp32": 22.2, "pipe_busy": 0.813, "kernel": "rollout_deferred_kernel"},
 }
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch in the same captures (the per-env
-# results stay in L2); with the per-step streams: bytes per env-step (4,384.5 MB for 1,048,576 x
+# results stay in L2); with the per-step streams: bytes per env-step (4,385.6 MB for 1,048,576 x
 # 1,000; the algorithmic figure is 4.125), which scale with N*T; the launch that zeroes the done bit
 # plane before the rollout writes another 0.125 B per env-step.
-ROLLOUT_DRAM_BYTES = {"random": 55.8e3, "linear": 62.2e3, "mlp": 58.6e3, "random+contracted": 55.0e3}
-STREAM_DRAM_BYTES_PER_ENV_STEP = 4.1814
+ROLLOUT_DRAM_BYTES = {"random": 55.6e3, "linear": 62.2e3, "mlp": 58.6e3, "random+contracted": 54.8e3}
+STREAM_DRAM_BYTES_PER_ENV_STEP = 4.1825
 STEP_DRAM_BYTES_16M = 567.2e6  # step_kernel at 16,777,216 envs, same kind of capture
 # Algorithmic HBM bytes per env-step of the step paths.
 LAST_TIMING: dict = {}  # median / best / worst of the per-iteration event times of the last timed() call

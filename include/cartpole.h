@@ -127,8 +127,8 @@ typedef struct cp_returns {
     uint64_t *totals;      /* [2] += {sum of ep_return_sum, sum of ep_count}; caller zeroes before the call */
     float *reward_stream;  /* [T][n_envs] reward of every step (1.0f) */
     uint32_t *done_bits;   /* [T][ceil(n_envs/32)] bit (i%32) of word (i/32) = done of env i at that step; every
-                              word is written, the caller need not clear it (for batches that fill the GPU
-                              a small launch zeroes the plane before the rollout kernel sets its bits) */
+                              word is written, the caller need not clear it (long launches of batches that fill
+                              the GPU zero the plane with a small launch before the rollout kernel sets its bits) */
     uint32_t *action_bits; /* [T][ceil(n_envs/32)] same packing, the action taken */
     float *final_state;    /* [4][n_envs] state after the last step */
     float *trajectory;     /* [T][4][n_envs] state after every step, after any reset (validation aid) */

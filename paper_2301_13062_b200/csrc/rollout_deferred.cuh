@@ -123,6 +123,14 @@ __host__ __device__ constexpr bool is_network(int policy) { return policy == 2 |
 // 51.0, 103.8 -> 98.5, 72.4 -> 59.0 ms).
 __host__ __device__ constexpr bool is_wide_network(int policy) { return is_network(policy) && policy != 2; }
 
+// The done bit plane of a launch that sets its bits by atomic OR has to be zeroed first.
+// A warp that clears its own words inside the rollout writes 4 bytes into each of T separate
+// sectors; contiguous stores (clear_words_kernel) are far cheaper per byte but cost a launch. With
+// the reward plane and done bits, in-kernel against separate clearing (us per launch): 65,536 envs
+// x 64 steps 20.7 / 24.9, 1,048,576 x 64 168.8 / 173.2, x 192 455.1 / 454.9, linear policy x 384
+// 831.0 / 795.1, 4,194,304 x 1,000 8.45 / 8.12 ms.
+constexpr uint32_t kClearApartFrom = 192u;
+
 // Actions of both slots, in sign-bit form. SHORT: every time of the launch is below 2^16, where
 // fold16(t) == t.
 template <int POLICY, bool SHORT, bool CONTRACT>
@@ -211,14 +219,21 @@ __global__ void __launch_bounds__(256, is_network(POLICY) ? 4 : 1) rollout_defer
         // Per-step outputs although the environments run on clocks of their own (RD):
         //  * every step of every environment earns reward 1, so row r of the reward plane does not
         //    depend on any clock: the warp writes it for its 64 environments in trip r, as full lines;
-        //  * a done bit is rare. The bit plane is zeroed by a launch of its own before this one
-        //    (clear_words_kernel: contiguous 16-byte stores; a warp clearing its own two words of
-        //    every row — 4 bytes in each of T separate sectors — cost 0.41 ms of config 4's 8.46),
-        //    and an environment whose episode ended at step t sets its bit in row t - t0 with one
+        //  * a done bit is rare. The bit plane is zeroed first — for launches of kClearApartFrom
+        //    steps or more by a launch of its own before this one (clear_words_kernel: contiguous
+        //    16-byte stores), for shorter ones here, every warp its own two words of every row — and
+        //    an environment whose episode ended at step t sets its bit in row t - t0 with one
         //    atomic OR — in the restart pass, where its stopped clock still tells that time.
         const int64_t words = (p.n + 31) >> 5;
         const int64_t word0 = task * 2;
         float *rew_row = RD ? p.reward_stream + base + lane : nullptr;
+        if (RD && p.T < kClearApartFrom) {
+            for (uint32_t r = lane; r < p.T; r += 32u) {
+                if (word0 < words) p.done_bits[(int64_t)r * words + word0] = 0u;
+                if (word0 + 1 < words) p.done_bits[(int64_t)r * words + word0 + 1] = 0u;
+            }
+            __syncwarp();  // orders the clearing stores before any lane's later atomic on the same word
+        }
         const bool has0 = base + lane < p.n, has1 = base + 32 + lane < p.n;
         // CHECK: the row may lie beyond the last one (only the tail's trips can)
         auto reward_row = [&](auto check, uint32_t row) {
@@ -419,7 +434,7 @@ __global__ void __launch_bounds__(256, is_network(POLICY) ? 4 : 1) rollout_defer
     }
 }
 
-// Zeroes n 32-bit words (the done bit plane of a launch that sets its bits by atomic OR).
+// Zeroes n 32-bit words (see kClearApartFrom).
 __global__ void __launch_bounds__(256) clear_words_kernel(uint32_t *w, int64_t n) {
     const int64_t i = ((int64_t)blockIdx.x * 256 + threadIdx.x) * 4;
     if (i + 4 <= n && (reinterpret_cast<uintptr_t>(w) & 15u) == 0u) {
@@ -435,7 +450,7 @@ cudaError_t launch_k(RolloutParams &p, int k, bool contracted, cudaStream_t s) {
     p.n_tasks = (p.n + 63) / 64;
     int64_t grid = (p.n_tasks + 7) / 8;
     if (grid > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    if (RD) {
+    if (RD && p.T >= kClearApartFrom) {
         const int64_t n_words = (int64_t)p.T * ((p.n + 31) >> 5);
         const int64_t clear_grid = (n_words + 1023) / 1024;
         if (clear_grid > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
